@@ -1,0 +1,213 @@
+"""ctypes binding over the C ABI declared in include/ls.h.
+
+Argument marshalling only: every step of the path runs in the library's kernels.
+Functions carry the C names.  Tensors are torch tensors (device memory and streams
+come from torch); page tables and plan arrays are numpy.  The library must be built
+(`build.build_library`); loading fails loudly when it is missing -- there is no
+CPU fallback.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+LS_OK = 0
+LS_ERR_INVALID_ARG, LS_ERR_BAD_PAGE_TABLE, LS_ERR_UNSUPPORTED_SHAPE, LS_ERR_ALIGNMENT = -1, -2, -3, -4
+LS_ERR_WORKSPACE, LS_ERR_STALE, LS_ERR_CUDA, LS_ERR_TIMEOUT, LS_ERR_NONFINITE = -5, -6, -7, -8, -9
+LS_SHARD_CONTIGUOUS, LS_SHARD_CYCLIC, LS_SHARD_ZIGZAG = 0, 1, 2
+LS_WORKSPACE_FWD, LS_WORKSPACE_BWD = 0, 1
+
+
+class ls_pages_desc_t(C.Structure):
+    _fields_ = [("prefix_len", C.c_int64), ("page_size", C.c_int32), ("num_shards", C.c_int32),
+                ("shard_policy", C.c_int32), ("num_kv_heads", C.c_int32), ("dim_k", C.c_int32),
+                ("dim_v", C.c_int32), ("v_aliases_k", C.c_int32), ("reserved", C.c_int32),
+                ("num_phys_pages", C.c_int64), ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
+                ("k_stride_page", C.c_int64), ("k_stride_tok", C.c_int64), ("k_stride_head", C.c_int64),
+                ("v_stride_page", C.c_int64), ("v_stride_tok", C.c_int64), ("v_stride_head", C.c_int64)]
+
+
+class ls_attn_params_t(C.Structure):
+    _fields_ = [("R", C.c_int32), ("num_q_heads", C.c_int32), ("scale", C.c_float), ("flags", C.c_int32)]
+
+
+class LsError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (where, lib().ls_status_string(status).decode(), status))
+
+
+_LIB = None
+
+
+def lib():
+    """Loads (building first if the sources are newer) the shared library."""
+    global _LIB
+    if _LIB is None:
+        path = _build.build_library() if os.environ.get("LS_NO_BUILD") != "1" else _build.LIB
+        if not os.path.exists(path):
+            raise RuntimeError("libls_replay.so is missing: run paper_2607_14952_b200/build.py")
+        L = C.CDLL(path)
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        L.ls_prefix_pages_build.argtypes = [C.POINTER(ls_pages_desc_t), vp, C.POINTER(vp)]
+        L.ls_prefix_pages_export.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.ls_prefix_pages_checksum.argtypes = [vp, vp, C.POINTER(C.c_uint64), vp]
+        L.ls_prefix_pages_destroy.argtypes = [vp]
+        L.ls_replay_attn_workspace_bytes.argtypes = [vp, C.POINTER(ls_attn_params_t), C.c_int]
+        L.ls_replay_attn_workspace_bytes.restype = C.c_size_t
+        L.ls_replay_attn_fwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+        L.ls_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
+        L.ls_replay_attn_bwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                         C.c_size_t, vp, vp]
+        L.ls_status_string.argtypes = [C.c_int]
+        L.ls_status_string.restype = C.c_char_p
+        for f in ("ls_prefix_pages_build", "ls_prefix_pages_export", "ls_prefix_pages_checksum",
+                  "ls_prefix_pages_destroy", "ls_replay_attn_fwd", "ls_lse_merge", "ls_replay_attn_bwd"):
+            getattr(L, f).restype = C.c_int
+        _LIB = L
+    return _LIB
+
+
+def _check(status, where):
+    if status != LS_OK:
+        raise LsError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Pages:
+    """Owner of an ls_pages_t handle (and of references to the pool tensors)."""
+
+    def __init__(self, handle, desc, k_pool, v_pool):
+        self.handle, self.desc, self.k_pool, self.v_pool = handle, desc, k_pool, v_pool
+        self.num_logical_pages = (desc.prefix_len + desc.page_size - 1) // desc.page_size
+
+    def close(self):
+        if self.handle:
+            lib().ls_prefix_pages_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def ls_prefix_pages_build(prefix_len, page_size, num_shards, num_kv_heads, dim_k, dim_v, num_phys_pages,
+                          page_table=None, k_pool=None, v_pool=None, shard_policy=LS_SHARD_CONTIGUOUS,
+                          v_aliases_k=False):
+    """k_pool/v_pool: bf16 CUDA tensors [num_phys_pages, page_size, num_kv_heads, dim] (last dim dense) or
+    None for a host-only plan.  page_table: int32 numpy array or None (identity)."""
+    d = ls_pages_desc_t()
+    d.prefix_len, d.page_size, d.num_shards, d.shard_policy = prefix_len, page_size, num_shards, shard_policy
+    d.num_kv_heads, d.dim_k, d.dim_v, d.v_aliases_k = num_kv_heads, dim_k, dim_v, int(bool(v_aliases_k))
+    d.num_phys_pages = num_phys_pages
+    if k_pool is not None:
+        assert k_pool.dtype == torch.bfloat16 and k_pool.stride(-1) == 1
+        d.k_pool = k_pool.data_ptr()
+        d.k_stride_page, d.k_stride_tok, d.k_stride_head = k_pool.stride(0), k_pool.stride(1), k_pool.stride(2)
+        if v_pool is not None and not v_aliases_k:
+            assert v_pool.dtype == torch.bfloat16 and v_pool.stride(-1) == 1
+            d.v_pool = v_pool.data_ptr()
+            d.v_stride_page, d.v_stride_tok, d.v_stride_head = v_pool.stride(0), v_pool.stride(1), v_pool.stride(2)
+    tbl = None
+    if page_table is not None:
+        tbl = np.ascontiguousarray(page_table, dtype=np.int32)
+    out = C.c_void_p()
+    st = lib().ls_prefix_pages_build(C.byref(d), None if tbl is None else tbl.ctypes.data_as(C.c_void_p), C.byref(out))
+    _check(st, "ls_prefix_pages_build")
+    return Pages(out, d, k_pool, v_pool)
+
+
+def ls_prefix_pages_export(pages):
+    Np, S = pages.num_logical_pages, pages.desc.num_shards
+    table = np.zeros(Np, np.int32)
+    owner = np.zeros(Np, np.int32)
+    offs = np.zeros(S + 1, np.int64)
+    order = np.zeros(Np, np.int32)
+    toks = np.zeros(S, np.int64)
+    p = lambda a: a.ctypes.data_as(C.c_void_p)
+    _check(lib().ls_prefix_pages_export(pages.handle, p(table), p(owner), p(offs), p(order), p(toks)),
+           "ls_prefix_pages_export")
+    return dict(page_table=table, shard_of_page=owner, shard_page_offset=offs, shard_logical_pages=order,
+                shard_tokens=toks)
+
+
+def ls_prefix_pages_checksum(pages):
+    scratch = torch.zeros(1, dtype=torch.int64, device=pages.k_pool.device)
+    out = C.c_uint64(0)
+    _check(lib().ls_prefix_pages_checksum(pages.handle, _ptr(scratch), C.byref(out), _stream()),
+           "ls_prefix_pages_checksum")
+    return int(out.value)
+
+
+def _params(R, Hq, scale):
+    return ls_attn_params_t(R, Hq, float(scale), 0)
+
+
+def ls_replay_attn_workspace_bytes(pages, R, Hq, scale, which):
+    prm = _params(R, Hq, scale)
+    return int(lib().ls_replay_attn_workspace_bytes(pages.handle, C.byref(prm), which))
+
+
+def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=None, status=None):
+    """Returns (o_part [(S+1),R,Hq,Dv] fp32, lse_part [(S+1),R,Hq] fp32)."""
+    R, Hq, _ = q.shape
+    S, Dv = pages.desc.num_shards, pages.desc.dim_v
+    if o_part is None:
+        o_part = torch.empty((S + 1, R, Hq, Dv), dtype=torch.float32, device=q.device)
+    if lse_part is None:
+        lse_part = torch.empty((S + 1, R, Hq), dtype=torch.float32, device=q.device)
+    prm = _params(R, Hq, scale)
+    st = lib().ls_replay_attn_fwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_part),
+                                  _ptr(lse_part), None, 0, _ptr(status), _stream())
+    _check(st, "ls_replay_attn_fwd")
+    return o_part, lse_part
+
+
+def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=True, want_f32=True):
+    """o_part [parts, ..., Dv] fp32, lse_part [parts, ...] fp32 -> (o_bf16, o_f32, lse)."""
+    parts, dv = o_part.shape[0], o_part.shape[-1]
+    rows = lse_part[0].numel()
+    shape = tuple(o_part.shape[1:])
+    if o_bf16 is None and want_bf16:
+        o_bf16 = torch.empty(shape, dtype=torch.bfloat16, device=o_part.device)
+    if o_f32 is None and want_f32:
+        o_f32 = torch.empty(shape, dtype=torch.float32, device=o_part.device)
+    if lse is None:
+        lse = torch.empty(shape[:-1], dtype=torch.float32, device=o_part.device)
+    st = lib().ls_lse_merge(parts, rows, dv, _ptr(o_part), _ptr(lse_part), _ptr(o_bf16), _ptr(o_f32), _ptr(lse),
+                            _stream())
+    _check(st, "ls_lse_merge")
+    return o_bf16, o_f32, lse
+
+
+def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspace=None, dq=None, dk_resp=None,
+                       dv_resp=None, status=None):
+    """Returns (dq, dk_resp, dv_resp) in bf16."""
+    R, Hq, _ = q.shape
+    if workspace is None:
+        nbytes = ls_replay_attn_workspace_bytes(pages, R, Hq, scale, LS_WORKSPACE_BWD)
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk_resp is None:
+        dk_resp = torch.empty_like(k_resp)
+    if dv_resp is None:
+        dv_resp = torch.empty_like(v_resp)
+    prm = _params(R, Hq, scale)
+    st = lib().ls_replay_attn_bwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_f32),
+                                  _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk_resp), _ptr(dv_resp), _ptr(workspace),
+                                  workspace.numel(), _ptr(status), _stream())
+    _check(st, "ls_replay_attn_bwd")
+    return dq, dk_resp, dv_resp

@@ -1,0 +1,60 @@
+// Host-side internals shared by the translation units of the library.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <vector>
+
+#include "ls.h"
+
+namespace ls {
+
+constexpr int kNumBoxSizes = 4;               // token extents of the TMA boxes we encode
+constexpr int kBoxTok[kNumBoxSizes] = {16, 32, 64, 128};
+
+inline int box_index(int tok) { return tok == 16 ? 0 : tok == 32 ? 1 : tok == 64 ? 2 : 3; }
+
+// TMA descriptors of one bf16 pool viewed as (d, token, head, page); [box][0] covers a
+// full page, [box][1] the partially filled last logical page (tokens past the valid
+// count read as zero).
+struct PoolMaps {
+  CUtensorMap full[kNumBoxSizes];
+  CUtensorMap tail[kNumBoxSizes];
+};
+
+}  // namespace ls
+
+struct ls_pages {
+  ls_pages_desc_t desc;
+  int64_t num_logical_pages;   // Np
+  int32_t last_valid;          // valid tokens of the last logical page (0 when P = 0)
+  std::vector<int32_t> page_table;            // [Np] logical -> physical
+  std::vector<int32_t> shard_of_page;         // [Np]
+  std::vector<int64_t> shard_page_offset;     // [S+1]
+  std::vector<int32_t> shard_logical_pages;   // [Np] shard-local order
+  std::vector<int32_t> shard_phys_pages;      // [Np] physical ids in shard-local order
+  std::vector<int64_t> shard_tokens;          // [S]
+  // per shard: position (in its page list) of the global last logical page, or -1
+  std::vector<int32_t> shard_tail_slot;       // [S]
+
+  bool on_device;
+  int device;
+  int32_t* d_shard_phys_pages;   // [Np]
+  int32_t* d_shard_page_offset;  // [S+1]
+  int32_t* d_shard_tail_slot;    // [S]
+  int64_t* d_shard_tokens;       // [S]
+  int32_t* d_page_table;         // [Np]
+  ls::PoolMaps k_maps, v_maps;
+};
+
+namespace ls {
+
+// Encodes a rank-4 bf16 tensor map (d, token, head, page) with a 128-byte swizzle and a
+// box of 64 channels x box_tok tokens.  Strides in elements.  Returns LS_OK or an error.
+ls_status_t encode_map(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok,
+                       int64_t dim_head, int64_t dim_page, int64_t stride_tok, int64_t stride_head,
+                       int64_t stride_page, int box_tok);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace ls

@@ -1,0 +1,177 @@
+"""Glue for the GPU parity tests: runs the CUDA path through the C-ABI binding and the
+fp64 oracle on the same seeded bytes, and compares them.  Not a test module itself."""
+import numpy as np
+import torch
+
+from oracle import attention as oa
+from oracle import pages as op
+from paper_2607_14952_b200 import binding as B
+from paper_2607_14952_b200 import workloads as W
+
+# Tolerances (the benchmark spec): max abs error 2e-2 on O/dQ/dK/dV, 1e-3 on LSE.  Because the
+# outputs themselves are ~1e-3 at long prefixes, a relative row-wise gate is applied too:
+# ||gpu - oracle||_2 <= REL * ||oracle||_2 + FLOOR * sqrt(D).
+ABS_TOL = 2e-2
+LSE_TOL = 1e-3
+REL = 1e-2
+FLOOR = 1e-5
+
+
+class Case:
+    """One prefix resident on the GPU plus the handles both sides need."""
+
+    def __init__(self, cfg, device="cuda", policy=B.LS_SHARD_CONTIGUOUS, extra_phys_pages=0):
+        self.cfg = cfg
+        self.device = device
+        self.k_pool, self.v_pool, self.table = W.make_prefix(cfg, device, extra_phys_pages)
+        self.pages = B.ls_prefix_pages_build(
+            cfg.P, cfg.page_size, cfg.num_shards, cfg.Hkv, cfg.Dk, cfg.Dv, self.k_pool.shape[0],
+            page_table=self.table, k_pool=self.k_pool, v_pool=None if cfg.v_aliases_k else self.v_pool,
+            shard_policy=policy, v_aliases_k=cfg.v_aliases_k)
+        self.policy = policy
+        self._host = {}
+
+    def member(self, m, cycle=0):
+        return W.make_member(self.cfg, m, self.device, cycle)
+
+    # ---- host copies for the oracle (bf16 bit patterns, one KV head at a time)
+    def host_pool(self, kv):
+        if kv not in self._host:
+            k = W.bf16_bits(self.k_pool[:, :, kv:kv + 1, :])
+            v = k if self.cfg.v_aliases_k else W.bf16_bits(self.v_pool[:, :, kv:kv + 1, :])
+            self._host[kv] = (k, v)
+        return self._host[kv]
+
+    def forward(self, q, k_resp, v_resp):
+        o_part, lse_part = B.ls_replay_attn_fwd(self.pages, q, k_resp, v_resp, self.cfg.scale)
+        o_bf16, o_f32, lse = B.ls_lse_merge(o_part, lse_part)
+        return o_part, lse_part, o_bf16, o_f32, lse
+
+    def backward(self, q, k_resp, v_resp, o_f32, lse, d_o):
+        return B.ls_replay_attn_bwd(self.pages, q, k_resp, v_resp, o_f32, lse, d_o, self.cfg.scale)
+
+    # ---- oracle on a set of (t, h) rows of one KV group
+    def oracle_rows(self, kv, t_rows, heads, q, k_resp, v_resp, d_o=None):
+        cfg = self.cfg
+        kp, vp = self.host_pool(kv)
+        qr = W.bf16_bits(q[t_rows, heads])
+        kr = W.bf16_bits(k_resp[:, kv:kv + 1])
+        vr = W.bf16_bits(v_resp[:, kv:kv + 1])
+        args = (qr, np.asarray(t_rows), 0, kp, vp, self.table, cfg.P, cfg.page_size, kr, vr, float(np.float32(cfg.scale)))
+        if d_o is None:
+            o, lse, _ = oa.forward_rows(*args)
+            return o, lse
+        return oa.backward_rows(*args, W.bf16_bits(d_o[t_rows, heads]))
+
+
+def rel_gate(gpu, ref, d):
+    """Row-wise relative L2 gate; returns the worst ratio err / allowed (<= 1 passes)."""
+    gpu = np.asarray(gpu, np.float64).reshape(-1, d)
+    ref = np.asarray(ref, np.float64).reshape(-1, d)
+    err = np.linalg.norm(gpu - ref, axis=1)
+    allowed = REL * np.linalg.norm(ref, axis=1) + FLOOR * np.sqrt(d)
+    return float((err / allowed).max())
+
+
+def f64(t):
+    return t.detach().double().cpu().numpy()
+
+
+def all_rows_of_group(cfg, kv):
+    g = cfg.Hq // cfg.Hkv
+    t = np.repeat(np.arange(cfg.R), g)
+    h = np.tile(np.arange(kv * g, (kv + 1) * g), cfg.R)
+    return t, h
+
+
+def sampled_rows(cfg, kv, tail=16, n_random=32, seed=0, extra=()):
+    """Rows {0,127,128,R/2,R-1} and the last `tail` rows for every head of the group, plus
+    seeded random (t, h) pairs and any extra pairs (needle rows) that fall in the group."""
+    g = cfg.Hq // cfg.Hkv
+    heads = list(range(kv * g, (kv + 1) * g))
+    ts = sorted({0, min(127, cfg.R - 1), min(128, cfg.R - 1), cfg.R // 2, cfg.R - 1} | set(range(max(0, cfg.R - tail), cfg.R)))
+    pairs = {(t, h) for t in ts for h in heads}
+    rng = np.random.default_rng(seed + 17 * kv)
+    for _ in range(n_random):
+        pairs.add((int(rng.integers(cfg.R)), int(rng.choice(heads))))
+    for t, h in extra:
+        if h in heads:
+            pairs.add((t, h))
+    pairs = sorted(pairs)
+    return np.array([p[0] for p in pairs]), np.array([p[1] for p in pairs])
+
+
+def check_forward(case, member=0, kv_groups=None, full=True, per_shard=True, extra_rows=()):
+    """Forward + merge parity.  Returns the tensors for reuse by the backward check."""
+    cfg = case.cfg
+    q, k_resp, v_resp, d_o = case.member(member)
+    o_part, lse_part, o_bf16, o_f32, lse = case.forward(q, k_resp, v_resp)
+    torch.cuda.synchronize()
+    report = {}
+    for kv in (range(cfg.Hkv) if kv_groups is None else kv_groups):
+        t_rows, heads = all_rows_of_group(cfg, kv) if full else sampled_rows(cfg, kv, extra=extra_rows)
+        o_ref, lse_ref = case.oracle_rows(kv, t_rows, heads, q, k_resp, v_resp)
+        g_lse = f64(lse[t_rows, heads])
+        g_o32 = f64(o_f32[t_rows, heads])
+        g_o16 = f64(o_bf16[t_rows, heads])
+        assert np.isfinite(g_lse).all() and np.isfinite(g_o32).all()
+        e_lse = np.abs(g_lse - lse_ref).max()
+        e_o = np.abs(g_o16 - o_ref).max()
+        r_o = rel_gate(g_o32, o_ref, cfg.Dv)
+        report[kv] = (e_lse, e_o, r_o)
+        assert e_lse <= LSE_TOL, ("LSE", kv, e_lse)
+        assert e_o <= ABS_TOL, ("O abs", kv, e_o)
+        assert r_o <= 1.0, ("O rel", kv, r_o)
+        if per_shard:
+            # every partial against Eq. qwen-local-attn evaluated on that shard's positions
+            kp, vp = case.host_pool(kv)
+            pos = op.shard_positions(cfg.P, cfg.page_size, cfg.num_shards,
+                                     {B.LS_SHARD_CONTIGUOUS: op.CONTIGUOUS, B.LS_SHARD_CYCLIC: op.CYCLIC,
+                                      B.LS_SHARD_ZIGZAG: op.ZIGZAG}[case.policy])
+            qr = W.bf16_bits(q[t_rows, heads])
+            for s in range(cfg.num_shards + 1):
+                if s < cfg.num_shards:
+                    po, pl = oa.local_attention(qr, 0, kp, vp, case.table, cfg.page_size, pos[s],
+                                                float(np.float32(cfg.scale)), dv=cfg.Dv)
+                else:
+                    po, pl = oa.local_attention_response(qr, t_rows, 0, W.bf16_bits(k_resp[:, kv:kv + 1]),
+                                                         W.bf16_bits(v_resp[:, kv:kv + 1]),
+                                                         float(np.float32(cfg.scale)))
+                gl = f64(lse_part[s][t_rows, heads])
+                go = f64(o_part[s][t_rows, heads])
+                fin = np.isfinite(pl)
+                assert np.array_equal(np.isfinite(gl), fin), ("empty partial", s)
+                if fin.any():
+                    assert np.abs(gl[fin] - pl[fin]).max() <= LSE_TOL, ("partial LSE", s)
+                    assert rel_gate(go[fin], po[fin], cfg.Dv) <= 1.0, ("partial O", s)
+                assert (go[~fin] == 0).all()
+    return dict(q=q, k_resp=k_resp, v_resp=v_resp, d_o=d_o, o_f32=o_f32, lse=lse, o_part=o_part,
+                lse_part=lse_part, o_bf16=o_bf16, report=report)
+
+
+def check_backward(case, fw, kv_groups=None, full=True, tail=16, extra_rows=()):
+    """Backward parity for dQ on the row set and for dK/dV on the response keys whose
+    contributing rows are all inside the set (all keys when full, the last `tail` otherwise)."""
+    cfg = case.cfg
+    q, k_resp, v_resp, d_o = fw["q"], fw["k_resp"], fw["v_resp"], fw["d_o"]
+    dq, dk, dv = case.backward(q, k_resp, v_resp, fw["o_f32"], fw["lse"], d_o)
+    torch.cuda.synchronize()
+    report = {}
+    for kv in (range(cfg.Hkv) if kv_groups is None else kv_groups):
+        t_rows, heads = all_rows_of_group(cfg, kv) if full else sampled_rows(cfg, kv, tail=tail, extra=extra_rows)
+        _, _, dq_ref, dk_ref, dv_ref = case.oracle_rows(kv, t_rows, heads, q, k_resp, v_resp, d_o)
+        g_dq = f64(dq[t_rows, heads])
+        assert np.isfinite(g_dq).all()
+        e_dq = np.abs(g_dq - dq_ref).max()
+        # bf16 output rounding adds up to 2^-9 relative per element on top of REL
+        r_dq = rel_gate(g_dq, dq_ref, cfg.Dk)
+        j0 = 0 if full else max(0, cfg.R - tail)
+        g_dk, g_dv = f64(dk[j0:, kv]), f64(dv[j0:, kv])
+        e_dk = np.abs(g_dk - dk_ref[j0:]).max()
+        e_dv = np.abs(g_dv - dv_ref[j0:]).max()
+        r_dk = rel_gate(g_dk, dk_ref[j0:], cfg.Dk)
+        r_dv = rel_gate(g_dv, dv_ref[j0:], cfg.Dv)
+        report[kv] = (e_dq, r_dq, e_dk, r_dk, e_dv, r_dv)
+        assert e_dq <= ABS_TOL and e_dk <= ABS_TOL and e_dv <= ABS_TOL, report[kv]
+        assert r_dq <= 1.0 and r_dk <= 1.0 and r_dv <= 1.0, report[kv]
+    return dict(dq=dq, dk=dk, dv=dv, report=report)

@@ -1,0 +1,42 @@
+"""ls_lse_merge against the oracle's merge (Eq. qwen-lse-parts, Eq. qwen-global-attn)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as oa
+from paper_2607_14952_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("parts", [1, 2, 5, 9, 33])
+@pytest.mark.parametrize("dv", [128, 256, 512])
+def test_merge_matches_oracle(parts, dv):
+    g = torch.Generator(device="cuda").manual_seed(parts * 1000 + dv)
+    rows = 1000 + parts                     # not a multiple of the warps per block
+    o = torch.randn(parts, rows, dv, generator=g, device="cuda")
+    l = torch.randn(parts, rows, generator=g, device="cuda") * 20.0          # spread of ~60 between partials
+    if parts > 1:
+        l[1, ::3] = -float("inf")           # empty partials
+        o[1, ::3] = 0.0
+    o_bf16, o_f32, lse = B.ls_lse_merge(o, l)
+    torch.cuda.synchronize()
+    ro, rl = oa.merge(o.double().cpu().numpy(), l.double().cpu().numpy())
+    assert np.abs(lse.double().cpu().numpy() - rl).max() < 1e-4
+    assert np.abs(o_f32.double().cpu().numpy() - ro).max() < 1e-4
+    assert np.abs(o_bf16.double().cpu().numpy() - ro).max() < 2e-2
+    assert torch.equal(o_f32.to(torch.bfloat16), o_bf16)
+
+
+def test_merge_all_empty_and_dominant_partial():
+    o = torch.zeros(3, 8, 128, device="cuda")
+    l = torch.full((3, 8), -float("inf"), device="cuda")
+    l[2, 4:] = 64.0
+    o[2, 4:] = 3.0
+    l[0, 4:] = 15.0                        # e^{-49} relative weight: vanishes without NaN
+    o[0, 4:] = -7.0
+    _, o_f32, lse = B.ls_lse_merge(o, l)
+    torch.cuda.synchronize()
+    assert torch.isinf(lse[:4]).all() and (lse[:4] < 0).all() and (o_f32[:4] == 0).all()
+    assert torch.allclose(lse[4:], torch.full_like(lse[4:], 64.0)) and torch.allclose(o_f32[4:], torch.full_like(o_f32[4:], 3.0))
+    assert torch.isfinite(o_f32).all()
