@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the replay-attention hot path (forward + merge + backward of one response
+against a resident paged prefix) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload p2m] [--impl reference]
+
+One "step" = one group member replayed against the resident prefix: ls_replay_attn_fwd,
+ls_lse_merge, ls_replay_attn_bwd.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun)
+every rank holds its own replica of the prefix and replays different members: no
+collective on the data path, weak scaling.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_14952_b200 import workloads as W  # noqa: E402
+
+METRIC = "replay_attn_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+
+
+def algorithmic_flops(cfg):
+    """Forward 2(Dk+Dv) per visible (query, key) pair; backward 2(2Dk+Dv) on a prefix key (the
+    prefix dK/dV products are not part of the method) and 2(3Dk+2Dv) on a response key."""
+    pre = cfg.Hq * cfg.R * cfg.P
+    resp = cfg.Hq * cfg.R * (cfg.R + 1) // 2
+    fwd = 2 * (cfg.Dk + cfg.Dv) * (pre + resp)
+    bwd_dq = 2 * (2 * cfg.Dk + cfg.Dv) * (pre + resp)
+    bwd_kv = 2 * (cfg.Dk + cfg.Dv) * resp
+    return fwd, bwd_dq, bwd_kv
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        time.sleep(0.25)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def run_cuda(args):
+    from paper_2607_14952_b200 import binding as B
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = W.CONFIGS[args.workload]
+    fwd_f, dq_f, kv_f = algorithmic_flops(cfg)
+    step_flops = fwd_f + dq_f + kv_f
+
+    k_pool, v_pool, table = W.make_prefix(cfg, dev)
+    pages = B.ls_prefix_pages_build(cfg.P, cfg.page_size, cfg.num_shards, cfg.Hkv, cfg.Dk, cfg.Dv, k_pool.shape[0],
+                                    page_table=table, k_pool=k_pool, v_pool=None if cfg.v_aliases_k else v_pool,
+                                    v_aliases_k=cfg.v_aliases_k)
+    S = cfg.num_shards
+    n_members = max(1, min(cfg.G, 4))
+    members = [W.make_member(cfg, (m + rank * n_members), dev) for m in range(n_members)]
+    o_part = torch.empty((S + 1, cfg.R, cfg.Hq, cfg.Dv), dtype=torch.float32, device=dev)
+    lse_part = torch.empty((S + 1, cfg.R, cfg.Hq), dtype=torch.float32, device=dev)
+    o_bf16 = torch.empty((cfg.R, cfg.Hq, cfg.Dv), dtype=torch.bfloat16, device=dev)
+    o_f32 = torch.empty((cfg.R, cfg.Hq, cfg.Dv), dtype=torch.float32, device=dev)
+    lse = torch.empty((cfg.R, cfg.Hq), dtype=torch.float32, device=dev)
+    ws = torch.empty(B.ls_replay_attn_workspace_bytes(pages, cfg.R, cfg.Hq, cfg.scale, B.LS_WORKSPACE_BWD),
+                     dtype=torch.uint8, device=dev)
+    dq = torch.empty((cfg.R, cfg.Hq, cfg.Dk), dtype=torch.bfloat16, device=dev)
+    dk = torch.empty((cfg.R, cfg.Hkv, cfg.Dk), dtype=torch.bfloat16, device=dev)
+    dv = torch.empty((cfg.R, cfg.Hkv, cfg.Dv), dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step(q, kr, vr, d_o):
+        B.ls_replay_attn_fwd(pages, q, kr, vr, cfg.scale, o_part=o_part, lse_part=lse_part, status=status)
+        B.ls_lse_merge(o_part, lse_part, o_bf16=o_bf16, o_f32=o_f32, lse=lse)
+        B.ls_replay_attn_bwd(pages, q, kr, vr, o_f32, lse, d_o, cfg.scale, workspace=ws, dq=dq, dk_resp=dk,
+                             dv_resp=dv, status=status)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    for w in range(args.warmup):
+        step(*members[w % n_members])
+    barrier()
+
+    # ---- device-resident timing; the dominant kernels are timed alone through armed events
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    kev = {k: [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+           for k in (B.LS_KERNEL_FWD, B.LS_KERNEL_BWD_DQ)}
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    for i in range(args.steps):
+        for k in kev:
+            B.ls_profile_arm_events(k, kev[k][i][0], kev[k][i][1])
+        ev[i][0].record()
+        step(*members[i % n_members])
+        ev[i][1].record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms = sum(a.elapsed_time(b) for a, b in ev)
+    k_ms = {k: sum(a.elapsed_time(b) for a, b in kev[k]) / args.steps for k in kev}
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    ms_total = float(t.item())
+    if int(status.item()) != 0:
+        raise RuntimeError("device status %d" % int(status.item()))
+
+    # ---- end to end: host buffers in, host results out, copies inside the timed region
+    host_in = [[x.cpu().pin_memory() for x in m] for m in members]
+    host_out = [torch.empty_like(x, device="cpu").pin_memory() for x in (o_bf16, dq, dk, dv)]
+    dev_in = [torch.empty_like(x) for x in members[0]]
+    h2d = sum(x.numel() * x.element_size() for x in host_in[0])
+    d2h = sum(x.numel() * x.element_size() for x in host_out)
+
+    def e2e_step(i):
+        for d, hsrc in zip(dev_in, host_in[i % n_members]):
+            d.copy_(hsrc, non_blocking=True)
+        step(*dev_in)
+        for hdst, d in zip(host_out, (o_bf16, dq, dk, dv)):
+            hdst.copy_(d, non_blocking=True)
+
+    e2e_step(0)
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    e2e_wall = time.perf_counter() - t0
+    te = torch.tensor([max(e0.elapsed_time(e1), e2e_wall * 1e3)], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(te, op=torch.distributed.ReduceOp.MAX)
+    e2e_ms = float(te.item())
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    ms_per_step = ms_total / args.steps
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    dq_tflops = dq_f / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e12
+    fwd_tflops = fwd_f / (k_ms[B.LS_KERNEL_FWD] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "%s: P=%d R=%d Hq=%d Hkv=%d Dk=%d Dv=%d page=%d shards=%d, one member per step" % (
+            cfg.name, cfg.P, cfg.R, cfg.Hq, cfg.Hkv, cfg.Dk, cfg.Dv, cfg.page_size, cfg.num_shards),
+            "l2": "inputs larger than L2 (%.2f GiB of K/V streamed per pass)" % (
+                (k_pool.numel() + (0 if cfg.v_aliases_k else v_pool.numel())) * 2 / 2**30),
+            "parallelism": "replicas x%d" % world, "flops_per_step": step_flops,
+            "prefix_positions_per_s": world * cfg.P / (ms_per_step * 1e-3)},
+        "clocks": clocks,
+        "e2e": {"value": world * step_flops / (e2e_ms / args.steps * 1e-3) / 1e12, "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": 7 * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "bwd_kernel<D,DQ> (query-gradient pass)",
+                     "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
+                     "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
+                     "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ], "traffic": None,
+                     "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peak,
+                                    "ms_per_launch": k_ms[B.LS_KERNEL_FWD]},
+                     "whole_step_frac": value / world / peak,
+                     "frac_of_nominal_2250": value / world / 2250.0},
+    }
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(cfg, seconds_target=15.0)
+    print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def _cpu_sample_inputs(cfg):
+    """Inputs of ONE KV head on the host, drawn with the CPU generator (same distributions)."""
+    one = W.scaled(cfg, Hkv=1, Hq=cfg.Hq // cfg.Hkv, needles=0)
+    k_pool, v_pool, table = W.make_prefix(one, "cpu")
+    q, kr, vr, d_o = W.make_member(one, 0, "cpu")
+    return one, W.bf16_bits(k_pool), (W.bf16_bits(k_pool) if cfg.v_aliases_k else W.bf16_bits(v_pool)), table, \
+        W.bf16_bits(q), W.bf16_bits(kr), W.bf16_bits(vr), W.bf16_bits(d_o)
+
+
+def _oracle_rows(one, kp, vp, table, q, kr, vr, d_o, rows):
+    from oracle import attention as oa
+    t_rows = np.linspace(0, one.R - 1, rows).astype(np.int64)
+    heads = np.arange(rows) % one.Hq
+    t0 = time.perf_counter()
+    oa.backward_rows(q[t_rows, heads], t_rows, 0, kp, vp, table, one.P, one.page_size, kr, vr,
+                     float(np.float32(one.scale)), d_o[t_rows, heads])
+    dt = time.perf_counter() - t0
+    # algorithmic flops of those rows: forward + dQ over every visible key (+ response dK/dV share)
+    vis = one.P + t_rows + 1
+    flops = float((vis * (2 * (one.Dk + one.Dv) + 2 * (2 * one.Dk + one.Dv))).sum()
+                  + ((t_rows + 1) * 2 * (one.Dk + one.Dv)).sum())
+    return dt, flops
+
+
+def cpu_baseline(cfg, seconds_target=15.0, inputs=None):
+    """The fp64 oracle as it stands, timed on this machine's host cores on a bounded row sample."""
+    inp = inputs or _cpu_sample_inputs(cfg)
+    dt, fl = _oracle_rows(*inp, rows=4)
+    rows = int(max(4, min(256, seconds_target / max(dt / 4, 1e-6))))
+    dt, fl = _oracle_rows(*inp, rows=rows)
+    return {"value": fl / dt / 1e12, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": "%d (row, head) pairs of one KV head of %s, forward + backward over all %d visible keys, "
+                      "%.1f s" % (rows, cfg.name, cfg.P + cfg.R, dt)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = W.CONFIGS[args.workload]
+    inp = _cpu_sample_inputs(cfg)
+    rows = args.ref_rows
+    for _ in range(args.warmup):
+        _oracle_rows(*inp, rows=max(1, rows // 4))
+    times, flops = [], 0.0
+    for _ in range(args.steps):
+        dt, fl = _oracle_rows(*inp, rows=rows)
+        times.append(dt)
+        flops += fl
+    value = flops / sum(times) / 1e12
+    sample = "%d (row, head) pairs of one KV head per step, forward + backward over all visible keys" % rows
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s (bounded sample: %s)" % (cfg.name, sample)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="p2m", choices=list(W.CONFIGS))
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -180,6 +180,21 @@ ls_status_t ls_replay_attn_bwd(const ls_pages_t* pages, const ls_attn_params_t* 
                                void* workspace, size_t workspace_bytes,
                                int32_t* status_dev, void* stream);
 
+/*
+ * Measurement aid (the paper has no counterpart): arms a one-shot pair of CUDA events
+ * (cudaEvent_t passed as void*) that the NEXT launch of the named kernel records on its
+ * own stream, start just before and stop just after the launch.  The pair is disarmed
+ * once used.  Passing NULL events disarms.  Not thread-safe; meant for benchmarks.
+ */
+typedef enum {
+  LS_KERNEL_FWD = 0,      /* replay forward (one launch per ls_replay_attn_fwd) */
+  LS_KERNEL_BWD_DQ = 1,   /* query-gradient pass over all partials */
+  LS_KERNEL_BWD_DK = 2,   /* response dK pass */
+  LS_KERNEL_BWD_DV = 3,   /* response dV pass */
+  LS_KERNEL_COUNT = 4
+} ls_kernel_t;
+ls_status_t ls_profile_arm_events(int kernel, void* start_event, void* stop_event);
+
 const char* ls_status_string(ls_status_t status);
 
 #ifdef __cplusplus

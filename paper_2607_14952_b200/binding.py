@@ -19,6 +19,7 @@ LS_ERR_INVALID_ARG, LS_ERR_BAD_PAGE_TABLE, LS_ERR_UNSUPPORTED_SHAPE, LS_ERR_ALIG
 LS_ERR_WORKSPACE, LS_ERR_STALE, LS_ERR_CUDA, LS_ERR_TIMEOUT, LS_ERR_NONFINITE = -5, -6, -7, -8, -9
 LS_SHARD_CONTIGUOUS, LS_SHARD_CYCLIC, LS_SHARD_ZIGZAG = 0, 1, 2
 LS_WORKSPACE_FWD, LS_WORKSPACE_BWD = 0, 1
+LS_KERNEL_FWD, LS_KERNEL_BWD_DQ, LS_KERNEL_BWD_DK, LS_KERNEL_BWD_DV = 0, 1, 2, 3
 
 
 class ls_pages_desc_t(C.Structure):
@@ -62,6 +63,8 @@ def lib():
         L.ls_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
         L.ls_replay_attn_bwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                          C.c_size_t, vp, vp]
+        L.ls_profile_arm_events.argtypes = [C.c_int, vp, vp]
+        L.ls_profile_arm_events.restype = C.c_int
         L.ls_status_string.argtypes = [C.c_int]
         L.ls_status_string.restype = C.c_char_p
         for f in ("ls_prefix_pages_build", "ls_prefix_pages_export", "ls_prefix_pages_checksum",
@@ -211,3 +214,13 @@ def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspa
                                   workspace.numel(), _ptr(status), _stream())
     _check(st, "ls_replay_attn_bwd")
     return dq, dk_resp, dv_resp
+
+
+def ls_profile_arm_events(kernel, start_event, stop_event):
+    """start/stop: torch.cuda.Event(enable_timing=True) that the next launch of `kernel` records."""
+    for e in (start_event, stop_event):
+        if e is not None and not e.cuda_event:
+            e.record()          # torch creates the CUDA event lazily; force it into existence
+    a = None if start_event is None else C.c_void_p(start_event.cuda_event)
+    b = None if stop_event is None else C.c_void_p(stop_event.cuda_event)
+    _check(lib().ls_profile_arm_events(kernel, a, b), "ls_profile_arm_events")

@@ -394,7 +394,9 @@ static ls_status_t launch_fwd(const FwdParams& prm, int grid, cudaStream_t st) {
       return LS_ERR_CUDA;
     configured = true;
   }
+  profile_begin(LS_KERNEL_FWD, st);
   fwd_kernel<DK, DV><<<grid, kFwdThreads, C::SMEM_BYTES, st>>>(prm);
+  profile_end(LS_KERNEL_FWD, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 

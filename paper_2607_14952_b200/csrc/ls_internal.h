@@ -55,6 +55,19 @@ ls_status_t encode_map(CUtensorMap* out, const void* base, int64_t dim_d, int64_
                        int64_t dim_head, int64_t dim_page, int64_t stride_tok, int64_t stride_head,
                        int64_t stride_page, int box_tok);
 
+// One-shot event pairs armed by ls_profile_arm_events.
+struct ProfileSlot {
+  cudaEvent_t start, stop;
+};
+extern ProfileSlot g_profile[LS_KERNEL_COUNT];
+inline void profile_begin(int k, cudaStream_t st) {
+  if (g_profile[k].start) cudaEventRecord(g_profile[k].start, st);
+}
+inline void profile_end(int k, cudaStream_t st) {
+  if (g_profile[k].stop) cudaEventRecord(g_profile[k].stop, st);
+  g_profile[k].start = g_profile[k].stop = nullptr;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace ls

@@ -290,6 +290,17 @@ extern "C" ls_status_t ls_prefix_pages_checksum(const ls_pages_t* h, uint64_t* s
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
+namespace ls {
+ProfileSlot g_profile[LS_KERNEL_COUNT] = {};
+}
+
+extern "C" ls_status_t ls_profile_arm_events(int kernel, void* start_event, void* stop_event) {
+  if (kernel < 0 || kernel >= LS_KERNEL_COUNT) return LS_ERR_INVALID_ARG;
+  ls::g_profile[kernel].start = static_cast<cudaEvent_t>(start_event);
+  ls::g_profile[kernel].stop = static_cast<cudaEvent_t>(stop_event);
+  return LS_OK;
+}
+
 extern "C" const char* ls_status_string(ls_status_t s) {
   switch (s) {
     case LS_OK: return "ok";

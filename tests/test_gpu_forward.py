@@ -20,7 +20,7 @@ def small(name, **kw):
 
 def test_config1_tiny_full():
     case = parity.Case(CONFIGS["tiny"])
-    parity.check_forward(case)
+    parity.check_forward(case, strict_abs=True)
 
 
 @pytest.mark.parametrize("cfg", [
