@@ -181,6 +181,34 @@ ls_status_t ls_replay_attn_bwd(const ls_pages_t* pages, const ls_attn_params_t* 
                                int32_t* status_dev, void* stream);
 
 /*
+ * ls_replay_attn_bwd for callers that cannot hand over scratch memory (the paper has no
+ * counterpart; this is a packaging variant, the arithmetic and the outputs are those of
+ * ls_replay_attn_bwd).  A replay scheduler that has sized the page pool to fill the GPU, or
+ * code running under a framework whose allocator already owns all device memory, has
+ * nowhere to take a workspace from at backward time: a late cudaMalloc there can fail or
+ * stall the whole device.  This call therefore allocates nothing, in the library or in
+ * CUDA: the per-partial dQ sums and Delta go to a fixed array of LS_STATIC_SCRATCH_BYTES
+ * that is part of the library's device image, so every GPU that loads the library holds
+ * that much memory until the process exits.
+ *  - Shapes whose backward workspace (ls_replay_attn_workspace_bytes) exceeds
+ *    LS_STATIC_SCRATCH_BYTES are rejected with LS_ERR_WORKSPACE before any launch.
+ *  - The first call on each device looks up the array's device address (the device must be
+ *    current); make that first call before starting any stream capture.
+ *  - All calls on a device share the one array, which keeps the previous call's contents.
+ *    Nothing needs clearing (every word that is read is written first by the same call),
+ *    but two calls whose kernels overlap on the GPU (different streams) race on it:
+ *    serialise them.
+ * Arguments and errors otherwise as ls_replay_attn_bwd.
+ */
+#define LS_STATIC_SCRATCH_BYTES (32u << 20)
+size_t ls_replay_attn_bwd_static_capacity(void);
+ls_status_t ls_replay_attn_bwd_static(const ls_pages_t* pages, const ls_attn_params_t* prm,
+                                      const void* q, const void* k_resp, const void* v_resp,
+                                      const float* o_f32, const float* lse, const void* d_o,
+                                      void* dq, void* dk_resp, void* dv_resp,
+                                      int32_t* status_dev, void* stream);
+
+/*
  * Measurement aid (the paper has no counterpart): arms a one-shot pair of CUDA events
  * (cudaEvent_t passed as void*) that the NEXT launch of the named kernel records on its
  * own stream, start just before and stop just after the launch.  The pair is disarmed

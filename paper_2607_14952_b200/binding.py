@@ -63,6 +63,11 @@ def lib():
         L.ls_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
         L.ls_replay_attn_bwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                          C.c_size_t, vp, vp]
+        L.ls_replay_attn_bwd_static.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                                vp, vp]
+        L.ls_replay_attn_bwd_static.restype = C.c_int
+        L.ls_replay_attn_bwd_static_capacity.argtypes = []
+        L.ls_replay_attn_bwd_static_capacity.restype = C.c_size_t
         L.ls_profile_arm_events.argtypes = [C.c_int, vp, vp]
         L.ls_profile_arm_events.restype = C.c_int
         L.ls_status_string.argtypes = [C.c_int]
@@ -213,6 +218,23 @@ def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspa
                                   _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk_resp), _ptr(dv_resp), _ptr(workspace),
                                   workspace.numel(), _ptr(status), _stream())
     _check(st, "ls_replay_attn_bwd")
+    return dq, dk_resp, dv_resp
+
+
+def ls_replay_attn_bwd_static_capacity():
+    return int(lib().ls_replay_attn_bwd_static_capacity())
+
+
+def ls_replay_attn_bwd_static(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, dq, dk_resp, dv_resp, status=None):
+    """Backward that takes no workspace: its scratch is a fixed array inside the library, for
+    callers that have no device memory left to lend (page pool sized to the whole GPU, or an
+    allocator that owns it all).  Outputs must be passed in; nothing is allocated here."""
+    R, Hq, _ = q.shape
+    prm = _params(R, Hq, scale)
+    st = lib().ls_replay_attn_bwd_static(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp),
+                                         _ptr(o_f32), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk_resp),
+                                         _ptr(dv_resp), _ptr(status), _stream())
+    _check(st, "ls_replay_attn_bwd_static")
     return dq, dk_resp, dv_resp
 
 

@@ -21,6 +21,8 @@
 // TMEM columns: ACC [0, D), then two buffers of (S 64 | T 64).
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "ls_internal.h"
 #include "ls_sm100.cuh"
 
@@ -588,4 +590,55 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DV>(P, grid_kv, cs) : ls::launch_bwd<256, ls::MODE_DV>(P, grid_kv, cs);
   if (st != LS_OK) return st;
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------
+// Backward without caller scratch: the per-partial dQ sums and Delta live in a fixed
+// array inside the library's device image instead of a caller-provided workspace.
+// ---------------------------------------------------------------------------------
+namespace ls {
+
+constexpr size_t kStaticScratchBytes = LS_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_bwd_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_scratch_ptr[kMaxDevices] = {};
+static std::mutex g_scratch_mutex;
+
+// Device address of g_bwd_scratch on the current device.  In host code the array's name is
+// only a handle for the runtime, never an address a kernel could use, so the address is
+// looked up once per device (with that device current) and cached.
+static ls_status_t static_scratch(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LS_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_bwd_scratch) != cudaSuccess || !ptr) return LS_ERR_CUDA;
+    g_scratch_ptr[dev] = ptr;
+  }
+  *out = g_scratch_ptr[dev];
+  return LS_OK;
+}
+
+}  // namespace ls
+
+extern "C" size_t ls_replay_attn_bwd_static_capacity(void) { return ls::kStaticScratchBytes; }
+
+extern "C" ls_status_t ls_replay_attn_bwd_static(const ls_pages_t* h, const ls_attn_params_t* prm, const void* q,
+                                                 const void* k_resp, const void* v_resp, const float* o_f32,
+                                                 const float* lse, const void* d_o, void* dq, void* dk_resp,
+                                                 void* dv_resp, int32_t* status_dev, void* stream) {
+  if (!h || !prm) return LS_ERR_INVALID_ARG;
+  const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_BWD);
+  if (need == 0) return LS_ERR_INVALID_ARG;
+  if (need > ls::kStaticScratchBytes) return LS_ERR_WORKSPACE;   // shape too large for the built-in scratch
+  void* scratch = nullptr;
+  ls_status_t st = ls::static_scratch(&scratch);
+  if (st != LS_OK) return st;
+  // Nothing in the scratch has to start at zero: the dQ pass writes every partial of every
+  // row (zeros for an empty partial) and the Delta kernel writes every row before either
+  // is read, so the previous call's leftovers are never observed.
+  return ls_replay_attn_bwd(h, prm, q, k_resp, v_resp, o_f32, lse, d_o, dq, dk_resp, dv_resp, scratch,
+                            ls::kStaticScratchBytes, status_dev, stream);
 }
