@@ -128,8 +128,17 @@ typedef struct {
   int32_t R;             /* response tokens, >= 1 */
   int32_t num_q_heads;   /* Hq */
   float scale;           /* softmax scale, e.g. 1/sqrt(dim_k) */
-  int32_t flags;         /* 0 */
+  int32_t flags;         /* 0, or LS_FLAG_* bits */
 } ls_attn_params_t;
+
+/* Diagnostic switches for profiling the kernel pipelines: they skip one stage (operand
+ * loads, tensor-core instructions, or the per-row arithmetic) while keeping every barrier
+ * hand-off, so the cost of the remaining stages can be timed.  Outputs are meaningless
+ * when any of them is set. */
+#define LS_FLAG_ABLATE_LOADS   (1 << 16)
+#define LS_FLAG_ABLATE_MMA     (1 << 17)
+#define LS_FLAG_ABLATE_SOFTMAX (1 << 18)
+#define LS_FLAG_ABLATE_MASK    (7 << 16)
 
 enum { LS_WORKSPACE_FWD = 0, LS_WORKSPACE_BWD = 1 };
 

@@ -159,8 +159,8 @@ def ls_prefix_pages_checksum(pages):
     return int(out.value)
 
 
-def _params(R, Hq, scale):
-    return ls_attn_params_t(R, Hq, float(scale), 0)
+def _params(R, Hq, scale, flags=0):
+    return ls_attn_params_t(R, Hq, float(scale), flags)
 
 
 def ls_replay_attn_workspace_bytes(pages, R, Hq, scale, which):
@@ -168,7 +168,7 @@ def ls_replay_attn_workspace_bytes(pages, R, Hq, scale, which):
     return int(lib().ls_replay_attn_workspace_bytes(pages.handle, C.byref(prm), which))
 
 
-def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=None, status=None):
+def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=None, status=None, flags=0):
     """Returns (o_part [(S+1),R,Hq,Dv] fp32, lse_part [(S+1),R,Hq] fp32)."""
     R, Hq, _ = q.shape
     S, Dv = pages.desc.num_shards, pages.desc.dim_v
@@ -176,7 +176,7 @@ def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=No
         o_part = torch.empty((S + 1, R, Hq, Dv), dtype=torch.float32, device=q.device)
     if lse_part is None:
         lse_part = torch.empty((S + 1, R, Hq), dtype=torch.float32, device=q.device)
-    prm = _params(R, Hq, scale)
+    prm = _params(R, Hq, scale, flags)
     st = lib().ls_replay_attn_fwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_part),
                                   _ptr(lse_part), None, 0, _ptr(status), _stream())
     _check(st, "ls_replay_attn_fwd")
@@ -201,7 +201,7 @@ def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=
 
 
 def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspace=None, dq=None, dk_resp=None,
-                       dv_resp=None, status=None):
+                       dv_resp=None, status=None, flags=0):
     """Returns (dq, dk_resp, dv_resp) in bf16."""
     R, Hq, _ = q.shape
     if workspace is None:
@@ -213,7 +213,7 @@ def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspa
         dk_resp = torch.empty_like(k_resp)
     if dv_resp is None:
         dv_resp = torch.empty_like(v_resp)
-    prm = _params(R, Hq, scale)
+    prm = _params(R, Hq, scale, flags)
     st = lib().ls_replay_attn_bwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_f32),
                                   _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk_resp), _ptr(dv_resp), _ptr(workspace),
                                   workspace.numel(), _ptr(status), _stream())

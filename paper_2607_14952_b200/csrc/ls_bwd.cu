@@ -31,9 +31,10 @@ namespace ls {
 enum { MODE_DQ = 0, MODE_DK = 1, MODE_DV = 2 };
 
 struct BwdParams {
-  CUtensorMap a1_map, a2_map;                 // stationary rows, 128-token boxes
-  CUtensorMap b1_map, b1_tail, b2_map, b2_tail, b3_map, b3_tail;   // prefix pool sources (mode DQ)
-  CUtensorMap b1r_map, b2r_map, b3r_map;      // dense sources: response K/V (DQ) or Q/dO (DK, DV)
+  CUtensorMap a1_map, a2_map;                 // stationary rows: box 64 x 128 tokens x 1 group
+  // streamed 64-column chunks, box 64 x 64 tokens x D/64 groups
+  CUtensorMap bk_map, bk_tail, bv_map, bv_tail;   // prefix pool K and V (mode DQ)
+  CUtensorMap b1r_map, b2r_map, b3r_map;          // dense sources: response K/V/K (DQ) or Q/dO/(Q|dO) (DK, DV)
   const int32_t* shard_phys_pages;
   const int32_t* shard_page_offset;
   const int32_t* shard_tail_slot;
@@ -43,23 +44,20 @@ struct BwdParams {
   float* dq_part;        // [(S+1), R, Hq, D] fp32, unscaled (mode DQ)
   __nv_bfloat16* out;    // dk_resp or dv_resp [R, Hkv, D] (modes DK, DV)
   int32_t* status;
-  int R, Hq, Hkv, g, S, pg, tiles_per_head, nq_tiles;
+  int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   float scale, scale_log2;
 };
 
 constexpr int kBwdThreads = 192;
-constexpr int kBwdChunk = 16384;
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
 struct BwdCfg {
-  static constexpr int SLABS = D / 64;           // 16 KB slabs per stationary operand
-  static constexpr int KCH = D / 128;            // K-major chunks per 64-column tile and operand
-  static constexpr int MKEYS = 8192 / D;         // columns per MN-major chunk
-  static constexpr int MCH = 64 / MKEYS;         // MN-major chunks per tile
-  static constexpr int RING = (D == 128) ? 8 : 6;
-  static constexpr int A_BYTES = 2 * SLABS * kBwdChunk;
-  static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * kBwdChunk + 512;
+  static constexpr int SLABS = D / 64;            // 64-channel groups
+  static constexpr int CHUNK = 64 * D * 2;        // one streamed chunk: 64 columns x D channels
+  static constexpr int RING = (D == 128) ? 8 : 3;
+  static constexpr int A_BYTES = 2 * SLABS * 16384;
+  static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * CHUNK + 512;
 };
 
 template <int D, int MODE>
@@ -69,9 +67,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a1_smem = smem;
-  uint8_t* a2_smem = smem + C::SLABS * kBwdChunk;
+  uint8_t* a2_smem = smem + C::SLABS * 16384;
   uint8_t* ring = smem + C::A_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kBwdChunk);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * C::CHUNK);
   uint64_t* a_full = bars;
   uint64_t* full = bars + 1;
   uint64_t* empty = full + C::RING;
@@ -142,152 +140,119 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   const uint32_t tmem_buf0 = tmem_base + D;
 
   if (warp == 0) {
-    // =========================================================== producer
-    if (n_tiles > 0) {
-      if (lane == 0) {
-        mbar_arrive_expect_tx(a_full, (HAS_T ? 2 : 1) * C::SLABS * kBwdChunk);
-        const int a_head = (MODE == MODE_DQ) ? h : kvh;
-        for (int c = 0; c < C::SLABS; ++c) {
-          tma_load_4d(a1_smem + c * kBwdChunk, &p.a1_map, a_full, c * 64, row0, a_head, 0);
-          if (HAS_T) tma_load_4d(a2_smem + c * kBwdChunk, &p.a2_map, a_full, c * 64, row0, a_head, 0);
-        }
+    // =========================================================== producer (one thread)
+    if (lane == 0 && n_tiles > 0) {
+      mbar_arrive_expect_tx(a_full, (HAS_T ? 2 : 1) * C::SLABS * 16384);
+      const int a_head = (MODE == MODE_DQ) ? h : kvh;
+      for (int c = 0; c < C::SLABS; ++c) {
+        tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, a_head, 0);
+        if (HAS_T) tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, a_head, 0);
       }
       const int32_t* pages = p.shard_phys_pages + page_off;
-      int win_tag[2] = {-1, -1};
-      int win_page[2] = {0, 0};
-      auto page_of = [&](int ps) -> int {
-        const int w = ps >> 5, b = w & 1;
-        if (win_tag[b] != w) {
-          win_tag[b] = w;
-          const int i = (w << 5) + lane;
-          win_page[b] = (i < n_pages) ? __ldg(pages + i) : 0x7fffffff;
-        }
-        return __shfl_sync(0xffffffffu, win_page[b], ps & 31);
-      };
-      uint32_t cc = 0;
-      bool ok = true;
-      auto acquire = [&]() -> uint8_t* {
-        const uint32_t slot = cc % C::RING, ph = (cc / C::RING) & 1;
-        ok = ok && mbar_wait(&empty[slot], ph ^ 1, abort_flag);
-        if (ok) mbar_arrive_expect_tx(&full[slot], kBwdChunk);
-        return ring + slot * kBwdChunk;
-      };
-      // TMA coordinates (token offset, head, page) and tail flag of column tile i (+ sub offset)
-      auto locate = [&](int i, int sub, int& off, int& head, int& page, bool& tail) {
-        if (MODE == MODE_DQ) {
-          const int tok = i * 64 + sub;
-          head = kvh;
-          if (is_resp) { off = tok; page = 0; tail = false; }
-          else {
-            const int ps = tok / p.pg;
-            page = page_of(ps);
-            off = tok % p.pg;
-            tail = (ps == tail_slot);
-          }
-        } else {
-          head = kvh * p.g + i / n_tt;
-          off = (tt_min + i % n_tt) * 64 + sub;
-          page = 0;
-          tail = false;
-        }
-      };
+      const int pg_mask = (1 << p.pg_shift) - 1;
       const bool dense = (MODE != MODE_DQ) || is_resp;
-      auto load_st = [&](int i) {     // chunks of S (and T) of tile i, K-major
-        int off, head, page;
-        bool tail;
-        locate(i, 0, off, head, page, tail);
-        if (lane == 0) {
-          for (int op = 0; op < (HAS_T ? 2 : 1); ++op) {
-            const CUtensorMap* m = op == 0 ? (dense ? &p.b1r_map : (tail ? &p.b1_tail : &p.b1_map))
-                                           : (dense ? &p.b2r_map : (tail ? &p.b2_tail : &p.b2_map));
-            for (int c = 0; c < C::KCH; ++c) {
-              uint8_t* dst = acquire();
-              if (ok) {
-                tma_load_4d(dst, m, &full[cc % C::RING], c * 128, off, head, page);
-                tma_load_4d(dst + 8192, m, &full[cc % C::RING], c * 128 + 64, off, head, page);
-              }
-              ++cc;
+      auto fetch = [&](int tile) -> int {     // physical page of column tile `tile` (prefix shards only)
+        const int ps = (tile * 64) >> p.pg_shift;
+        return (!dense && tile < n_tiles && ps < n_pages) ? __ldg(pages + ps) : 0;
+      };
+      uint32_t slot = 0, phase = 0, issued = 0;
+      bool ok = true;
+      // one chunk: 64 columns x D channels of source `which` (0: B1, 1: B2, 2: B3) of column tile i
+      auto load = [&](int which, int i, int page) {
+        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
+        if (ok) {
+          mbar_arrive_expect_tx(&full[slot], C::CHUNK);
+          uint8_t* dst = ring + slot * C::CHUNK;
+          if (MODE == MODE_DQ) {
+            const int tok = i * 64;
+            if (is_resp) {
+              tma_load_5d(dst, which == 1 ? &p.b2r_map : &p.b1r_map, &full[slot], 0, tok, 0, kvh, 0);
+            } else {
+              const bool tail = (tok >> p.pg_shift) == tail_slot;
+              const CUtensorMap* m = which == 1 ? (tail ? &p.bv_tail : &p.bv_map) : (tail ? &p.bk_tail : &p.bk_map);
+              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 0, kvh, page);
             }
+          } else {
+            const int hh = kvh * p.g + i / n_tt;
+            const int tq = (tt_min + i % n_tt) * 64;
+            const CUtensorMap* m = which == 0 ? &p.b1r_map : which == 1 ? &p.b2r_map : &p.b3r_map;
+            tma_load_5d(dst, m, &full[slot], 0, tq, 0, hh, 0);
           }
         }
+        ++issued;
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
-      auto load_m = [&](int i) {      // chunks of B3 of tile i, MN-major
-        int off[C::MCH], head[C::MCH], page[C::MCH];
-        bool tail[C::MCH];
-        for (int r = 0; r < C::MCH; ++r) locate(i, r * C::MKEYS, off[r], head[r], page[r], tail[r]);
-        if (lane == 0) {
-          for (int r = 0; r < C::MCH; ++r) {
-            const CUtensorMap* m = dense ? &p.b3r_map : (tail[r] ? &p.b3_tail : &p.b3_map);
-            uint8_t* dst = acquire();
-            if (ok)
-              for (int c = 0; c < D / 64; ++c)
-                tma_load_4d(dst + c * C::MKEYS * 128, m, &full[cc % C::RING], c * 64, off[r], head[r], page[r]);
-            ++cc;
-          }
-        }
-      };
-      load_st(0);
-      if (n_tiles > 1) load_st(1);
-      for (int i = 0; i < n_tiles; ++i) {
-        load_m(i);
-        if (i + 2 < n_tiles) load_st(i + 2);
+      // chunk order = consumption order: ST(0) ST(1) [M(i) ST(i+2)] ...
+      int pg0 = fetch(0), pg1 = fetch(1), pg2 = fetch(2);      // pages of tiles i, i+1, i+2
+      load(0, 0, pg0);
+      if (HAS_T) load(1, 0, pg0);
+      if (n_tiles > 1) {
+        load(0, 1, pg1);
+        if (HAS_T) load(1, 1, pg1);
       }
-      if (lane == 0 && *abort_flag) {   // aborted: wait (bounded) for the copies already started
-        for (uint32_t s = 0; s < (uint32_t)C::RING && s < cc; ++s) {
-          const uint32_t last = ((cc - 1 - s) / C::RING) * C::RING + s;
+      for (int i = 0; i < n_tiles; ++i) {
+        const int pg3 = fetch(i + 3);                          // used two iterations from now
+        load(2, i, pg0);
+        if (i + 2 < n_tiles) {
+          load(0, i + 2, pg2);
+          if (HAS_T) load(1, i + 2, pg2);
+        }
+        pg0 = pg1; pg1 = pg2; pg2 = pg3;
+      }
+      if (*abort_flag) {   // aborted: wait (bounded) for the copies already started
+        for (uint32_t s = 0; s < (uint32_t)C::RING && s < issued; ++s) {
+          const uint32_t last = ((issued - 1 - s) / C::RING) * C::RING + s;
           const uint64_t t_start = globaltimer_ns();
-          while (!mbar_try_wait(&full[s], (last / C::RING) & 1) && globaltimer_ns() - t_start < 100000000ull) {
+          while (!mbar_try_wait(&full[s], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
           }
         }
       }
     }
   } else if (warp == 1) {
-    // =========================================================== MMA issuer
+    // =========================================================== MMA issuer (one thread)
     if (lane == 0 && n_tiles > 0) {
       constexpr uint32_t idesc_st = make_idesc(128, 64, 0, 0);
       constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);
-      const uint32_t a1_addr = smem_u32(a1_smem), a2_addr = smem_u32(a2_smem);
-      const uint32_t ring_addr = smem_u32(ring);
-      uint32_t cc = 0;
+      constexpr uint32_t hi = sdesc_hi(1024);
+      const uint32_t a1_lo = sdesc_lo(smem_u32(a1_smem), 16), a2_lo = sdesc_lo(smem_u32(a2_smem), 16);
+      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);      // K-major view of a chunk
+      const uint32_t ring_m_lo = sdesc_lo(smem_u32(ring), 8192);    // MN-major view: 8 KB group pitch
+      uint32_t slot = 0, phase = 0;
       bool ok = mbar_wait(a_full, 0, abort_flag);
+      auto advance = [&]() {
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
       auto issue_st = [&](int i) {
         const uint32_t buf = tmem_buf0 + (i & 1) * 128;
+#pragma unroll
         for (int op = 0; op < (HAS_T ? 2 : 1); ++op) {
-          const uint32_t d = buf + op * 64;
-          const uint32_t a_addr = op == 0 ? a1_addr : a2_addr;
-          for (int c = 0; c < C::KCH; ++c) {
-            const uint32_t slot = cc % C::RING, ph = (cc / C::RING) & 1;
-            ok = ok && mbar_wait(&full[slot], ph, abort_flag);
-            if (!ok) return;
-            tc_fence_after();
-            const uint32_t b0 = ring_addr + slot * kBwdChunk;
+          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
+          const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
+          const uint32_t b_lo = ring_k_lo + slot * (C::CHUNK >> 4);
 #pragma unroll
-            for (int sl = 0; sl < 2; ++sl)
+          for (int s = 0; s < C::SLABS; ++s)
 #pragma unroll
-              for (int k = 0; k < 4; ++k)
-                mma_ss(d, make_sdesc(a_addr + (2 * c + sl) * kBwdChunk + k * 32, 16, 1024),
-                       make_sdesc(b0 + sl * 8192 + k * 32, 16, 1024), idesc_st, (c | sl | k) != 0);
-            mma_commit(&empty[slot]);
-            ++cc;
-          }
+            for (int k = 0; k < 4; ++k)
+              mma_ss(buf + op * 64, sdesc(a_lo + ((s * 16384 + k * 32) >> 4), hi),
+                     sdesc(b_lo + ((s * 8192 + k * 32) >> 4), hi), idesc_st, (s | k) != 0);
+          mma_commit(&empty[slot]);
+          advance();
         }
         mma_commit(&st_full[i & 1]);
       };
       auto issue_acc = [&](int i) {
         const uint32_t e_base = tmem_buf0 + (i & 1) * 128;
-        for (int r = 0; r < C::MCH; ++r) {
-          const uint32_t slot = cc % C::RING, ph = (cc / C::RING) & 1;
-          ok = ok && mbar_wait(&full[slot], ph, abort_flag);
-          if (!ok) return;
-          tc_fence_after();
-          const uint32_t b0 = ring_addr + slot * kBwdChunk;
+        ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t b_lo = ring_m_lo + slot * (C::CHUNK >> 4);
 #pragma unroll
-          for (int kk = 0; kk < C::MKEYS / 16; ++kk)
-            mma_ts(tmem_acc, e_base + (r * (C::MKEYS / 16) + kk) * 8, make_sdesc(b0 + kk * 2048, C::MKEYS * 128, 1024),
-                   idesc_acc, (i | r | kk) != 0);
-          mma_commit(&empty[slot]);
-          ++cc;
-        }
+        for (int kk = 0; kk < 4; ++kk)
+          mma_ts(tmem_acc, e_base + kk * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi), idesc_acc, (i | kk) != 0);
+        mma_commit(&empty[slot]);
+        advance();
         if (i == n_tiles - 1) mma_commit(acc_final);
       };
       if (ok) issue_st(0);
@@ -522,14 +487,14 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   float* dq_part = static_cast<float*>(workspace);
   float* delta = dq_part + (size_t)(d.num_shards + 1) * rows * D;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  const int mkeys = 8192 / D;
 
   ls::delta_kernel<<<(int)((rows + 7) / 8), 256, 0, cs>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows,
                                                         d.dim_v, delta);
 
-  auto dense_map = [&](CUtensorMap* m, const void* base, int heads, int box) {
-    return ls::encode_map(m, base, D, R, heads, 1, (int64_t)heads * D, D, (int64_t)R * heads * D, box);
+  auto dense_map = [&](CUtensorMap* m, const void* base, int heads, int box_tok, int groups) {
+    return ls::encode_map5(m, base, D, R, heads, 1, (int64_t)heads * D, D, (int64_t)R * heads * D, box_tok, groups);
   };
+  const int groups = D / 64;
   ls::BwdParams P;
   P.shard_phys_pages = h->d_shard_phys_pages;
   P.shard_page_offset = h->d_shard_page_offset;
@@ -545,25 +510,24 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   P.Hkv = Hkv;
   P.g = Hq / Hkv;
   P.S = d.num_shards;
-  P.pg = d.page_size;
+  P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 127) / 128;
   P.nq_tiles = P.g * P.tiles_per_head;
+  P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * ls::kLog2e;
 
   // ---- dQ: rows = queries, columns = keys of every partial
-  ls_status_t st = dense_map(&P.a1_map, q, Hq, 128);
-  if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128);
-  if (st == LS_OK) st = dense_map(&P.b1r_map, k_resp, Hkv, 64);
-  if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 64);
-  if (st == LS_OK) st = dense_map(&P.b3r_map, k_resp, Hkv, mkeys);
+  ls_status_t st = dense_map(&P.a1_map, q, Hq, 128, 1);
+  if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128, 1);
+  if (st == LS_OK) st = dense_map(&P.b1r_map, k_resp, Hkv, 64, groups);
+  if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 64, groups);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_map, h, 0, 64, groups, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_tail, h, 0, 64, groups, true);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_map, h, 1, 64, groups, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_tail, h, 1, 64, groups, true);
   if (st != LS_OK) return st;
-  P.b1_map = h->k_maps.full[ls::box_index(64)];
-  P.b1_tail = h->k_maps.tail[ls::box_index(64)];
-  P.b2_map = h->v_maps.full[ls::box_index(64)];
-  P.b2_tail = h->v_maps.tail[ls::box_index(64)];
-  P.b3_map = h->k_maps.full[ls::box_index(mkeys)];
-  P.b3_tail = h->k_maps.tail[ls::box_index(mkeys)];
+  P.b3r_map = P.b1r_map;
   const int64_t grid_dq = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;
   if (grid_dq > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DQ>(P, (int)grid_dq, cs)
@@ -575,17 +539,16 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
 
   // ---- dK and dV of the response keys: rows = keys, columns = queries of the KV group
   const int grid_kv = Hkv * P.tiles_per_head;
-  st = dense_map(&P.a1_map, k_resp, Hkv, 128);
-  if (st == LS_OK) st = dense_map(&P.a2_map, v_resp, Hkv, 128);
-  if (st == LS_OK) st = dense_map(&P.b1r_map, q, Hq, 64);
-  if (st == LS_OK) st = dense_map(&P.b2r_map, d_o, Hq, 64);
-  if (st == LS_OK) st = dense_map(&P.b3r_map, q, Hq, mkeys);
+  st = dense_map(&P.a1_map, k_resp, Hkv, 128, 1);
+  if (st == LS_OK) st = dense_map(&P.a2_map, v_resp, Hkv, 128, 1);
+  if (st == LS_OK) st = dense_map(&P.b1r_map, q, Hq, 64, groups);
+  if (st == LS_OK) st = dense_map(&P.b2r_map, d_o, Hq, 64, groups);
   if (st != LS_OK) return st;
+  P.b3r_map = P.b1r_map;
   P.out = static_cast<__nv_bfloat16*>(dk_resp);
   st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DK>(P, grid_kv, cs) : ls::launch_bwd<256, ls::MODE_DK>(P, grid_kv, cs);
   if (st != LS_OK) return st;
-  st = dense_map(&P.b3r_map, d_o, Hq, mkeys);
-  if (st != LS_OK) return st;
+  P.b3r_map = P.b2r_map;
   P.out = static_cast<__nv_bfloat16*>(dv_resp);
   st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DV>(P, grid_kv, cs) : ls::launch_bwd<256, ls::MODE_DV>(P, grid_kv, cs);
   if (st != LS_OK) return st;

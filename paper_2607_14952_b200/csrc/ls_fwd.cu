@@ -22,10 +22,10 @@
 namespace ls {
 
 struct FwdParams {
-  CUtensorMap q_map;
-  CUtensorMap k_map, k_tail_map;
-  CUtensorMap v_map, v_tail_map;
-  CUtensorMap kr_map, vr_map;
+  CUtensorMap q_map;               // box 64 x 128 tokens x KSLABS channel groups
+  CUtensorMap k_map, k_tail_map;   // pool K: box 64 x 128 x KSLABS (pages >= 128 tokens) or 64 x 64 x 1
+  CUtensorMap v_map, v_tail_map;   // pool V: box 64 x 64 tokens x DV/64 groups
+  CUtensorMap kr_map, vr_map;      // response K (64 x 128 x KSLABS) and V (64 x 64 x DV/64)
   const int32_t* shard_phys_pages;
   const int32_t* shard_page_offset;
   const int32_t* shard_tail_slot;
@@ -33,22 +33,37 @@ struct FwdParams {
   float* o_part;
   float* lse_part;
   int32_t* status;
-  int R, Hq, Hkv, g, S, pg, box_tok_k, tiles_per_head, nq_tiles, num_phys_pages;
+  int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  int ablate;   // diagnostic: LS_FLAG_ABLATE_* bits (results are then meaningless)
   float scale, scale_log2;
 };
 
-constexpr int kChunkBytes = 16384;
+// Build with -DLS_TIMING to make CTA 0 write per-role cycle counts (time spent in each kind
+// of wait, and in total) as int64 words starting 64 bytes past `status`; a profiling aid.
+#ifdef LS_TIMING
+#define LS_TWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
+#define LS_TDUMP(slot, val) do { if (blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
+#else
+#define LS_TWAIT(acc, expr) (expr)
+#define LS_TDUMP(slot, val) do { } while (0)
+#endif
+
 constexpr int kFwdThreads = 192;
 constexpr float kRescaleLog2 = 8.0f;   // the reference max lags the true max by at most 2^8
 
 template <int DK, int DV>
 struct FwdCfg {
-  static constexpr int KCH = DK / 64;            // K chunks per 128-key tile
-  static constexpr int VKEYS = 8192 / DV;        // keys per V chunk
-  static constexpr int NVCH = 128 / VKEYS;       // V chunks per tile
-  static constexpr int RING = (DK == 128) ? 10 : 8;
-  static constexpr int Q_BYTES = KCH * kChunkBytes;
-  static constexpr int SMEM_BYTES = 1024 + Q_BYTES + RING * kChunkBytes + 512;
+  static_assert(DK == DV, "the shared-latent (576/512) variant has its own kernel");
+  static constexpr int CHUNK = (DK == 256) ? 32768 : 16384;   // bytes per ring slot
+  static constexpr int KSLABS = CHUNK / 16384;     // 64-channel slabs (128 keys x 128 B) per K chunk
+  static constexpr int KCH = (DK / 64) / KSLABS;   // K chunks per 128-key tile
+  static constexpr int VKEYS = 64;                 // keys per V chunk
+  static constexpr int NVCH = 128 / VKEYS;         // V chunks per tile
+  static constexpr int VSUB = DV / 64;             // 8 KB sub-slabs (64 keys x 128 B) per V chunk
+  static_assert(VSUB * 8192 == CHUNK, "a V chunk fills one ring slot");
+  static constexpr int RING = (DK == 256) ? 4 : 10;
+  static constexpr int Q_BYTES = (DK / 64) * 16384;
+  static constexpr int SMEM_BYTES = 1024 + Q_BYTES + RING * CHUNK + 512;
 };
 
 template <int DK, int DV>
@@ -58,7 +73,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = smem;
   uint8_t* ring = smem + C::Q_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kChunkBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * C::CHUNK);
   uint64_t* q_full = bars;
   uint64_t* full = bars + 1;
   uint64_t* empty = full + C::RING;
@@ -70,6 +85,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
+  (void)tw0; (void)tw1; (void)tw2;
 
   // ---- work item
   int idx = blockIdx.x;
@@ -120,140 +137,164 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   const uint32_t tmem_s0 = tmem_base + DV;
 
   if (warp == 0) {
-    // =========================================================== producer
-    if (n_tiles > 0) {
-      if (lane == 0) {
-        mbar_arrive_expect_tx(q_full, C::Q_BYTES);
-        for (int c = 0; c < C::KCH; ++c) tma_load_4d(q_smem + c * kChunkBytes, &p.q_map, q_full, c * 64, t0, h, 0);
-      }
+    // =========================================================== producer (one thread)
+    if (lane == 0 && n_tiles > 0) {
+      const bool no_loads = (p.ablate & LS_FLAG_ABLATE_LOADS) != 0;
+      mbar_arrive_expect_tx(q_full, C::Q_BYTES);
+      for (int c = 0; c < C::KCH; ++c)
+        tma_load_5d(q_smem + c * C::CHUNK, &p.q_map, q_full, 0, t0, c * C::KSLABS, h, 0);
+
       const int32_t* pages = p.shard_phys_pages + page_off;
-      int win_tag[2] = {-1, -1};
-      int win_page[2] = {0, 0};
-      // physical page of the shard's page slot `ps` (warp-uniform); out of range -> a page
-      // coordinate past the pool, which TMA fills with zeros
-      auto page_of = [&](int ps) -> int {
-        const int w = ps >> 5, b = w & 1;
-        if (win_tag[b] != w) {
-          win_tag[b] = w;
-          const int i = (w << 5) + lane;
-          win_page[b] = (i < n_pages) ? __ldg(pages + i) : p.num_phys_pages;
-        }
-        return __shfl_sync(0xffffffffu, win_page[b], ps & 31);
+      const int pg_mask = (1 << p.pg_shift) - 1;
+      const bool small_pages = p.pg_shift == 6;          // 64-token pages: a tile spans two pages
+      // physical page of the shard's page slot; past the shard's last page the coordinate points
+      // beyond the pool and TMA fills zeros
+      auto fetch = [&](int slot_idx) -> int {
+        return (slot_idx < n_pages) ? __ldg(pages + slot_idx) : p.num_phys_pages;
       };
-      uint32_t cc = 0;      // chunks issued so far
+      uint32_t slot = 0, phase = 0, issued = 0;
       bool ok = true;
-      auto acquire = [&]() -> uint8_t* {          // lane 0 only
-        const uint32_t slot = cc % C::RING, ph = (cc / C::RING) & 1;
-        ok = ok && mbar_wait(&empty[slot], ph ^ 1, abort_flag);
-        if (ok) mbar_arrive_expect_tx(&full[slot], kChunkBytes);
-        return ring + slot * kChunkBytes;
-      };
-      auto load_k = [&](int tile) {
-        const int box_tok = is_resp ? 128 : p.box_tok_k;   // the response maps use 128-token boxes
-        const int nbox = 128 / box_tok;
-        int pg_id[2], off[2], tl[2];
-        for (int b = 0; b < nbox; ++b) {
-          const int tok = tile * 128 + b * box_tok;
-          if (is_resp) { pg_id[b] = 0; off[b] = tok; tl[b] = 0; }
-          else {
-            const int ps = tok / p.pg;
-            pg_id[b] = page_of(ps);
-            off[b] = tok % p.pg;
-            tl[b] = (ps == tail_slot);
-          }
+      auto acquire = [&]() -> uint8_t* {
+        ok = ok && LS_TWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
+        uint8_t* dst = ring + slot * C::CHUNK;
+        if (ok) {
+          if (no_loads) mbar_arrive(&full[slot]);
+          else mbar_arrive_expect_tx(&full[slot], C::CHUNK);
         }
-        if (lane == 0) {
-          for (int c = 0; c < C::KCH; ++c) {
-            uint8_t* dst = acquire();
-            if (ok) {
-              for (int b = 0; b < nbox; ++b) {
-                const CUtensorMap* m = is_resp ? &p.kr_map : (tl[b] ? &p.k_tail_map : &p.k_map);
-                tma_load_4d(dst + b * box_tok * 128, m, &full[cc % C::RING], c * 64, off[b], kvh, pg_id[b]);
+        return dst;
+      };
+      auto advance = [&]() {
+        ++issued;
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      // K of one tile: KCH chunks of 128 keys x (64 * KSLABS) channels
+      auto load_k = [&](int tile, int pa, int pb) {
+        const int tok = tile * 128;
+        for (int c = 0; c < C::KCH; ++c) {
+          uint8_t* dst = acquire();
+          if (ok && !no_loads) {
+            if (is_resp) {
+              tma_load_5d(dst, &p.kr_map, &full[slot], 0, tok, c * C::KSLABS, kvh, 0);
+            } else if (!small_pages) {
+              const CUtensorMap* m = ((tok >> p.pg_shift) == tail_slot) ? &p.k_tail_map : &p.k_map;
+              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, c * C::KSLABS, kvh, pa);
+            } else {
+              const int sa = tok >> 6;
+              const CUtensorMap* ma = (sa == tail_slot) ? &p.k_tail_map : &p.k_map;
+              const CUtensorMap* mb = (sa + 1 == tail_slot) ? &p.k_tail_map : &p.k_map;
+              for (int s = 0; s < C::KSLABS; ++s) {
+                tma_load_5d(dst + s * 16384, ma, &full[slot], 0, 0, c * C::KSLABS + s, kvh, pa);
+                tma_load_5d(dst + s * 16384 + 8192, mb, &full[slot], 0, 0, c * C::KSLABS + s, kvh, pb);
               }
             }
-            ++cc;
           }
+          advance();
         }
       };
-      auto load_v = [&](int tile) {
-        int pg_id[C::NVCH], off[C::NVCH], tl[C::NVCH];
+      // V of one tile: two chunks of 64 keys x DV channels
+      auto load_v = [&](int tile, int pa, int pb) {
         for (int r = 0; r < C::NVCH; ++r) {
-          const int tok = tile * 128 + r * C::VKEYS;
-          if (is_resp) { pg_id[r] = 0; off[r] = tok; tl[r] = 0; }
-          else {
-            const int ps = tok / p.pg;
-            pg_id[r] = page_of(ps);
-            off[r] = tok % p.pg;
-            tl[r] = (ps == tail_slot);
-          }
-        }
-        if (lane == 0) {
-          for (int r = 0; r < C::NVCH; ++r) {
-            uint8_t* dst = acquire();
-            if (ok) {
-              const CUtensorMap* m = is_resp ? &p.vr_map : (tl[r] ? &p.v_tail_map : &p.v_map);
-              for (int c = 0; c < DV / 64; ++c)
-                tma_load_4d(dst + c * C::VKEYS * 128, m, &full[cc % C::RING], c * 64, off[r], kvh, pg_id[r]);
+          uint8_t* dst = acquire();
+          if (ok && !no_loads) {
+            const int tok = tile * 128 + r * 64;
+            if (is_resp) {
+              tma_load_5d(dst, &p.vr_map, &full[slot], 0, tok, 0, kvh, 0);
+            } else {
+              const CUtensorMap* m = ((tok >> p.pg_shift) == tail_slot) ? &p.v_tail_map : &p.v_map;
+              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 0, kvh, (small_pages && r) ? pb : pa);
             }
-            ++cc;
           }
+          advance();
         }
       };
-      load_k(0);
-      for (int i = 0; i < n_tiles; ++i) {
-        if (i + 1 < n_tiles) load_k(i + 1);
-        load_v(i);
+      const long long t_begin_p = clock64();
+      // page ids of tile i: slots (128 i) >> pg_shift and, for 64-token pages, the next one
+      int pa0 = 0, pb0 = 0, pa1 = 0, pb1 = 0;
+      if (!is_resp) {
+        pa0 = fetch(0);
+        pb0 = small_pages ? fetch(1) : pa0;
+        if (n_tiles > 1) {
+          pa1 = fetch(128 >> p.pg_shift);
+          pb1 = small_pages ? fetch(3) : pa1;
+        }
       }
+      load_k(0, pa0, pb0);
+      for (int i = 0; i < n_tiles; ++i) {
+        int pa2 = 0, pb2 = 0;                       // prefetched two tiles ahead, used next iteration
+        if (!is_resp && i + 2 < n_tiles) {
+          const int s2 = ((i + 2) * 128) >> p.pg_shift;
+          pa2 = fetch(s2);
+          pb2 = small_pages ? fetch(s2 + 1) : pa2;
+        }
+        if (i + 1 < n_tiles) load_k(i + 1, pa1, pb1);
+        load_v(i, pa0, pb0);
+        pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
+      }
+      LS_TDUMP(0, tw0);
+      LS_TDUMP(1, clock64() - t_begin_p);
       // On an aborted run, wait (bounded) until every copy this thread started has landed.
-      if (lane == 0 && *abort_flag) {
-        for (uint32_t s = 0; s < (uint32_t)C::RING && s < cc; ++s) {
-          const uint32_t last = ((cc - 1 - s) / C::RING) * C::RING + s;   // last chunk index in slot s
+      if (*abort_flag) {
+        for (uint32_t s = 0; s < (uint32_t)C::RING && s < issued; ++s) {
+          const uint32_t last = ((issued - 1 - s) / C::RING) * C::RING + s;   // last chunk index in slot s
           const uint64_t t_start = globaltimer_ns();
-          while (!mbar_try_wait(&full[s], (last / C::RING) & 1) && globaltimer_ns() - t_start < 100000000ull) {
+          while (!mbar_try_wait(&full[s], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
           }
         }
       }
     }
   } else if (warp == 1) {
-    // =========================================================== MMA issuer
+    // =========================================================== MMA issuer (one thread)
     if (lane == 0 && n_tiles > 0) {
       constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);
       constexpr uint32_t idesc_pv = make_idesc(128, DV, 0, 1);
-      const uint32_t q_addr = smem_u32(q_smem);
-      const uint32_t ring_addr = smem_u32(ring);
-      uint32_t cc = 0;
+      constexpr uint32_t hi = sdesc_hi(1024);
+      const uint32_t q_lo = sdesc_lo(smem_u32(q_smem), 16);
+      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major chunk
+      const uint32_t ring_v_lo = sdesc_lo(smem_u32(ring), 8192);     // MN-major chunk: 8 KB sub-slab pitch
+      uint32_t slot = 0, phase = 0;
+      const bool no_mma = (p.ablate & LS_FLAG_ABLATE_MMA) != 0;
       bool ok = mbar_wait(q_full, 0, abort_flag);
+      const long long t_begin = clock64();
+      auto advance = [&]() {
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
       auto issue_s = [&](int tile) {
         const uint32_t d = tmem_s0 + (tile & 1) * 128;
+#pragma unroll
         for (int c = 0; c < C::KCH; ++c) {
-          const uint32_t slot = cc % C::RING, ph = (cc / C::RING) & 1;
-          ok = ok && mbar_wait(&full[slot], ph, abort_flag);
+          ok = ok && LS_TWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
           if (!ok) return;
           tc_fence_after();
-          const uint32_t a0 = q_addr + c * kChunkBytes, b0 = ring_addr + slot * kChunkBytes;
+          const uint32_t b_lo = ring_k_lo + slot * (C::CHUNK >> 4);
+          if (!no_mma) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            mma_ss(d, make_sdesc(a0 + k * 32, 16, 1024), make_sdesc(b0 + k * 32, 16, 1024), idesc_s,
-                   (c | k) != 0);
+            for (int s = 0; s < C::KSLABS; ++s)
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                mma_ss(d, sdesc(q_lo + (((c * C::KSLABS + s) * 16384 + k * 32) >> 4), hi),
+                       sdesc(b_lo + ((s * 16384 + k * 32) >> 4), hi), idesc_s, (c | s | k) != 0);
+          }
           mma_commit(&empty[slot]);
-          ++cc;
+          advance();
         }
         mma_commit(&s_full[tile & 1]);
       };
       auto issue_pv = [&](int tile) {
         const uint32_t a_base = tmem_s0 + (tile & 1) * 128;   // P over the S columns
+#pragma unroll
         for (int r = 0; r < C::NVCH; ++r) {
-          const uint32_t slot = cc % C::RING, ph = (cc / C::RING) & 1;
-          ok = ok && mbar_wait(&full[slot], ph, abort_flag);
+          ok = ok && LS_TWAIT(tw1, mbar_wait(&full[slot], phase, abort_flag));
           if (!ok) return;
           tc_fence_after();
-          const uint32_t b0 = ring_addr + slot * kChunkBytes;
+          const uint32_t b_lo = ring_v_lo + slot * (C::CHUNK >> 4);
+          if (!no_mma) {
 #pragma unroll
-          for (int kk = 0; kk < C::VKEYS / 16; ++kk)
-            mma_ts(tmem_o, a_base + (r * (C::VKEYS / 16) + kk) * 8, make_sdesc(b0 + kk * 2048, C::VKEYS * 128, 1024),
-                   idesc_pv, (tile | r | kk) != 0);
+            for (int kk = 0; kk < 4; ++kk)
+              mma_ts(tmem_o, a_base + (r * 4 + kk) * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi), idesc_pv,
+                     (tile | r | kk) != 0);
+          }
           mma_commit(&empty[slot]);
-          ++cc;
+          advance();
         }
         mma_commit(pv_done);
         if (tile == n_tiles - 1) mma_commit(o_final);
@@ -261,11 +302,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       if (ok) issue_s(0);
       for (int i = 0; i < n_tiles && ok; ++i) {
         if (i + 1 < n_tiles) issue_s(i + 1);
-        ok = ok && mbar_wait(&p_full[i & 1], (i >> 1) & 1, abort_flag);
+        ok = ok && LS_TWAIT(tw2, mbar_wait(&p_full[i & 1], (i >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         issue_pv(i);
       }
+      LS_TDUMP(8, tw0);
+      LS_TDUMP(9, tw1);
+      LS_TDUMP(10, tw2);
+      LS_TDUMP(11, clock64() - t_begin);
     }
   } else {
     // =========================================================== softmax + epilogue
@@ -284,13 +329,19 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       // last visible key index of this row inside this partial
       const int64_t lim = is_resp ? (int64_t)min(t, p.R - 1) : tokens - 1;
       float m_ref = -INFINITY, l = 0.f;
+      const long long t_begin_sm = clock64();
       const float thresh = kRescaleLog2 / p.scale_log2;
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
         const uint32_t ts = tmem_s0 + (i & 1) * 128 + lane_sel;
-        ok = mbar_wait(&s_full[i & 1], (i >> 1) & 1, abort_flag);
+        ok = LS_TWAIT(tw0, mbar_wait(&s_full[i & 1], (i >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
+        if (p.ablate & LS_FLAG_ABLATE_SOFTMAX) {
+          tc_fence_before();
+          mbar_arrive(&p_full[i & 1]);
+          continue;
+        }
         uint32_t sr[128];
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(ts + c * 32, sr + c * 32);
@@ -316,7 +367,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           m_ref = (mx == -INFINITY) ? 0.f : mx;
         } else if (__any_sync(0xffffffffu, mx > m_ref + thresh)) {
           // rare: raise the reference maximum and rescale the running sum and O
-          ok = mbar_wait(pv_done, (i - 1) & 1, abort_flag);
+          ok = LS_TWAIT(tw1, mbar_wait(pv_done, (i - 1) & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
           const float m_new = fmaxf(m_ref, mx);
@@ -353,6 +404,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         mbar_arrive(&p_full[i & 1]);
       }
       // (pv_done may still be two phases behind here, where a parity wait would alias)
+      if (threadIdx.x == 64) {
+        LS_TDUMP(16, tw0);
+        LS_TDUMP(17, tw1);
+        LS_TDUMP(18, clock64() - t_begin_sm);
+      }
       if (ok) ok = mbar_wait(o_final, 0, abort_flag);
       if (ok) {
         tc_fence_after();
@@ -427,21 +483,22 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
 
   ls::FwdParams P;
   const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads;
-  const int vkeys = 8192 / d.dim_v;
-  const int box_k = d.page_size >= 128 ? 128 : 64;
-  ls_status_t st = ls::encode_map(&P.q_map, q, d.dim_k, R, Hq, 1, (int64_t)Hq * d.dim_k, d.dim_k,
-                                  (int64_t)R * Hq * d.dim_k, 128);
+  const int kslabs = d.dim_k == 256 ? 2 : 1;
+  const bool small_pages = d.page_size == 64;
+  ls_status_t st = ls::encode_map5(&P.q_map, q, d.dim_k, R, Hq, 1, (int64_t)Hq * d.dim_k, d.dim_k,
+                                   (int64_t)R * Hq * d.dim_k, 128, kslabs);
   if (st == LS_OK)
-    st = ls::encode_map(&P.kr_map, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k,
-                        (int64_t)R * Hkv * d.dim_k, 128);
+    st = ls::encode_map5(&P.kr_map, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k,
+                         (int64_t)R * Hkv * d.dim_k, 128, kslabs);
   if (st == LS_OK)
-    st = ls::encode_map(&P.vr_map, v_resp, d.dim_v, R, Hkv, 1, (int64_t)Hkv * d.dim_v, d.dim_v,
-                        (int64_t)R * Hkv * d.dim_v, vkeys);
+    st = ls::encode_map5(&P.vr_map, v_resp, d.dim_v, R, Hkv, 1, (int64_t)Hkv * d.dim_v, d.dim_v,
+                         (int64_t)R * Hkv * d.dim_v, 64, d.dim_v / 64);
+  const int kbox = small_pages ? 64 : 128, kgroups = small_pages ? 1 : kslabs;
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.k_map, h, 0, kbox, kgroups, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.k_tail_map, h, 0, kbox, kgroups, true);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_map, h, 1, 64, d.dim_v / 64, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_tail_map, h, 1, 64, d.dim_v / 64, true);
   if (st != LS_OK) return st;
-  P.k_map = h->k_maps.full[ls::box_index(box_k)];
-  P.k_tail_map = h->k_maps.tail[ls::box_index(box_k)];
-  P.v_map = h->v_maps.full[ls::box_index(vkeys)];
-  P.v_tail_map = h->v_maps.tail[ls::box_index(vkeys)];
   P.shard_phys_pages = h->d_shard_phys_pages;
   P.shard_page_offset = h->d_shard_page_offset;
   P.shard_tail_slot = h->d_shard_tail_slot;
@@ -454,11 +511,11 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.Hkv = Hkv;
   P.g = Hq / Hkv;
   P.S = d.num_shards;
-  P.pg = d.page_size;
-  P.box_tok_k = box_k;
+  P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 127) / 128;
   P.nq_tiles = P.g * P.tiles_per_head;
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
+  P.ablate = prm->flags & LS_FLAG_ABLATE_MASK;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * 1.4426950408889634f;
   const int64_t grid = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;

@@ -68,6 +68,17 @@ inline void profile_end(int k, cudaStream_t st) {
   g_profile[k].start = g_profile[k].stop = nullptr;
 }
 
+// Rank-5 view (64 channels, token, channel group, head, page) with a box of
+// 64 x box_tok x box_groups: one TMA instruction fills box_groups swizzled slabs.
+ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok, int64_t dim_head,
+                        int64_t dim_page, int64_t stride_tok, int64_t stride_head, int64_t stride_page,
+                        int box_tok, int box_groups);
+
+// The pool's K (which = 0) or V (which = 1) map for the given box; tail = bounded to the valid
+// tokens of the partially filled last logical page.
+ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
+                             bool tail);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace ls

@@ -45,6 +45,40 @@ ls_status_t encode_map(CUtensorMap* out, const void* base, int64_t dim_d, int64_
   return r == CUDA_SUCCESS ? LS_OK : LS_ERR_CUDA;
 }
 
+ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok, int64_t dim_head,
+                        int64_t dim_page, int64_t stride_tok, int64_t stride_head, int64_t stride_page,
+                        int box_tok, int box_groups) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return LS_ERR_CUDA;
+  if (!aligned16(base)) return LS_ERR_ALIGNMENT;
+  if ((stride_tok * 2) % 16 || (stride_head * 2) % 16 || (stride_page * 2) % 16 || dim_d % 64) return LS_ERR_ALIGNMENT;
+  cuuint64_t dims[5] = {64, (cuuint64_t)dim_tok, (cuuint64_t)(dim_d / 64), (cuuint64_t)dim_head,
+                        (cuuint64_t)dim_page};
+  cuuint64_t strides[4] = {(cuuint64_t)stride_tok * 2, 128, (cuuint64_t)stride_head * 2,
+                           (cuuint64_t)stride_page * 2};
+  cuuint32_t box[5] = {64, (cuuint32_t)box_tok, (cuuint32_t)box_groups, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LS_OK : LS_ERR_CUDA;
+}
+
+ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
+                             bool tail) {
+  const ls_pages_desc_t& d = h->desc;
+  const bool v = which == 1;
+  const bool alias = v && d.v_aliases_k;
+  const void* base = (v && !alias) ? d.v_pool : d.k_pool;
+  const int64_t s_tok = (v && !alias) ? d.v_stride_tok : d.k_stride_tok;
+  const int64_t s_head = (v && !alias) ? d.v_stride_head : d.k_stride_head;
+  const int64_t s_page = (v && !alias) ? d.v_stride_page : d.k_stride_page;
+  const int64_t dim = v ? d.dim_v : d.dim_k;
+  const int64_t tok = tail && h->last_valid > 0 ? h->last_valid : d.page_size;
+  return encode_map5(out, base, dim, tok, d.num_kv_heads, std::max<int64_t>(d.num_phys_pages, 1), s_tok, s_head,
+                     s_page, std::min<int>(box_tok, d.page_size), box_groups);
+}
+
 static void even_chunks(int64_t n, int64_t parts, std::vector<int64_t>& bounds) {
   bounds.assign(parts + 1, 0);
   int64_t base = n / parts, rem = n % parts;
