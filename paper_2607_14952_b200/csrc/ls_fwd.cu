@@ -13,9 +13,13 @@
 //   warps 2-5  softmax: one thread per query row (TMEM lane); online softmax with a lazily
 //           updated reference maximum, P written back to TMEM as bf16 over the S columns
 //
-// TMEM columns: O [0, DV), S/P buffer 0 [DV, DV+128), S/P buffer 1 [DV+128, DV+256).
-// K chunk  = 128 keys x 64 channels (K-major, 128-byte swizzle): one k-slice of S.
-// V chunk  = VKEYS keys x DV channels as DV/64 sub-slabs (MN-major): VKEYS/16 k-steps of PV.
+// A CTA owns DVT output channels (all of them for head dims 128 and 256).  The shared-latent
+// shape (576/512, V = first 512 channels of the K page) runs as two work items per Q tile,
+// one per 256-channel half of O, because O alone would fill all 512 TMEM columns.
+//
+// TMEM columns: O [0, DVT), S/P buffer 0 [DVT, DVT+128), S/P buffer 1 [DVT+128, DVT+256).
+// K chunk  = 128 keys x 64*KSLABS channels (K-major, 128-byte swizzle): k-slices of S.
+// V chunk  = VKEYS keys x DVT channels as DVT/64 sub-slabs (MN-major): VKEYS/16 k-steps of PV.
 #include "ls_internal.h"
 #include "ls_sm100.cuh"
 
@@ -34,6 +38,7 @@ struct FwdParams {
   float* lse_part;
   int32_t* status;
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  int dv_total;   // channels of one output row (DVT times the number of O tiles)
   int ablate;   // diagnostic: LS_FLAG_ABLATE_* bits (results are then meaningless)
   float scale, scale_log2;
 };
@@ -51,24 +56,24 @@ struct FwdParams {
 constexpr int kFwdThreads = 192;
 constexpr float kRescaleLog2 = 8.0f;   // the reference max lags the true max by at most 2^8
 
-template <int DK, int DV>
+template <int DK, int DVT>
 struct FwdCfg {
-  static_assert(DK == DV, "the shared-latent (576/512) variant has its own kernel");
   static constexpr int CHUNK = (DK == 256) ? 32768 : 16384;   // bytes per ring slot
   static constexpr int KSLABS = CHUNK / 16384;     // 64-channel slabs (128 keys x 128 B) per K chunk
   static constexpr int KCH = (DK / 64) / KSLABS;   // K chunks per 128-key tile
-  static constexpr int VKEYS = 64;                 // keys per V chunk
+  static constexpr int VKEYS = CHUNK / (DVT * 2);  // keys per V chunk
   static constexpr int NVCH = 128 / VKEYS;         // V chunks per tile
-  static constexpr int VSUB = DV / 64;             // 8 KB sub-slabs (64 keys x 128 B) per V chunk
-  static_assert(VSUB * 8192 == CHUNK, "a V chunk fills one ring slot");
-  static constexpr int RING = (DK == 256) ? 4 : 10;
+  static constexpr int VSUB = DVT / 64;            // sub-slabs (VKEYS rows x 128 B) per V chunk
+  static_assert(VSUB * VKEYS * 128 == CHUNK && VKEYS % 16 == 0 && VKEYS <= 64, "a V chunk fills one ring slot");
+  static constexpr int RING = (DK == 256) ? 4 : (DK == 128) ? 10 : 5;
   static constexpr int Q_BYTES = (DK / 64) * 16384;
   static constexpr int SMEM_BYTES = 1024 + Q_BYTES + RING * CHUNK + 512;
 };
 
-template <int DK, int DV>
+template <int DK, int DVT, int NDV>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_constant__ FwdParams p) {
-  using C = FwdCfg<DK, DV>;
+  using C = FwdCfg<DK, DVT>;
+  constexpr int DV = DVT;   // O columns held by this CTA
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = smem;
@@ -90,6 +95,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 
   // ---- work item
   int idx = blockIdx.x;
+  const int dvh = idx % NDV;            // which DVT-wide slice of the value channels
+  idx /= NDV;
   const int qtile = idx % p.nq_tiles;
   idx /= p.nq_tiles;
   const int part = idx % (p.S + 1);
@@ -191,17 +198,18 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           advance();
         }
       };
-      // V of one tile: two chunks of 64 keys x DV channels
+      // V of one tile: NVCH chunks of VKEYS keys x DVT channels (channel groups dvh*VSUB ..)
       auto load_v = [&](int tile, int pa, int pb) {
         for (int r = 0; r < C::NVCH; ++r) {
           uint8_t* dst = acquire();
           if (ok && !no_loads) {
-            const int tok = tile * 128 + r * 64;
+            const int tok = tile * 128 + r * C::VKEYS;
             if (is_resp) {
-              tma_load_5d(dst, &p.vr_map, &full[slot], 0, tok, 0, kvh, 0);
+              tma_load_5d(dst, &p.vr_map, &full[slot], 0, tok, dvh * C::VSUB, kvh, 0);
             } else {
               const CUtensorMap* m = ((tok >> p.pg_shift) == tail_slot) ? &p.v_tail_map : &p.v_map;
-              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 0, kvh, (small_pages && r) ? pb : pa);
+              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, dvh * C::VSUB, kvh,
+                          (small_pages && r * C::VKEYS >= 64) ? pb : pa);
             }
           }
           advance();
@@ -250,7 +258,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       constexpr uint32_t hi = sdesc_hi(1024);
       const uint32_t q_lo = sdesc_lo(smem_u32(q_smem), 16);
       const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major chunk
-      const uint32_t ring_v_lo = sdesc_lo(smem_u32(ring), 8192);     // MN-major chunk: 8 KB sub-slab pitch
+      const uint32_t ring_v_lo = sdesc_lo(smem_u32(ring), C::VKEYS * 128);   // MN-major chunk: sub-slab pitch
       uint32_t slot = 0, phase = 0;
       const bool no_mma = (p.ablate & LS_FLAG_ABLATE_MMA) != 0;
       bool ok = mbar_wait(q_full, 0, abort_flag);
@@ -289,9 +297,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           const uint32_t b_lo = ring_v_lo + slot * (C::CHUNK >> 4);
           if (!no_mma) {
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              mma_ts(tmem_o, a_base + (r * 4 + kk) * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi), idesc_pv,
-                     (tile | r | kk) != 0);
+            for (int kk = 0; kk < C::VKEYS / 16; ++kk)
+              mma_ts(tmem_o, a_base + (r * (C::VKEYS / 16) + kk) * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi),
+                     idesc_pv, (tile | r | kk) != 0);
           }
           mma_commit(&empty[slot]);
           advance();
@@ -319,11 +327,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     const int t = t0 + row;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const size_t out_row = ((size_t)part * p.R + (size_t)min(t, p.R - 1)) * p.Hq + h;
-    float* o_dst = p.o_part + out_row * DV;
+    float* o_dst = p.o_part + out_row * p.dv_total + dvh * DVT;
     if (n_tiles == 0) {
       if (t < p.R) {
         for (int c = 0; c < DV; c += 4) *reinterpret_cast<float4*>(o_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-        p.lse_part[out_row] = -INFINITY;
+        if (dvh == 0) p.lse_part[out_row] = -INFINITY;
       }
     } else {
       // last visible key index of this row inside this partial
@@ -426,7 +434,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                               __uint_as_float(o[j + 2]) * inv_l, __uint_as_float(o[j + 3]) * inv_l);
           }
         }
-        if (t < p.R) p.lse_part[out_row] = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
+        if (t < p.R && dvh == 0) p.lse_part[out_row] = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
       }
     }
   }
@@ -440,18 +448,19 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
 }
 
-template <int DK, int DV>
-static ls_status_t launch_fwd(const FwdParams& prm, int grid, cudaStream_t st) {
-  using C = FwdCfg<DK, DV>;
+template <int DK, int DVT, int NDV>
+static ls_status_t launch_fwd(const FwdParams& prm, int64_t grid, cudaStream_t st) {
+  using C = FwdCfg<DK, DVT>;
   static bool configured = false;
+  if (grid * NDV > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   if (!configured) {
-    if (cudaFuncSetAttribute(fwd_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(fwd_kernel<DK, DVT, NDV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::SMEM_BYTES) != cudaSuccess)
       return LS_ERR_CUDA;
     configured = true;
   }
   profile_begin(LS_KERNEL_FWD, st);
-  fwd_kernel<DK, DV><<<grid, kFwdThreads, C::SMEM_BYTES, st>>>(prm);
+  fwd_kernel<DK, DVT, NDV><<<(int)(grid * NDV), kFwdThreads, C::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_FWD, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
@@ -479,11 +488,15 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;
   if (!ls::aligned16(q) || !ls::aligned16(k_resp) || !ls::aligned16(v_resp) || !ls::aligned16(o_part))
     return LS_ERR_ALIGNMENT;
-  if (!((d.dim_k == 128 && d.dim_v == 128) || (d.dim_k == 256 && d.dim_v == 256))) return LS_ERR_UNSUPPORTED_SHAPE;
+  const bool mla = d.dim_k == 576 && d.dim_v == 512;
+  if (!((d.dim_k == 128 && d.dim_v == 128) || (d.dim_k == 256 && d.dim_v == 256) || mla))
+    return LS_ERR_UNSUPPORTED_SHAPE;
 
   ls::FwdParams P;
   const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads;
   const int kslabs = d.dim_k == 256 ? 2 : 1;
+  const int dvt = mla ? 256 : d.dim_v;                    // O channels per CTA
+  const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
   const bool small_pages = d.page_size == 64;
   ls_status_t st = ls::encode_map5(&P.q_map, q, d.dim_k, R, Hq, 1, (int64_t)Hq * d.dim_k, d.dim_k,
                                    (int64_t)R * Hq * d.dim_k, 128, kslabs);
@@ -492,12 +505,12 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
                          (int64_t)R * Hkv * d.dim_k, 128, kslabs);
   if (st == LS_OK)
     st = ls::encode_map5(&P.vr_map, v_resp, d.dim_v, R, Hkv, 1, (int64_t)Hkv * d.dim_v, d.dim_v,
-                         (int64_t)R * Hkv * d.dim_v, 64, d.dim_v / 64);
+                         (int64_t)R * Hkv * d.dim_v, vkeys, dvt / 64);
   const int kbox = small_pages ? 64 : 128, kgroups = small_pages ? 1 : kslabs;
   if (st == LS_OK) st = ls::encode_pool_map5(&P.k_map, h, 0, kbox, kgroups, false);
   if (st == LS_OK) st = ls::encode_pool_map5(&P.k_tail_map, h, 0, kbox, kgroups, true);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_map, h, 1, 64, d.dim_v / 64, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_tail_map, h, 1, 64, d.dim_v / 64, true);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_map, h, 1, vkeys, dvt / 64, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_tail_map, h, 1, vkeys, dvt / 64, true);
   if (st != LS_OK) return st;
   P.shard_phys_pages = h->d_shard_phys_pages;
   P.shard_page_offset = h->d_shard_page_offset;
@@ -515,12 +528,13 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.tiles_per_head = (R + 127) / 128;
   P.nq_tiles = P.g * P.tiles_per_head;
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
+  P.dv_total = d.dim_v;
   P.ablate = prm->flags & LS_FLAG_ABLATE_MASK;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * 1.4426950408889634f;
   const int64_t grid = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;
-  if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (d.dim_k == 128) return ls::launch_fwd<128, 128>(P, (int)grid, cs);
-  return ls::launch_fwd<256, 256>(P, (int)grid, cs);
+  if (mla) return ls::launch_fwd<576, 256, 2>(P, grid, cs);
+  if (d.dim_k == 128) return ls::launch_fwd<128, 128, 1>(P, grid, cs);
+  return ls::launch_fwd<256, 256, 1>(P, grid, cs);
 }

@@ -32,6 +32,9 @@ def test_config1_tiny_full():
     small("d128_small_p", Dk=128, Dv=128, P=50, page_size=64, num_shards=2, R=64),   # prefix below one tile
     small("d256_empty_shards", P=512, page_size=256, num_shards=5),      # S > Np leaves empty partials
     small("d256_p0", P=0, num_shards=2, R=300),                          # pure causal response block
+    # shared-latent shape: 576-wide key page whose first 512 channels are the value
+    small("mla_pg64", Dk=576, Dv=512, v_aliases_k=True, Hq=8, Hkv=1, P=64 * 20 + 5, page_size=64, num_shards=3, R=130),
+    small("mla_pg256", Dk=576, Dv=512, v_aliases_k=True, Hq=4, Hkv=1, P=2048, page_size=256, num_shards=2, R=256),
 ], ids=lambda c: c.name)
 def test_forward_small_cases(cfg):
     case = parity.Case(cfg, extra_phys_pages=2)
