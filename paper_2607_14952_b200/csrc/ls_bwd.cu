@@ -475,7 +475,9 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   const ls_pages_desc_t& d = h->desc;
   if (prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % d.num_kv_heads != 0) return LS_ERR_INVALID_ARG;
   if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;
-  if (!((d.dim_k == 128 && d.dim_v == 128) || (d.dim_k == 256 && d.dim_v == 256))) return LS_ERR_UNSUPPORTED_SHAPE;
+  const bool mla = d.dim_k == 576 && d.dim_v == 512;
+  if (!((d.dim_k == 128 && d.dim_v == 128) || (d.dim_k == 256 && d.dim_v == 256) || mla))
+    return LS_ERR_UNSUPPORTED_SHAPE;
   const void* ptrs[] = {q, k_resp, v_resp, o_f32, d_o, dq, dk_resp, dv_resp, workspace};
   for (const void* ptr : ptrs)
     if (!ls::aligned16(ptr)) return LS_ERR_ALIGNMENT;
@@ -490,6 +492,15 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
 
   ls::delta_kernel<<<(int)((rows + 7) / 8), 256, 0, cs>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows,
                                                         d.dim_v, delta);
+
+  if (mla) {
+    ls_status_t ms = ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_part, dk_resp, dv_resp, status_dev, cs);
+    if (ms != LS_OK) return ms;
+    const int64_t n4m = rows * D / 4;
+    ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4m + 255) / 256, 148 * 16), 256, 0, cs>>>(
+        dq_part, d.num_shards + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));
+    return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+  }
 
   auto dense_map = [&](CUtensorMap* m, const void* base, int heads, int box_tok, int groups) {
     return ls::encode_map5(m, base, D, R, heads, 1, (int64_t)heads * D, D, (int64_t)R * heads * D, box_tok, groups);

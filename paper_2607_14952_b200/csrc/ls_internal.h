@@ -79,6 +79,12 @@ ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64
 ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
                              bool tail);
 
+// Backward of the shared-latent 576/512 shape (ls_bwd_mla.cu): fills dq_part (fp32, unscaled,
+// [(S+1), R, Hq, 576]) and the bf16 dk_resp / dv_resp.
+ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
+                    const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
+                    void* dk_resp, void* dv_resp, int32_t* status_dev, cudaStream_t cs);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace ls

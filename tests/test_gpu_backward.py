@@ -35,12 +35,18 @@ def test_config1_tiny_full():
     # P = 0: pure causal self-attention, where dK/dV are O(1) and the absolute tolerance bites
     small("d256_p0", P=0, num_shards=2, R=300),
     small("d128_p0", Dk=128, Dv=128, P=0, num_shards=1, R=257, Hq=2, Hkv=1, page_size=64),
+    # shared-latent shape: 576-wide key page whose first 512 channels are the value
+    small("mla_pg64", Dk=576, Dv=512, v_aliases_k=True, Hq=8, Hkv=1, P=64 * 20 + 5, page_size=64, num_shards=3, R=130),
+    small("mla_pg256", Dk=576, Dv=512, v_aliases_k=True, Hq=4, Hkv=1, P=2048, page_size=256, num_shards=2, R=256),
+    small("mla_p0", Dk=576, Dv=512, v_aliases_k=True, Hq=2, Hkv=1, P=0, page_size=64, num_shards=1, R=200),
 ], ids=lambda c: c.name)
 def test_backward_small_cases(cfg):
     case = parity.Case(cfg, extra_phys_pages=2)
     before = B.ls_prefix_pages_checksum(case.pages)
     fw = parity.check_forward(case, per_shard=False)
-    parity.check_backward(case, fw)
+    # with P = 0 the first rows see one or two keys: ds = p (dp - Delta) cancels to ~0 and what is
+    # left is the fp32 rounding of two 512-term dot products, a few 1e-4 against a reference of 0
+    parity.check_backward(case, fw, rel_slack=2.0 if (cfg.P == 0 and cfg.Dk == 576) else 1.0)
     assert B.ls_prefix_pages_checksum(case.pages) == before      # the prefix is read-only
 
 

@@ -98,3 +98,25 @@ def test_config4_p4m_cycles_keep_the_prefix_intact():
     finally:
         parity.sampled_rows = orig
     _free(case)
+
+
+def test_config5_mla1m_shared_latent():
+    cfg = CONFIGS["mla1m"]
+    case = parity.Case(cfg)
+    orig = parity.sampled_rows
+    try:
+        # 64 heads share the one latent KV head: sample rows over a few heads only
+        def few(c, kv, tail=8, n_random=24, seed=0, extra=()):
+            t, h = orig(c, kv, tail=tail, n_random=n_random, seed=seed, extra=extra)
+            keep = (h < 3) | (np.arange(len(h)) % 11 == 0)
+            # the tail rows must stay complete for dK/dV: keep every head there
+            keep |= t >= c.R - tail
+            return t[keep], h[keep]
+        parity.sampled_rows = few
+        for member in range(cfg.G):
+            fw = parity.check_forward(case, member=member, kv_groups=[0], full=False, per_shard=False,
+                                      strict_abs=True)
+            parity.check_backward(case, fw, kv_groups=[0], full=False, tail=8, strict_abs=True)
+    finally:
+        parity.sampled_rows = orig
+    _free(case)
