@@ -6,11 +6,13 @@
 //   dK_j  = scale * sum_{t>=j,h} ds_tj q_th,   dV_j = sum_{t>=j,h} p_tj dO_th   (response keys only)
 //
 // One row-stationary kernel serves all three gradients.  A CTA keeps 128 "rows" resident in
-// shared memory (operands A1, A2) and streams 64-wide "column" tiles through a ring of
-// 16 KB chunks:
-//     S = A1 B1^T,  T = A2 B2^T      (tcgen05.mma, operands in shared memory, K-major)
-//     E = f(S, T)                     (one thread per row, bf16 written over S in TMEM)
-//     ACC += E B3                     (E read from TMEM, B3 MN-major from shared memory)
+// shared memory (operands A1, A2) and streams 128-wide "column" tiles through a small ring of
+// chunks (128 columns x 128 channels each):
+//     S = A1 B1^T,  T = A2 B2^T      (tcgen05.mma 128x128x16, operands in shared memory)
+//     E = f(S, T)                     (one thread per row; bf16, written over S in TMEM,
+//                                      in four 32-column quarters, each with its own barrier)
+//     ACC += E B3                     (E read from TMEM, B3 MN-major from shared memory; the
+//                                      MMAs of a quarter start as soon as that quarter is ready)
 //   mode DQ: rows = 128 queries of one head, columns = keys of one partial (prefix shard
 //            through the page table, or the causal response block); A1 = Q, A2 = dO,
 //            B1 = B3 = K, B2 = V; E = p (T - Delta_row).  The prefix needs no dK/dV, so this
@@ -18,7 +20,9 @@
 //   mode DK: rows = 128 response keys, columns = queries (t >= j) of every head of the group;
 //            A1 = K_resp, A2 = V_resp, B1 = B3 = Q, B2 = dO; E = p (T - Delta_col).
 //   mode DV: as DK without T; B3 = dO; E = p.
-// TMEM columns: ACC [0, D), then two buffers of (S 64 | T 64).
+// The 128-wide tile halves how often the resident operand is re-read from shared memory per
+// key (a 64-wide S/T MMA is bound by that re-read, not by the tensor pipe).  It leaves TMEM
+// room for one S and one T buffer only: ACC [0, D), S [D, D+128), T [D+128, D+256).
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -32,7 +36,8 @@ enum { MODE_DQ = 0, MODE_DK = 1, MODE_DV = 2 };
 
 struct BwdParams {
   CUtensorMap a1_map, a2_map;                 // stationary rows: box 64 x 128 tokens x 1 group
-  // streamed 64-column chunks, box 64 x 64 tokens x D/64 groups
+  // streamed chunks of 128 columns x 128 channels: box 64 x 128 tokens x 2 groups, or, when the
+  // pages hold 64 tokens, 64 x 64 x 1 (four boxes per chunk)
   CUtensorMap bk_map, bk_tail, bv_map, bv_tail;   // prefix pool K and V (mode DQ)
   CUtensorMap b1r_map, b2r_map, b3r_map;          // dense sources: response K/V/K (DQ) or Q/dO/(Q|dO) (DK, DV)
   const int32_t* shard_phys_pages;
@@ -48,16 +53,25 @@ struct BwdParams {
   float scale, scale_log2;
 };
 
-constexpr int kBwdThreads = 192;
+#ifdef LS_TIMING
+#define LS_BTWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
+#define LS_BTDUMP(slot, val) do { if (MODE == MODE_DQ && blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
+#else
+#define LS_BTWAIT(acc, expr) (expr)
+#define LS_BTDUMP(slot, val) do { } while (0)
+#endif
+
+constexpr int kBwdThreads = 320;        // producer warp, MMA warp, 8 elementwise warps (2 threads per row)
+constexpr int kBwdChunk = 32768;        // 128 columns x 128 channels
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
 struct BwdCfg {
-  static constexpr int SLABS = D / 64;            // 64-channel groups
-  static constexpr int CHUNK = 64 * D * 2;        // one streamed chunk: 64 columns x D channels
-  static constexpr int RING = (D == 128) ? 8 : 3;
+  static constexpr int SLABS = D / 64;            // 64-channel groups of the resident operands
+  static constexpr int NC = D / 128;              // chunks per streamed operand and tile
+  static constexpr int RING = (D == 128) ? 4 : 3;
   static constexpr int A_BYTES = 2 * SLABS * 16384;
-  static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * CHUNK + 512;
+  static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * kBwdChunk + 512;
 };
 
 template <int D, int MODE>
@@ -69,17 +83,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   uint8_t* a1_smem = smem;
   uint8_t* a2_smem = smem + C::SLABS * 16384;
   uint8_t* ring = smem + C::A_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * C::CHUNK);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kBwdChunk);
   uint64_t* a_full = bars;
   uint64_t* full = bars + 1;
   uint64_t* empty = full + C::RING;
-  uint64_t* st_full = empty + C::RING;   // [2] S (and T) of a tile are in TMEM
-  uint64_t* e_full = st_full + 2;        // [2] E of a tile is in TMEM
-  uint64_t* acc_final = e_full + 2;
+  uint64_t* s_full = empty + C::RING;    // S of a tile is in TMEM
+  uint64_t* t_full = s_full + 1;         // T of a tile is in TMEM (S only in mode DV)
+  uint64_t* e_full = t_full + 1;         // [4] quarter q of E is in TMEM
+  uint64_t* acc_final = e_full + 4;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
+  (void)tw0; (void)tw1; (void)tw2;
+  const long long t_kernel = clock64();
+  (void)t_kernel;
 
   // ---- work item
   int part = 0, kvh, h = 0, row0;          // row0: first query (DQ) or first key (DK, DV) of the tile
@@ -87,7 +106,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   int64_t tokens = 0;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   int n_tiles;
-  int tt_min = 0, n_tt = 0;                // DK/DV: first 64-query tile and tiles per head
+  int tt_min = 0, n_tt = 0;                // DK/DV: first 128-query tile and tiles per head
   if (MODE == MODE_DQ) {
     int idx = blockIdx.x;
     const int qtile = idx % p.nq_tiles;
@@ -105,12 +124,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       n_pages = p.shard_page_offset[part + 1] - page_off;
       tail_slot = p.shard_tail_slot[part];
     }
-    n_tiles = (int)((tokens + 63) / 64);
+    n_tiles = (int)((tokens + 127) / 128);
   } else {
     kvh = blockIdx.x / p.tiles_per_head;
     row0 = (blockIdx.x % p.tiles_per_head) * 128;
-    tt_min = row0 / 64;
-    n_tt = (p.R + 63) / 64 - tt_min;
+    tt_min = row0 / 128;
+    n_tt = p.tiles_per_head - tt_min;
     n_tiles = p.g * n_tt;
   }
 
@@ -120,10 +139,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], 1);
     }
-    mbar_init(&st_full[0], 1);
-    mbar_init(&st_full[1], 1);
-    mbar_init(&e_full[0], 128);
-    mbar_init(&e_full[1], 128);
+    mbar_init(s_full, 1);
+    mbar_init(t_full, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 256);
     mbar_init(acc_final, 1);
     *abort_flag = 0;
     fence_barrier_init();
@@ -137,7 +155,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
   const uint32_t tmem_acc = tmem_base;
-  const uint32_t tmem_buf0 = tmem_base + D;
+  const uint32_t tmem_s = tmem_base + D;
+  const uint32_t tmem_t = tmem_base + D + 128;
 
   if (warp == 0) {
     // =========================================================== producer (one thread)
@@ -151,54 +170,67 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       const int32_t* pages = p.shard_phys_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
       const bool dense = (MODE != MODE_DQ) || is_resp;
-      auto fetch = [&](int tile) -> int {     // physical page of column tile `tile` (prefix shards only)
-        const int ps = (tile * 64) >> p.pg_shift;
-        return (!dense && tile < n_tiles && ps < n_pages) ? __ldg(pages + ps) : 0;
+      const bool small_pages = !dense && p.pg_shift == 6;   // a 128-key tile spans two 64-token pages
+      auto fetch = [&](int ps) -> int {      // physical page of the shard's page slot (prefix shards only)
+        if (dense) return 0;
+        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
       };
       uint32_t slot = 0, phase = 0, issued = 0;
       bool ok = true;
-      // one chunk: 64 columns x D channels of source `which` (0: B1, 1: B2, 2: B3) of column tile i
-      auto load = [&](int which, int i, int page) {
-        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
+      // one chunk: 128 columns x channels [128 c, 128 c + 128) of source `which` (0: B1, 1: B2, 2: B3)
+      auto load = [&](int which, int i, int c, int pa, int pb) {
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
         if (ok) {
-          mbar_arrive_expect_tx(&full[slot], C::CHUNK);
-          uint8_t* dst = ring + slot * C::CHUNK;
+          mbar_arrive_expect_tx(&full[slot], kBwdChunk);
+          uint8_t* dst = ring + slot * kBwdChunk;
           if (MODE == MODE_DQ) {
-            const int tok = i * 64;
+            const int tok = i * 128;
             if (is_resp) {
-              tma_load_5d(dst, which == 1 ? &p.b2r_map : &p.b1r_map, &full[slot], 0, tok, 0, kvh, 0);
-            } else {
+              tma_load_5d(dst, which == 1 ? &p.b2r_map : &p.b1r_map, &full[slot], 0, tok, 2 * c, kvh, 0);
+            } else if (!small_pages) {
               const bool tail = (tok >> p.pg_shift) == tail_slot;
               const CUtensorMap* m = which == 1 ? (tail ? &p.bv_tail : &p.bv_map) : (tail ? &p.bk_tail : &p.bk_map);
-              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 0, kvh, page);
+              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 2 * c, kvh, pa);
+            } else {
+              const int sa = tok >> 6;
+              const CUtensorMap* ma = which == 1 ? (sa == tail_slot ? &p.bv_tail : &p.bv_map)
+                                                 : (sa == tail_slot ? &p.bk_tail : &p.bk_map);
+              const CUtensorMap* mb = which == 1 ? (sa + 1 == tail_slot ? &p.bv_tail : &p.bv_map)
+                                                 : (sa + 1 == tail_slot ? &p.bk_tail : &p.bk_map);
+              for (int s = 0; s < 2; ++s) {
+                tma_load_5d(dst + s * 16384, ma, &full[slot], 0, 0, 2 * c + s, kvh, pa);
+                tma_load_5d(dst + s * 16384 + 8192, mb, &full[slot], 0, 0, 2 * c + s, kvh, pb);
+              }
             }
           } else {
             const int hh = kvh * p.g + i / n_tt;
-            const int tq = (tt_min + i % n_tt) * 64;
+            const int tq = (tt_min + i % n_tt) * 128;
             const CUtensorMap* m = which == 0 ? &p.b1r_map : which == 1 ? &p.b2r_map : &p.b3r_map;
-            tma_load_5d(dst, m, &full[slot], 0, tq, 0, hh, 0);
+            tma_load_5d(dst, m, &full[slot], 0, tq, 2 * c, hh, 0);
           }
         }
         ++issued;
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
-      // chunk order = consumption order: ST(0) ST(1) [M(i) ST(i+2)] ...
-      int pg0 = fetch(0), pg1 = fetch(1), pg2 = fetch(2);      // pages of tiles i, i+1, i+2
-      load(0, 0, pg0);
-      if (HAS_T) load(1, 0, pg0);
-      if (n_tiles > 1) {
-        load(0, 1, pg1);
-        if (HAS_T) load(1, 1, pg1);
-      }
+      auto load_st = [&](int i, int pa, int pb) {
+        for (int c = 0; c < C::NC; ++c) load(0, i, c, pa, pb);
+        if (HAS_T)
+          for (int c = 0; c < C::NC; ++c) load(1, i, c, pa, pb);
+      };
+      // chunk order = consumption order: ST(0) [M(i) ST(i+1)] ...
+      const int sh = small_pages ? 1 : (p.pg_shift - 7);            // page slot of tile i = (128 i) >> pg_shift
+      auto slot_of = [&](int i) { return small_pages ? 2 * i : (i >> sh); };
+      int pa0 = fetch(slot_of(0)), pb0 = small_pages ? fetch(1) : pa0;         // pages of tile i
+      int pa1 = fetch(slot_of(1)), pb1 = small_pages ? fetch(3) : pa1;         // pages of tile i + 1
+      load_st(0, pa0, pb0);
       for (int i = 0; i < n_tiles; ++i) {
-        const int pg3 = fetch(i + 3);                          // used two iterations from now
-        load(2, i, pg0);
-        if (i + 2 < n_tiles) {
-          load(0, i + 2, pg2);
-          if (HAS_T) load(1, i + 2, pg2);
-        }
-        pg0 = pg1; pg1 = pg2; pg2 = pg3;
+        const int pa2 = fetch(slot_of(i + 2)), pb2 = small_pages ? fetch(2 * i + 5) : pa2;   // used next round
+        for (int c = 0; c < C::NC; ++c) load(2, i, c, pa0, pb0);
+        if (i + 1 < n_tiles) load_st(i + 1, pa1, pb1);
+        pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
       }
+      LS_BTDUMP(0, tw0);
+      LS_BTDUMP(1, clock64() - t_kernel);
       if (*abort_flag) {   // aborted: wait (bounded) for the copies already started
         for (uint32_t s = 0; s < (uint32_t)C::RING && s < issued; ++s) {
           const uint32_t last = ((issued - 1 - s) / C::RING) * C::RING + s;
@@ -211,63 +243,88 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   } else if (warp == 1) {
     // =========================================================== MMA issuer (one thread)
     if (lane == 0 && n_tiles > 0) {
-      constexpr uint32_t idesc_st = make_idesc(128, 64, 0, 0);
-      constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);
+      constexpr uint32_t idesc_st = make_idesc(128, 128, 0, 0);
+      constexpr uint32_t idesc_acc = make_idesc(128, 128, 0, 1);
       constexpr uint32_t hi = sdesc_hi(1024);
       const uint32_t a1_lo = sdesc_lo(smem_u32(a1_smem), 16), a2_lo = sdesc_lo(smem_u32(a2_smem), 16);
-      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);      // K-major view of a chunk
-      const uint32_t ring_m_lo = sdesc_lo(smem_u32(ring), 8192);    // MN-major view: 8 KB group pitch
+      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major view of a chunk
+      const uint32_t ring_m_lo = sdesc_lo(smem_u32(ring), 16384);    // MN-major view: 16 KB group pitch
       uint32_t slot = 0, phase = 0;
       bool ok = mbar_wait(a_full, 0, abort_flag);
       auto advance = [&]() {
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
       auto issue_st = [&](int i) {
-        const uint32_t buf = tmem_buf0 + (i & 1) * 128;
 #pragma unroll
         for (int op = 0; op < (HAS_T ? 2 : 1); ++op) {
-          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
-          if (!ok) return;
-          tc_fence_after();
           const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
-          const uint32_t b_lo = ring_k_lo + slot * (C::CHUNK >> 4);
+          const uint32_t d = op == 0 ? tmem_s : tmem_t;
 #pragma unroll
-          for (int s = 0; s < C::SLABS; ++s)
+          for (int c = 0; c < C::NC; ++c) {
+            ok = ok && LS_BTWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
+            if (!ok) return;
+            tc_fence_after();
+            const uint32_t b_lo = ring_k_lo + slot * (kBwdChunk >> 4);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              mma_ss(buf + op * 64, sdesc(a_lo + ((s * 16384 + k * 32) >> 4), hi),
-                     sdesc(b_lo + ((s * 8192 + k * 32) >> 4), hi), idesc_st, (s | k) != 0);
-          mma_commit(&empty[slot]);
-          advance();
+            for (int s = 0; s < 2; ++s)
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                mma_ss(d, sdesc(a_lo + (((2 * c + s) * 16384 + k * 32) >> 4), hi),
+                       sdesc(b_lo + ((s * 16384 + k * 32) >> 4), hi), idesc_st, (c | s | k) != 0);
+            mma_commit(&empty[slot]);
+            advance();
+          }
+          mma_commit(op == 0 ? s_full : t_full);
         }
-        mma_commit(&st_full[i & 1]);
+        if (!HAS_T) mma_commit(t_full);
       };
       auto issue_acc = [&](int i) {
-        const uint32_t e_base = tmem_buf0 + (i & 1) * 128;
-        ok = ok && mbar_wait(&full[slot], phase, abort_flag);
-        if (!ok) return;
-        tc_fence_after();
-        const uint32_t b_lo = ring_m_lo + slot * (C::CHUNK >> 4);
+        // the NC chunks of B3 sit in consecutive ring slots starting at `slot`
+        uint32_t cs[C::NC], cph[C::NC];
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk)
-          mma_ts(tmem_acc, e_base + kk * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi), idesc_acc, (i | kk) != 0);
-        mma_commit(&empty[slot]);
-        advance();
+        for (int c = 0; c < C::NC; ++c) {
+          cs[c] = slot;
+          cph[c] = phase;
+          advance();
+        }
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          ok = ok && LS_BTWAIT(tw1, mbar_wait(&e_full[qd], i & 1, abort_flag));
+          if (!ok) return;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < C::NC; ++c) {
+            if (qd == 0) {
+              ok = ok && LS_BTWAIT(tw2, mbar_wait(&full[cs[c]], cph[c], abort_flag));
+              if (!ok) return;
+              tc_fence_after();
+            }
+            const uint32_t b_lo = ring_m_lo + cs[c] * (kBwdChunk >> 4);
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk)
+              mma_ts(tmem_acc + c * 128, tmem_s + (2 * qd + kk) * 8, sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi),
+                     idesc_acc, (i | qd | kk) != 0);
+            if (qd == 3) mma_commit(&empty[cs[c]]);
+          }
+        }
         if (i == n_tiles - 1) mma_commit(acc_final);
       };
       if (ok) issue_st(0);
-      if (ok && n_tiles > 1) issue_st(1);
       for (int i = 0; i < n_tiles && ok; ++i) {
-        ok = ok && mbar_wait(&e_full[i & 1], (i >> 1) & 1, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
         issue_acc(i);
-        if (ok && i + 2 < n_tiles) issue_st(i + 2);
+        if (ok && i + 1 < n_tiles) issue_st(i + 1);
       }
+      LS_BTDUMP(8, tw0);
+      LS_BTDUMP(9, tw1);
+      LS_BTDUMP(10, tw2);
+      LS_BTDUMP(11, clock64() - t_kernel);
     }
   } else {
     // =========================================================== elementwise + epilogue
+    // two threads per row: warps 2-5 take the lower 16 columns of every 32-column quarter,
+    // warps 6-9 the upper 16 (a warp may only touch the TMEM lanes of its quadrant, warp % 4)
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;
     const int r_idx = row0 + row;                 // query t (DQ) or key j (DK, DV)
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
@@ -276,7 +333,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     if (MODE == MODE_DQ) dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + h) * D;
     if (n_tiles == 0) {
       if (MODE == MODE_DQ && row_ok)
-        for (int c = 0; c < D; c += 4) *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 4)
+          *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
     } else {
       float lse2_row = 0.f, delta_row = 0.f;
       int64_t lim = 0;
@@ -288,86 +346,97 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
       }
       bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
-        const uint32_t tb = tmem_buf0 + (i & 1) * 128 + lane_sel;
-        // per-column constants (DK, DV): lane L holds columns L and L + 32
-        float cl0 = 0.f, cl1 = 0.f, cd0 = 0.f, cd1 = 0.f;
+        // per-column constants (DK, DV): lane L holds columns L + 32 q of the tile
+        float cl[4] = {0.f, 0.f, 0.f, 0.f}, cd[4] = {0.f, 0.f, 0.f, 0.f};
         int tq0 = 0;
         if (MODE != MODE_DQ) {
           const int hh = kvh * p.g + i / n_tt;
-          tq0 = (tt_min + i % n_tt) * 64;
-          const int ta = min(tq0 + lane, p.R - 1), tb2 = min(tq0 + lane + 32, p.R - 1);
-          cl0 = __ldg(p.lse + (size_t)ta * p.Hq + hh) * kLog2e;
-          cl1 = __ldg(p.lse + (size_t)tb2 * p.Hq + hh) * kLog2e;
-          if (MODE == MODE_DK) {
-            cd0 = __ldg(p.delta + (size_t)ta * p.Hq + hh);
-            cd1 = __ldg(p.delta + (size_t)tb2 * p.Hq + hh);
+          tq0 = (tt_min + i % n_tt) * 128;
+#pragma unroll
+          for (int qd = 0; qd < 4; ++qd) {
+            const int tc = min(tq0 + 32 * qd + lane, p.R - 1);
+            cl[qd] = __ldg(p.lse + (size_t)tc * p.Hq + hh) * kLog2e;
+            if (MODE == MODE_DK) cd[qd] = __ldg(p.delta + (size_t)tc * p.Hq + hh);
           }
         }
-        ok = mbar_wait(&st_full[i & 1], (i >> 1) & 1, abort_flag);
+        const int key0 = i * 128;
+        const bool edge = (MODE == MODE_DQ) ? __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim)
+                                            : ((tq0 < row0 + 127) || (tq0 + 127 >= p.R));
+        // ---- p = exp(s - LSE) for this thread's 4 x 16 columns, as soon as S is complete
+        // (the T MMAs are still running)
+        ok = LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        uint32_t sr[64], tr[64];
-        tmem_ld32(tb, sr);
-        tmem_ld32(tb + 32, sr + 32);
-        if (HAS_T) {
-          tmem_ld32(tb + 64, tr);
-          tmem_ld32(tb + 96, tr + 32);
-        }
-        tc_wait_ld32(sr);
-        tc_wait_ld32(sr + 32);
-        if (HAS_T) {
-          tc_wait_ld32(tr);
-          tc_wait_ld32(tr + 32);
-        }
-        uint32_t pk[32];
-        if (MODE == MODE_DQ) {
-          const int key0 = i * 64;
-          const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 63 > lim);
+        float pr[64];
 #pragma unroll
-          for (int j = 0; j < 64; j += 2) {
-            float p0 = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
-            float p1 = ex2(fmaf(__uint_as_float(sr[j + 1]), p.scale_log2, -lse2_row));
-            if (edge) {
-              if ((int64_t)key0 + j > lim) p0 = 0.f;
-              if ((int64_t)key0 + j + 1 > lim) p1 = 0.f;
-            }
-            pk[j >> 1] = pack_bf16(p0 * (__uint_as_float(tr[j]) - delta_row),
-                                   p1 * (__uint_as_float(tr[j + 1]) - delta_row));
-          }
-        } else {
-          // column t is visible to key row j when j <= t < R
-          const bool edge = (tq0 < row0 + 127) || (tq0 + 63 >= p.R);
+        for (int qd = 0; qd < 4; ++qd) {
+          uint32_t sr[16];
+          tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr);
+          tc_wait_ld16(sr);
 #pragma unroll
-          for (int j = 0; j < 64; j += 2) {
-            const float l0 = __shfl_sync(0xffffffffu, (j < 32) ? cl0 : cl1, j & 31);
-            const float l1 = __shfl_sync(0xffffffffu, (j + 1 < 32) ? cl0 : cl1, (j + 1) & 31);
-            float p0 = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -l0));
-            float p1 = ex2(fmaf(__uint_as_float(sr[j + 1]), p.scale_log2, -l1));
-            if (edge) {
-              const int ta = tq0 + j;
-              if (ta < r_idx || ta >= p.R) p0 = 0.f;
-              if (ta + 1 < r_idx || ta + 1 >= p.R) p1 = 0.f;
+          for (int j = 0; j < 16; ++j) {
+            const int col = 32 * qd + 16 * half + j;
+            float e;
+            if (MODE == MODE_DQ) {
+              e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
+              if (edge && (int64_t)key0 + col > lim) e = 0.f;
+            } else {
+              const float l0 = __shfl_sync(0xffffffffu, cl[qd], 16 * half + j);
+              e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -l0));
+              if (edge) {                      // column t is visible to key row j when j <= t < R
+                const int ta = tq0 + col;
+                if (ta < r_idx || ta >= p.R) e = 0.f;
+              }
             }
-            if (MODE == MODE_DK) {
-              const float d0 = __shfl_sync(0xffffffffu, (j < 32) ? cd0 : cd1, j & 31);
-              const float d1 = __shfl_sync(0xffffffffu, (j + 1 < 32) ? cd0 : cd1, (j + 1) & 31);
-              p0 *= __uint_as_float(tr[j]) - d0;
-              p1 *= __uint_as_float(tr[j + 1]) - d1;
-            }
-            pk[j >> 1] = pack_bf16(p0, p1);
+            pr[16 * qd + j] = e;
           }
         }
-        tmem_st32(tb, pk);
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(&e_full[i & 1]);
+        // E overwrites S columns that the row's other thread reads: all 256 threads must be done
+        // reading S before anyone writes (named barrier 1; the T MMAs normally still run here)
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // ---- E = p (T - Delta), quarter by quarter, once T is complete
+        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          uint32_t pk[8];
+          if (HAS_T) {
+            uint32_t tr[16];
+            tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr);
+            tc_wait_ld16(tr);
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+              float d0 = delta_row, d1 = delta_row;
+              if (MODE == MODE_DK) {
+                d0 = __shfl_sync(0xffffffffu, cd[qd], 16 * half + j);
+                d1 = __shfl_sync(0xffffffffu, cd[qd], 16 * half + j + 1);
+              }
+              pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[j]) - d0),
+                                     pr[16 * qd + j + 1] * (__uint_as_float(tr[j + 1]) - d1));
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) pk[j >> 1] = pack_bf16(pr[16 * qd + j], pr[16 * qd + j + 1]);
+          }
+          // quarter q of E (bf16 pairs) lands in columns [16 q, 16 q + 16) of the S region, whose
+          // fp32 contents every thread has already pulled into registers
+          tmem_st8(tmem_s + lane_sel + 16 * qd + 8 * half, pk);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(&e_full[qd]);
+        }
+      }
+      if (threadIdx.x == 64) {
+        LS_BTDUMP(16, tw0);
+        LS_BTDUMP(18, clock64() - t_kernel);
       }
       if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
       if (ok) {
         tc_fence_after();
         const float out_scale = (MODE == MODE_DK) ? p.scale : 1.0f;
 #pragma unroll 1
-        for (int c = 0; c < D; c += 32) {
+        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 32) {
           uint32_t o[32];
           tmem_ld32(tmem_acc + lane_sel + c, o);
           tc_wait_ld32(o);
@@ -505,7 +574,8 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   auto dense_map = [&](CUtensorMap* m, const void* base, int heads, int box_tok, int groups) {
     return ls::encode_map5(m, base, D, R, heads, 1, (int64_t)heads * D, D, (int64_t)R * heads * D, box_tok, groups);
   };
-  const int groups = D / 64;
+  const bool small_pages = d.page_size == 64;
+  const int pbox = small_pages ? 64 : 128, pgroups = small_pages ? 1 : 2;   // pool boxes
   ls::BwdParams P;
   P.shard_phys_pages = h->d_shard_phys_pages;
   P.shard_page_offset = h->d_shard_page_offset;
@@ -531,12 +601,12 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   // ---- dQ: rows = queries, columns = keys of every partial
   ls_status_t st = dense_map(&P.a1_map, q, Hq, 128, 1);
   if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128, 1);
-  if (st == LS_OK) st = dense_map(&P.b1r_map, k_resp, Hkv, 64, groups);
-  if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 64, groups);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_map, h, 0, 64, groups, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_tail, h, 0, 64, groups, true);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_map, h, 1, 64, groups, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_tail, h, 1, 64, groups, true);
+  if (st == LS_OK) st = dense_map(&P.b1r_map, k_resp, Hkv, 128, 2);
+  if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 128, 2);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_map, h, 0, pbox, pgroups, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_tail, h, 0, pbox, pgroups, true);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_map, h, 1, pbox, pgroups, false);
+  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_tail, h, 1, pbox, pgroups, true);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
   const int64_t grid_dq = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;
@@ -552,8 +622,8 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   const int grid_kv = Hkv * P.tiles_per_head;
   st = dense_map(&P.a1_map, k_resp, Hkv, 128, 1);
   if (st == LS_OK) st = dense_map(&P.a2_map, v_resp, Hkv, 128, 1);
-  if (st == LS_OK) st = dense_map(&P.b1r_map, q, Hq, 64, groups);
-  if (st == LS_OK) st = dense_map(&P.b2r_map, d_o, Hq, 64, groups);
+  if (st == LS_OK) st = dense_map(&P.b1r_map, q, Hq, 128, 2);
+  if (st == LS_OK) st = dense_map(&P.b2r_map, d_o, Hq, 128, 2);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
   P.out = static_cast<__nv_bfloat16*>(dk_resp);

@@ -20,6 +20,8 @@
 // TMEM columns: O [0, DVT), S/P buffer 0 [DVT, DVT+128), S/P buffer 1 [DVT+128, DVT+256).
 // K chunk  = 128 keys x 64*KSLABS channels (K-major, 128-byte swizzle): k-slices of S.
 // V chunk  = VKEYS keys x DVT channels as DVT/64 sub-slabs (MN-major): VKEYS/16 k-steps of PV.
+#include <cstdlib>
+
 #include "ls_internal.h"
 #include "ls_sm100.cuh"
 
@@ -39,6 +41,7 @@ struct FwdParams {
   int32_t* status;
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   int dv_total;   // channels of one output row (DVT times the number of O tiles)
+  int prefetch;   // L2 prefetch distance in 128-key tiles (0 = off)
   int ablate;   // diagnostic: LS_FLAG_ABLATE_* bits (results are then meaningless)
   float scale, scale_log2;
 };
@@ -215,6 +218,28 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           advance();
         }
       };
+      // L2 prefetch of the K and V boxes of a tile that will be loaded `prefetch` tiles later
+      auto prefetch_tile = [&](int tile, int pa, int pb) {
+        if (is_resp || tile >= n_tiles) return;
+        const int tok = tile * 128;
+        if (!small_pages) {
+          const bool tail = (tok >> p.pg_shift) == tail_slot;
+          for (int c = 0; c < C::KCH; ++c)
+            tma_prefetch_5d(tail ? &p.k_tail_map : &p.k_map, 0, tok & pg_mask, c * C::KSLABS, kvh, pa);
+          for (int r = 0; r < C::NVCH; ++r)
+            tma_prefetch_5d(tail ? &p.v_tail_map : &p.v_map, 0, (tok + r * C::VKEYS) & pg_mask, dvh * C::VSUB, kvh, pa);
+        } else {
+          for (int c = 0; c < C::KCH * C::KSLABS; ++c) {
+            tma_prefetch_5d((tok >> 6) == tail_slot ? &p.k_tail_map : &p.k_map, 0, 0, c, kvh, pa);
+            tma_prefetch_5d((tok >> 6) + 1 == tail_slot ? &p.k_tail_map : &p.k_map, 0, 0, c, kvh, pb);
+          }
+          for (int r = 0; r < C::NVCH; ++r) {
+            const int tk = tok + r * C::VKEYS;
+            tma_prefetch_5d((tk >> 6) == tail_slot ? &p.v_tail_map : &p.v_map, 0, tk & 63, dvh * C::VSUB, kvh,
+                            (r * C::VKEYS >= 64) ? pb : pa);
+          }
+        }
+      };
       const long long t_begin_p = clock64();
       // page ids of tile i: slots (128 i) >> pg_shift and, for 64-token pages, the next one
       int pa0 = 0, pb0 = 0, pa1 = 0, pb1 = 0;
@@ -227,12 +252,29 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         }
       }
       load_k(0, pa0, pb0);
+      const int pf = p.prefetch;
+      int pfa = 0, pfb = 0;                          // pages of tile i + pf (fetched one round early)
+      if (pf > 0 && !is_resp && pf < n_tiles) {
+        const int sp = (pf * 128) >> p.pg_shift;
+        pfa = fetch(sp);
+        pfb = small_pages ? fetch(sp + 1) : pfa;
+      }
       for (int i = 0; i < n_tiles; ++i) {
         int pa2 = 0, pb2 = 0;                       // prefetched two tiles ahead, used next iteration
         if (!is_resp && i + 2 < n_tiles) {
           const int s2 = ((i + 2) * 128) >> p.pg_shift;
           pa2 = fetch(s2);
           pb2 = small_pages ? fetch(s2 + 1) : pa2;
+        }
+        if (pf > 0) {
+          int na = 0, nb = 0;
+          if (!is_resp && i + 1 + pf < n_tiles) {
+            const int sp = ((i + 1 + pf) * 128) >> p.pg_shift;
+            na = fetch(sp);
+            nb = small_pages ? fetch(sp + 1) : na;
+          }
+          prefetch_tile(i + pf, pfa, pfb);
+          pfa = na; pfb = nb;
         }
         if (i + 1 < n_tiles) load_k(i + 1, pa1, pb1);
         load_v(i, pa0, pb0);
@@ -529,6 +571,10 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.nq_tiles = P.g * P.tiles_per_head;
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.dv_total = d.dim_v;
+  {
+    const char* e = getenv("LS_FWD_PREFETCH");
+    P.prefetch = e ? atoi(e) : 0;
+  }
   P.ablate = prm->flags & LS_FLAG_ABLATE_MASK;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * 1.4426950408889634f;
