@@ -25,6 +25,7 @@
 // room for one S and one T buffer only: ACC [0, D), S [D, D+128), T [D+128, D+256).
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "ls_internal.h"
@@ -40,6 +41,11 @@ struct BwdParams {
   // pages hold 64 tokens, 64 x 64 x 1 (four boxes per chunk)
   CUtensorMap bk_map, bk_tail, bv_map, bv_tail;   // prefix pool K and V (mode DQ)
   CUtensorMap b1r_map, b2r_map, b3r_map;          // dense sources: response K/V/K (DQ) or Q/dO/(Q|dO) (DK, DV)
+  // CTA-pair variant of the dQ pass: each CTA loads half of every streamed operand.
+  //   *_s: 64 columns x 128 channels (box 64 x 64 tokens x 2 groups) for S and T
+  //   *_m: 128 columns x 64 channels (box 64 x 128 x 1, or 64 x 64 x 1 on 64-token pages) for ACC
+  CUtensorMap pk_s, pk_s_tail, pv_s, pv_s_tail, pk_m, pk_m_tail;   // prefix pool
+  CUtensorMap rk_s, rv_s, rk_m;                                     // response K, V, K
   const int32_t* shard_phys_pages;
   const int32_t* shard_page_offset;
   const int32_t* shard_tail_slot;
@@ -55,7 +61,7 @@ struct BwdParams {
 
 #ifdef LS_TIMING
 #define LS_BTWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
-#define LS_BTDUMP(slot, val) do { if (MODE == MODE_DQ && blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
+#define LS_BTDUMP(slot, val) do { if (kTimedMode && blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
 #else
 #define LS_BTWAIT(acc, expr) (expr)
 #define LS_BTDUMP(slot, val) do { } while (0)
@@ -95,8 +101,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr bool kTimedMode = (MODE == MODE_DQ);
   long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
-  (void)tw0; (void)tw1; (void)tw2;
+  (void)tw0; (void)tw1; (void)tw2; (void)kTimedMode;
   const long long t_kernel = clock64();
   (void)t_kernel;
 
@@ -474,6 +481,360 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------
+// dQ pass on CTA pairs (cta_group::2).  Two neighbouring SMs take two Q tiles of the same
+// (KV head, partial) and stream the keys once between them: each CTA loads only half of
+// every K/V chunk (64 of the 128 keys for S and T, 64 of the 128 channels for ACC), so the
+// ring covers twice as many keys and the shared-memory write traffic halves.  One thread of
+// the even CTA issues all MMAs (256 rows); completions are multicast to both CTAs' barriers;
+// the odd CTA's row threads report their E quarters to the even CTA's barrier.
+// ---------------------------------------------------------------------------------
+constexpr int kDq2Chunk = 16384;
+
+template <int D>
+struct Dq2Cfg {
+  static constexpr int SLABS = D / 64;
+  static constexpr int NC = D / 128;
+  static constexpr int RING = (D == 128) ? 8 : 6;
+  static constexpr int A_BYTES = 2 * SLABS * 16384;
+  static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * kDq2Chunk + 512;
+};
+
+template <int D>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
+    bwd_dq2_kernel(const __grid_constant__ BwdParams p) {
+  using C = Dq2Cfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a1_smem = smem;
+  uint8_t* a2_smem = smem + C::SLABS * 16384;
+  uint8_t* ring = smem + C::A_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kDq2Chunk);
+  uint64_t* a_full = bars;               // (even CTA) both CTAs' resident operands landed
+  uint64_t* full = bars + 1;             // (even CTA) both halves of a chunk landed
+  uint64_t* empty = full + C::RING;      // (each CTA) chunk consumed
+  uint64_t* s_full = empty + C::RING;    // (each CTA) S in TMEM
+  uint64_t* t_full = s_full + 1;         // (each CTA) T in TMEM
+  uint64_t* e_full = t_full + 1;         // [4] (even CTA) quarter of E in both CTAs' TMEM: 16 warp arrivals
+  uint64_t* acc_final = e_full + 4;      // (each CTA)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  constexpr bool kTimedMode = true;
+  long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
+  (void)tw0; (void)tw1; (void)tw2; (void)kTimedMode;
+  const long long t_kernel0 = clock64();
+  (void)t_kernel0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+
+  // ---- work item of the pair, and this CTA's Q tile
+  const int npairs = (p.nq_tiles + 1) / 2;
+  int idx = blockIdx.x >> 1;
+  const int pairi = idx % npairs;
+  idx /= npairs;
+  const int part = idx % (p.S + 1);
+  const int kvh = idx / (p.S + 1);
+  const bool is_resp = (part == p.S);
+  auto tile_of = [&](int qt, int& hh, int& r0) {
+    if (qt < p.nq_tiles) {
+      hh = kvh * p.g + qt / p.tiles_per_head;
+      r0 = (qt % p.tiles_per_head) * 128;
+    } else {                                 // odd tile count: the pair's second CTA works on zero rows
+      hh = kvh * p.g + p.g - 1;
+      r0 = p.tiles_per_head * 128;
+    }
+  };
+  int h, row0, h_o, row0_o;
+  tile_of(2 * pairi + (int)rank, h, row0);
+  tile_of(2 * pairi + 1 - (int)rank, h_o, row0_o);
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, max(row0, row0_o) + 128);      // both CTAs walk the longer causal range
+  } else {
+    tokens = p.shard_tokens[part];
+    page_off = p.shard_page_offset[part];
+    n_pages = p.shard_page_offset[part + 1] - page_off;
+    tail_slot = p.shard_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 127) / 128);
+
+  if (threadIdx.x == 0) {
+    mbar_init(a_full, 1);
+    for (int i = 0; i < C::RING; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    mbar_init(s_full, 1);
+    mbar_init(t_full, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 16);
+    mbar_init(acc_final, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_holder, 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                      // both CTAs' barriers exist before any remote signal
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const uint32_t tmem_acc = tmem_base;
+  const uint32_t tmem_s = tmem_base + D;
+  const uint32_t tmem_t = tmem_base + D + 128;
+
+  if (warp == 0) {
+    // =========================================================== producer (one thread per CTA)
+    if (lane == 0 && n_tiles > 0) {
+      if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * 16384);
+      for (int c = 0; c < C::SLABS; ++c) {
+        tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
+        tma_load_5d_pair(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, h, 0);
+      }
+      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int pg_mask = (1 << p.pg_shift) - 1;
+      const bool small_pages = !is_resp && p.pg_shift == 6;
+      auto fetch = [&](int ps) -> int {
+        if (is_resp) return 0;
+        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
+      };
+      uint32_t slot = 0, phase = 0, issued = 0;
+      bool ok = true;
+      // `which` 0: this CTA's 64 keys of K for S; 1: of V for T; 2: this CTA's 64 channels of K for ACC
+      auto load = [&](int which, int i, int c, int pa, int pb) {
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
+        if (ok) {
+          if (leader) mbar_arrive_expect_tx(&full[slot], 2 * kDq2Chunk);
+          uint8_t* dst = ring + slot * kDq2Chunk;
+          const int tok = i * 128;
+          if (which < 2) {
+            const int tk = tok + (int)rank * 64;
+            if (is_resp) {
+              tma_load_5d_pair(dst, which ? &p.rv_s : &p.rk_s, &full[slot], 0, tk, 2 * c, kvh, 0);
+            } else {
+              const bool tail = (tk >> p.pg_shift) == tail_slot;
+              const CUtensorMap* m = which ? (tail ? &p.pv_s_tail : &p.pv_s) : (tail ? &p.pk_s_tail : &p.pk_s);
+              tma_load_5d_pair(dst, m, &full[slot], 0, tk & pg_mask, 2 * c, kvh, (small_pages && rank) ? pb : pa);
+            }
+          } else {
+            const int grp = 2 * c + (int)rank;
+            if (is_resp) {
+              tma_load_5d_pair(dst, &p.rk_m, &full[slot], 0, tok, grp, kvh, 0);
+            } else if (!small_pages) {
+              const bool tail = (tok >> p.pg_shift) == tail_slot;
+              tma_load_5d_pair(dst, tail ? &p.pk_m_tail : &p.pk_m, &full[slot], 0, tok & pg_mask, grp, kvh, pa);
+            } else {
+              const int sa = tok >> 6;
+              tma_load_5d_pair(dst, sa == tail_slot ? &p.pk_m_tail : &p.pk_m, &full[slot], 0, 0, grp, kvh, pa);
+              tma_load_5d_pair(dst + 8192, sa + 1 == tail_slot ? &p.pk_m_tail : &p.pk_m, &full[slot], 0, 0, grp, kvh, pb);
+            }
+          }
+        }
+        ++issued;
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      auto load_st = [&](int i, int pa, int pb) {
+        for (int c = 0; c < C::NC; ++c) load(0, i, c, pa, pb);
+        for (int c = 0; c < C::NC; ++c) load(1, i, c, pa, pb);
+      };
+      const int sh = p.pg_shift - 7;
+      auto slot_of = [&](int i) { return small_pages ? 2 * i : (i >> sh); };
+      int pa0 = fetch(slot_of(0)), pb0 = small_pages ? fetch(1) : pa0;
+      int pa1 = fetch(slot_of(1)), pb1 = small_pages ? fetch(3) : pa1;
+      load_st(0, pa0, pb0);
+      for (int i = 0; i < n_tiles; ++i) {
+        const int pa2 = fetch(slot_of(i + 2)), pb2 = small_pages ? fetch(2 * i + 5) : pa2;
+        for (int c = 0; c < C::NC; ++c) load(2, i, c, pa0, pb0);
+        if (i + 1 < n_tiles) load_st(i + 1, pa1, pb1);
+        pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
+      }
+      LS_BTDUMP(0, tw0);
+      LS_BTDUMP(1, clock64() - t_kernel0);
+      if (*abort_flag && leader) {   // aborted: wait (bounded) for the copies credited to this CTA's barriers
+        for (uint32_t s = 0; s < (uint32_t)C::RING && s < issued; ++s) {
+          const uint32_t last = ((issued - 1 - s) / C::RING) * C::RING + s;
+          const uint64_t t_start = globaltimer_ns();
+          while (!mbar_try_wait(&full[s], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer (one thread of the even CTA)
+    if (leader && lane == 0 && n_tiles > 0) {
+      constexpr uint32_t idesc_st = make_idesc(256, 128, 0, 0);
+      constexpr uint32_t idesc_acc = make_idesc(256, 128, 0, 1);
+      constexpr uint32_t hi = sdesc_hi(1024);
+      const uint32_t a1_lo = sdesc_lo(smem_u32(a1_smem), 16), a2_lo = sdesc_lo(smem_u32(a2_smem), 16);
+      const uint32_t ring_lo = sdesc_lo(smem_u32(ring), 16);
+      uint32_t slot = 0, phase = 0;
+      bool ok = mbar_wait(a_full, 0, abort_flag);
+      auto advance = [&]() {
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      auto issue_st = [&](int i) {
+#pragma unroll
+        for (int op = 0; op < 2; ++op) {
+          const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
+          const uint32_t d = op == 0 ? tmem_s : tmem_t;
+#pragma unroll
+          for (int c = 0; c < C::NC; ++c) {
+            ok = ok && LS_BTWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
+            if (!ok) return;
+            tc_fence_after();
+            const uint32_t b_lo = ring_lo + slot * (kDq2Chunk >> 4);
+#pragma unroll
+            for (int s = 0; s < 2; ++s)
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                mma_ss_pair(d, sdesc(a_lo + (((2 * c + s) * 16384 + k * 32) >> 4), hi),
+                            sdesc(b_lo + ((s * 8192 + k * 32) >> 4), hi), idesc_st, (c | s | k) != 0);
+            mma_commit_pair(&empty[slot]);
+            advance();
+          }
+          mma_commit_pair(op == 0 ? s_full : t_full);
+        }
+      };
+      auto issue_acc = [&](int i) {
+        uint32_t cs[C::NC], cph[C::NC];
+#pragma unroll
+        for (int c = 0; c < C::NC; ++c) {
+          cs[c] = slot;
+          cph[c] = phase;
+          advance();
+        }
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          ok = ok && LS_BTWAIT(tw1, mbar_wait(&e_full[qd], i & 1, abort_flag));
+          if (!ok) return;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < C::NC; ++c) {
+            if (qd == 0) {
+              ok = ok && LS_BTWAIT(tw2, mbar_wait(&full[cs[c]], cph[c], abort_flag));
+              if (!ok) return;
+              tc_fence_after();
+            }
+            const uint32_t b_lo = ring_lo + cs[c] * (kDq2Chunk >> 4);
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk)
+              mma_ts_pair(tmem_acc + c * 128, tmem_s + (2 * qd + kk) * 8,
+                          sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi), idesc_acc, (i | qd | kk) != 0);
+            if (qd == 3) mma_commit_pair(&empty[cs[c]]);
+          }
+        }
+        if (i == n_tiles - 1) mma_commit_pair(acc_final);
+      };
+      if (ok) issue_st(0);
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        issue_acc(i);
+        if (ok && i + 1 < n_tiles) issue_st(i + 1);
+      }
+      LS_BTDUMP(8, tw0);
+      LS_BTDUMP(9, tw1);
+      LS_BTDUMP(10, tw2);
+      LS_BTDUMP(11, clock64() - t_kernel0);
+    }
+  } else {
+    // =========================================================== elementwise + epilogue (both CTAs)
+    const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const int row = quad * 32 + lane;
+    const int r_idx = row0 + row;
+    const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+    const bool row_ok = r_idx < p.R;
+    float* dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + h) * D;
+    if (n_tiles == 0) {
+      if (row_ok)
+        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 4)
+          *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+      const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + h;
+      const float lse2_row = p.lse[ri] * kLog2e;
+      const float delta_row = p.delta[ri];
+      const int64_t lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
+      uint32_t e_remote[4];
+#pragma unroll
+      for (int qd = 0; qd < 4; ++qd) e_remote[qd] = mapa_u32(smem_u32(&e_full[qd]), 0);
+      bool ok = true;
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const int key0 = i * 128;
+        const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim);
+        ok = LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        float pr[64];
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          uint32_t sr[16];
+          tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr);
+          tc_wait_ld16(sr);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
+            if (edge && (int64_t)key0 + 32 * qd + 16 * half + j > lim) e = 0.f;
+            pr[16 * qd + j] = e;
+          }
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");   // all S reads of this CTA done before any E write
+        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          uint32_t tr[16], pk[8];
+          tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr);
+          tc_wait_ld16(tr);
+#pragma unroll
+          for (int j = 0; j < 16; j += 2)
+            pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[j]) - delta_row),
+                                   pr[16 * qd + j + 1] * (__uint_as_float(tr[j + 1]) - delta_row));
+          tmem_st8(tmem_s + lane_sel + 16 * qd + 8 * half, pk);
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(e_remote[qd]);   // one arrival per warp, at the even CTA
+        }
+      }
+      if (threadIdx.x == 64) {
+        LS_BTDUMP(16, tw0);
+        LS_BTDUMP(17, tw1);
+        LS_BTDUMP(18, clock64() - t_kernel0);
+      }
+      if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 32) {
+          uint32_t o[32];
+          tmem_ld32(tmem_acc + lane_sel + c, o);
+          tc_wait_ld32(o);
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(dq_dst + c + j) =
+                  make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
+                              __uint_as_float(o[j + 3]));
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();          // neither CTA leaves while the other may still touch its shared memory
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+}
+
 // Delta[t,h] = sum_d dO[t,h,d] * O[t,h,d], one warp per row.
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ o, int64_t rows,
                              int dv, float* __restrict__ delta) {
@@ -528,6 +889,23 @@ static ls_status_t launch_bwd(const BwdParams& prm, int grid, cudaStream_t st) {
   profile_begin(which, st);
   bwd_kernel<D, MODE><<<grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
   profile_end(which, st);
+  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
+template <int D>
+static ls_status_t launch_dq2(const BwdParams& prm, int64_t grid, cudaStream_t st) {
+  using C = Dq2Cfg<D>;
+  static bool configured = false;
+  if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
+  if (!configured) {
+    if (cudaFuncSetAttribute(bwd_dq2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
+        cudaSuccess)
+      return LS_ERR_CUDA;
+    configured = true;
+  }
+  profile_begin(LS_KERNEL_BWD_DQ, st);
+  bwd_dq2_kernel<D><<<(int)grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
+  profile_end(LS_KERNEL_BWD_DQ, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
@@ -611,8 +989,26 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   P.b3r_map = P.b1r_map;
   const int64_t grid_dq = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;
   if (grid_dq > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DQ>(P, (int)grid_dq, cs)
-                  : ls::launch_bwd<256, ls::MODE_DQ>(P, (int)grid_dq, cs);
+  const char* pair_env = getenv("LS_BWD_PAIR");
+  const bool use_pairs = !(pair_env && pair_env[0] == '0');
+  if (use_pairs) {
+    const int mbox = small_pages ? 64 : 128;
+    st = dense_map(&P.rk_s, k_resp, Hkv, 64, 2);
+    if (st == LS_OK) st = dense_map(&P.rv_s, v_resp, Hkv, 64, 2);
+    if (st == LS_OK) st = dense_map(&P.rk_m, k_resp, Hkv, 128, 1);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_s, h, 0, 64, 2, false);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_s_tail, h, 0, 64, 2, true);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_s, h, 1, 64, 2, false);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_s_tail, h, 1, 64, 2, true);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m, h, 0, mbox, 1, false);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m_tail, h, 0, mbox, 1, true);
+    if (st != LS_OK) return st;
+    const int64_t grid2 = (int64_t)Hkv * (d.num_shards + 1) * ((P.nq_tiles + 1) / 2) * 2;
+    st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq2<256>(P, grid2, cs);
+  } else {
+    st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DQ>(P, (int)grid_dq, cs)
+                    : ls::launch_bwd<256, ls::MODE_DQ>(P, (int)grid_dq, cs);
+  }
   if (st != LS_OK) return st;
   const int64_t n4 = rows * D / 4;
   ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 16), 256, 0, cs>>>(
