@@ -56,6 +56,7 @@ struct BwdParams {
   __nv_bfloat16* out;    // dk_resp or dv_resp [R, Hkv, D] (modes DK, DV)
   int32_t* status;
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  int packed;    // pair dQ pass only: one Q tile holds every (head, token) row of a KV group
   float scale, scale_log2;
 };
 
@@ -539,11 +540,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   const bool is_resp = (part == p.S);
   auto tile_of = [&](int qt, int& hh, int& r0) {
     if (qt < p.nq_tiles) {
-      hh = kvh * p.g + qt / p.tiles_per_head;
+      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
       r0 = (qt % p.tiles_per_head) * 128;
     } else {                                 // odd tile count: the pair's second CTA works on zero rows
-      hh = kvh * p.g + p.g - 1;
-      r0 = p.tiles_per_head * 128;
+      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
     }
   };
   int h, row0, h_o, row0_o;
@@ -590,7 +591,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
-      if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * 16384);
+      const int a_rows = p.packed ? p.g * p.R : 128;
+      if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * a_rows * 128);
       for (int c = 0; c < C::SLABS; ++c) {
         tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
         tma_load_5d_pair(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, h, 0);
@@ -744,16 +746,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;
-    const int r_idx = row0 + row;
+    // this thread's (token, head): 128 tokens of one head, or all rows of a KV group when packed
+    const int r_idx = p.packed ? row0 + row % p.R : row0 + row;
+    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const bool row_ok = r_idx < p.R;
-    float* dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + h) * D;
+    const bool row_ok = r_idx < p.R && (!p.packed || row < p.g * p.R);
+    float* dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + hr) * D;
     if (n_tiles == 0) {
       if (row_ok)
         for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 4)
           *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
     } else {
-      const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + h;
+      const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
       const float lse2_row = p.lse[ri] * kLog2e;
       const float delta_row = p.delta[ri];
       const int64_t lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
@@ -991,7 +995,16 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   if (grid_dq > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   const char* pair_env = getenv("LS_BWD_PAIR");
   const bool use_pairs = !(pair_env && pair_env[0] == '0');
+  P.packed = 0;
   if (use_pairs) {
+    const int g = Hq / Hkv;
+    if (g > 1 && g * R <= 128) {           // short response: all rows of a KV group in one Q tile
+      P.packed = 1;
+      P.nq_tiles = 1;
+      st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, R, g);
+      if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, R, g);
+      if (st != LS_OK) return st;
+    }
     const int mbox = small_pages ? 64 : 128;
     st = dense_map(&P.rk_s, k_resp, Hkv, 64, 2);
     if (st == LS_OK) st = dense_map(&P.rv_s, v_resp, Hkv, 64, 2);

@@ -42,6 +42,9 @@ struct FwdParams {
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   int dv_total;   // channels of one output row (DVT times the number of O tiles)
   int prefetch;   // L2 prefetch distance in 128-key tiles (0 = off)
+  int packed;     // 1: one Q tile holds every (head, token) row of a KV group (g * R <= 128 rows);
+                  //    row r is head r / R, token r % R.  Lets a short response stream K/V once.
+  int q_bytes;    // bytes the Q loads deliver
   int ablate;   // diagnostic: LS_FLAG_ABLATE_* bits (results are then meaningless)
   float scale, scale_log2;
 };
@@ -150,9 +153,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     // =========================================================== producer (one thread)
     if (lane == 0 && n_tiles > 0) {
       const bool no_loads = (p.ablate & LS_FLAG_ABLATE_LOADS) != 0;
-      mbar_arrive_expect_tx(q_full, C::Q_BYTES);
-      for (int c = 0; c < C::KCH; ++c)
-        tma_load_5d(q_smem + c * C::CHUNK, &p.q_map, q_full, 0, t0, c * C::KSLABS, h, 0);
+      mbar_arrive_expect_tx(q_full, p.q_bytes);
+      for (int c = 0; c < DK / 64; ++c) tma_load_5d(q_smem + c * 16384, &p.q_map, q_full, 0, t0, c, h, 0);
 
       const int32_t* pages = p.shard_phys_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
@@ -366,12 +368,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     // =========================================================== softmax + epilogue
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    const int t = t0 + row;
+    // this thread's (token, head): a tile is 128 tokens of one head, or all rows of a KV group
+    const int t = p.packed ? row % p.R : t0 + row;
+    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
+    const bool row_ok = p.packed ? row < p.g * p.R : t < p.R;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const size_t out_row = ((size_t)part * p.R + (size_t)min(t, p.R - 1)) * p.Hq + h;
+    const size_t out_row = ((size_t)part * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
     float* o_dst = p.o_part + out_row * p.dv_total + dvh * DVT;
     if (n_tiles == 0) {
-      if (t < p.R) {
+      if (row_ok) {
         for (int c = 0; c < DV; c += 4) *reinterpret_cast<float4*>(o_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
         if (dvh == 0) p.lse_part[out_row] = -INFINITY;
       }
@@ -468,7 +473,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           uint32_t o[32];
           tmem_ld32(tmem_o + lane_sel + c, o);
           tc_wait_ld32(o);
-          if (t < p.R) {
+          if (row_ok) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
               *reinterpret_cast<float4*>(o_dst + c + j) =
@@ -476,7 +481,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                               __uint_as_float(o[j + 2]) * inv_l, __uint_as_float(o[j + 3]) * inv_l);
           }
         }
-        if (t < p.R && dvh == 0) p.lse_part[out_row] = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
+        if (row_ok && dvh == 0) p.lse_part[out_row] = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
       }
     }
   }
@@ -540,8 +545,10 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   const int dvt = mla ? 256 : d.dim_v;                    // O channels per CTA
   const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
   const bool small_pages = d.page_size == 64;
-  ls_status_t st = ls::encode_map5(&P.q_map, q, d.dim_k, R, Hq, 1, (int64_t)Hq * d.dim_k, d.dim_k,
-                                   (int64_t)R * Hq * d.dim_k, 128, kslabs);
+  const int g = Hq / Hkv;
+  const bool packed = g * R <= 128 && g > 1;
+  ls_status_t st = packed ? ls::encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, R, g)
+                          : ls::encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, 128, 1);
   if (st == LS_OK)
     st = ls::encode_map5(&P.kr_map, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k,
                          (int64_t)R * Hkv * d.dim_k, 128, kslabs);
@@ -568,7 +575,9 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.S = d.num_shards;
   P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 127) / 128;
-  P.nq_tiles = P.g * P.tiles_per_head;
+  P.nq_tiles = packed ? 1 : P.g * P.tiles_per_head;
+  P.packed = packed ? 1 : 0;
+  P.q_bytes = (d.dim_k / 64) * (packed ? g * R : 128) * 128;
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.dv_total = d.dim_v;
   {

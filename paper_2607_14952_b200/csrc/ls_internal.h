@@ -74,6 +74,11 @@ ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64
                         int64_t dim_page, int64_t stride_tok, int64_t stride_head, int64_t stride_page,
                         int box_tok, int box_groups);
 
+// Map of a dense [R, heads, dim] bf16 tensor whose box spans box_tok tokens of box_heads
+// consecutive heads and one 64-channel group: fills a slab with rows (head, token).
+ls_status_t encode_map_rows(CUtensorMap* out, const void* base, int64_t dim_d, int64_t R, int64_t heads,
+                            int box_tok, int box_heads);
+
 // The pool's K (which = 0) or V (which = 1) map for the given box; tail = bounded to the valid
 // tokens of the partially filled last logical page.
 ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,

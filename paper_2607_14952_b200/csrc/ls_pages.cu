@@ -64,6 +64,22 @@ ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64
   return r == CUDA_SUCCESS ? LS_OK : LS_ERR_CUDA;
 }
 
+ls_status_t encode_map_rows(CUtensorMap* out, const void* base, int64_t dim_d, int64_t R, int64_t heads,
+                            int box_tok, int box_heads) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return LS_ERR_CUDA;
+  if (!aligned16(base) || dim_d % 64) return LS_ERR_ALIGNMENT;
+  cuuint64_t dims[5] = {64, (cuuint64_t)R, (cuuint64_t)(dim_d / 64), (cuuint64_t)heads, 1};
+  cuuint64_t strides[4] = {(cuuint64_t)(heads * dim_d * 2), 128, (cuuint64_t)(dim_d * 2),
+                           (cuuint64_t)(R * heads * dim_d * 2)};
+  cuuint32_t box[5] = {64, (cuuint32_t)box_tok, 1, (cuuint32_t)box_heads, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? LS_OK : LS_ERR_CUDA;
+}
+
 ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
                              bool tail) {
   const ls_pages_desc_t& d = h->desc;

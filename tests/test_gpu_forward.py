@@ -35,6 +35,11 @@ def test_config1_tiny_full():
     # shared-latent shape: 576-wide key page whose first 512 channels are the value
     small("mla_pg64", Dk=576, Dv=512, v_aliases_k=True, Hq=8, Hkv=1, P=64 * 20 + 5, page_size=64, num_shards=3, R=130),
     small("mla_pg256", Dk=576, Dv=512, v_aliases_k=True, Hq=4, Hkv=1, P=2048, page_size=256, num_shards=2, R=256),
+    # short responses: every (head, token) row of a KV group shares one Q tile
+    small("short_r5", P=3000, page_size=128, num_shards=5, R=5, Hq=6, Hkv=2),
+    small("short_r16", P=4096, page_size=256, num_shards=4, R=16, Hq=24, Hkv=4),
+    small("short_r1", P=1500, page_size=64, num_shards=3, R=1, Hq=8, Hkv=2, Dk=128, Dv=128),
+    small("short_r32_full_tile", P=2048, page_size=256, num_shards=2, R=32, Hq=8, Hkv=2),
 ], ids=lambda c: c.name)
 def test_forward_small_cases(cfg):
     case = parity.Case(cfg, extra_phys_pages=2)
