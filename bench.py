@@ -111,6 +111,8 @@ def run_cuda(args):
         # every SM streams its own slice of K/V -> bound by HBM, not by the tensor pipe
         cfg = W.scaled(cfg, name="%s-R%d" % (cfg.name, args.small_r), R=args.small_r,
                        num_shards=args.shards or 64, needles=0)
+    elif args.shards:
+        cfg = W.scaled(cfg, name="%s-S%d" % (cfg.name, args.shards), num_shards=args.shards)
     fwd_f, dq_f, kv_f = algorithmic_flops(cfg)
     step_flops = fwd_f + dq_f + kv_f
 

@@ -168,7 +168,8 @@ def ls_replay_attn_workspace_bytes(pages, R, Hq, scale, which):
     return int(lib().ls_replay_attn_workspace_bytes(pages.handle, C.byref(prm), which))
 
 
-def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=None, status=None, flags=0):
+def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=None, status=None, flags=0,
+                       workspace=None):
     """Returns (o_part [(S+1),R,Hq,Dv] fp32, lse_part [(S+1),R,Hq] fp32)."""
     R, Hq, _ = q.shape
     S, Dv = pages.desc.num_shards, pages.desc.dim_v
@@ -177,8 +178,13 @@ def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=No
     if lse_part is None:
         lse_part = torch.empty((S + 1, R, Hq), dtype=torch.float32, device=q.device)
     prm = _params(R, Hq, scale, flags)
+    if workspace is None:
+        nbytes = ls_replay_attn_workspace_bytes(pages, R, Hq, scale, LS_WORKSPACE_FWD)
+        if nbytes:
+            workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
     st = lib().ls_replay_attn_fwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_part),
-                                  _ptr(lse_part), None, 0, _ptr(status), _stream())
+                                  _ptr(lse_part), _ptr(workspace), 0 if workspace is None else workspace.numel(),
+                                  _ptr(status), _stream())
     _check(st, "ls_replay_attn_fwd")
     return o_part, lse_part
 

@@ -938,7 +938,8 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads, D = d.dim_k;
   const int64_t rows = (int64_t)R * Hq;
   float* dq_part = static_cast<float*>(workspace);
-  float* delta = dq_part + (size_t)(d.num_shards + 1) * rows * D;
+  const int parts = d.num_shards * h->fine;        // sub-shards; the kernels see `parts` prefix partials
+  float* delta = dq_part + (size_t)(parts + 1) * rows * D;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
   ls::delta_kernel<<<(int)((rows + 7) / 8), 256, 0, cs>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows,
@@ -949,7 +950,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     if (ms != LS_OK) return ms;
     const int64_t n4m = rows * D / 4;
     ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4m + 255) / 256, 148 * 16), 256, 0, cs>>>(
-        dq_part, d.num_shards + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));
+        dq_part, parts + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));
     return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
   }
 
@@ -972,7 +973,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   P.Hq = Hq;
   P.Hkv = Hkv;
   P.g = Hq / Hkv;
-  P.S = d.num_shards;
+  P.S = parts;
   P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 127) / 128;
   P.nq_tiles = P.g * P.tiles_per_head;
@@ -991,7 +992,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_tail, h, 1, pbox, pgroups, true);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
-  const int64_t grid_dq = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;
+  const int64_t grid_dq = (int64_t)Hkv * (parts + 1) * P.nq_tiles;
   if (grid_dq > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   const char* pair_env = getenv("LS_BWD_PAIR");
   const bool use_pairs = !(pair_env && pair_env[0] == '0');
@@ -1016,7 +1017,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m, h, 0, mbox, 1, false);
     if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m_tail, h, 0, mbox, 1, true);
     if (st != LS_OK) return st;
-    const int64_t grid2 = (int64_t)Hkv * (d.num_shards + 1) * ((P.nq_tiles + 1) / 2) * 2;
+    const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
     st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq2<256>(P, grid2, cs);
   } else {
     st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DQ>(P, (int)grid_dq, cs)
@@ -1025,7 +1026,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   if (st != LS_OK) return st;
   const int64_t n4 = rows * D / 4;
   ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 16), 256, 0, cs>>>(
-      dq_part, d.num_shards + 1, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
+      dq_part, parts + 1, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
 
   // ---- dK and dV of the response keys: rows = keys, columns = queries of the KV group
   const int grid_kv = Hkv * P.tiles_per_head;

@@ -443,7 +443,7 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   P.Hq = Hq;
   P.Hkv = Hkv;
   P.g = Hq / Hkv;
-  P.S = d.num_shards;
+  P.S = d.num_shards * h->fine;
   P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 63) / 64;
   P.nq_tiles = P.g * P.tiles_per_head;
@@ -460,7 +460,7 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   if (st == LS_OK) st = encode_pool_map5(&P.bv_tail, h, 1, 64, 1, true);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
-  st = launch_mla<MLA_DQ>(P, (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles * 3, cs);
+  st = launch_mla<MLA_DQ>(P, (int64_t)Hkv * (d.num_shards * h->fine + 1) * P.nq_tiles * 3, cs);
   if (st != LS_OK) return st;
 
   st = dense_map(&P.a1_map, k_resp, Hkv, kD1);

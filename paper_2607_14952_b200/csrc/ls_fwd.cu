@@ -36,8 +36,10 @@ struct FwdParams {
   const int32_t* shard_page_offset;
   const int32_t* shard_tail_slot;
   const int64_t* shard_tokens;
-  float* o_part;
+  float* o_part;       // prefix partials [S, R, Hq, dv] (S = sub-shards seen by the kernel)
   float* lse_part;
+  float* o_resp;       // the response block's partial [R, Hq, dv]
+  float* lse_resp;
   int32_t* status;
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   int dv_total;   // channels of one output row (DVT times the number of O tiles)
@@ -373,12 +375,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
     const bool row_ok = p.packed ? row < p.g * p.R : t < p.R;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const size_t out_row = ((size_t)part * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
-    float* o_dst = p.o_part + out_row * p.dv_total + dvh * DVT;
+    const size_t out_row = ((size_t)(is_resp ? 0 : part) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
+    float* o_dst = (is_resp ? p.o_resp : p.o_part) + out_row * p.dv_total + dvh * DVT;
+    float* lse_dst = (is_resp ? p.lse_resp : p.lse_part) + out_row;
     if (n_tiles == 0) {
       if (row_ok) {
         for (int c = 0; c < DV; c += 4) *reinterpret_cast<float4*>(o_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (dvh == 0) p.lse_part[out_row] = -INFINITY;
+        if (dvh == 0) *lse_dst = -INFINITY;
       }
     } else {
       // last visible key index of this row inside this partial
@@ -481,7 +484,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
                               __uint_as_float(o[j + 2]) * inv_l, __uint_as_float(o[j + 3]) * inv_l);
           }
         }
-        if (row_ok && dvh == 0) p.lse_part[out_row] = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
+        if (row_ok && dvh == 0) *lse_dst = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
       }
     }
   }
@@ -516,18 +519,18 @@ static ls_status_t launch_fwd(const FwdParams& prm, int64_t grid, cudaStream_t s
 
 extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_attn_params_t* prm, int which) {
   if (!h || !prm || prm->R < 1 || prm->num_q_heads < 1) return 0;
-  if (which == LS_WORKSPACE_FWD) return 0;
-  // backward: per-partial dQ (fp32) + Delta (fp32)
   const size_t rows = (size_t)prm->R * prm->num_q_heads;
-  return (size_t)(h->desc.num_shards + 1) * rows * h->desc.dim_k * sizeof(float) + rows * sizeof(float);
+  const size_t parts = (size_t)h->desc.num_shards * h->fine;      // sub-shard partials
+  // forward: sub-shard partials (O and LSE) when shards are sub-split, else nothing
+  if (which == LS_WORKSPACE_FWD) return h->fine > 1 ? parts * rows * (h->desc.dim_v + 1) * sizeof(float) : 0;
+  // backward: per-partial dQ (fp32) + Delta (fp32)
+  return (parts + 1) * rows * h->desc.dim_k * sizeof(float) + rows * sizeof(float);
 }
 
 extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_params_t* prm, const void* q,
                                           const void* k_resp, const void* v_resp, float* o_part, float* lse_part,
                                           void* workspace, size_t workspace_bytes, int32_t* status_dev,
                                           void* stream) {
-  (void)workspace;
-  (void)workspace_bytes;
   if (!h || !prm || !q || !k_resp || !v_resp || !o_part || !lse_part) return LS_ERR_INVALID_ARG;
   if (!h->on_device) return LS_ERR_INVALID_ARG;
   const ls_pages_desc_t& d = h->desc;
@@ -565,14 +568,27 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.shard_page_offset = h->d_shard_page_offset;
   P.shard_tail_slot = h->d_shard_tail_slot;
   P.shard_tokens = h->d_shard_tokens;
-  P.o_part = o_part;
-  P.lse_part = lse_part;
+  const int64_t rows_all = (int64_t)R * Hq;
+  const int fine = h->fine;
+  const int parts = d.num_shards * fine;
+  float* fine_o = nullptr;
+  float* fine_lse = nullptr;
+  if (fine > 1) {
+    const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_FWD);
+    if (!workspace || workspace_bytes < need || !ls::aligned16(workspace)) return LS_ERR_WORKSPACE;
+    fine_o = static_cast<float*>(workspace);
+    fine_lse = fine_o + (size_t)parts * rows_all * d.dim_v;
+  }
+  P.o_part = fine > 1 ? fine_o : o_part;
+  P.lse_part = fine > 1 ? fine_lse : lse_part;
+  P.o_resp = o_part + (size_t)d.num_shards * rows_all * d.dim_v;
+  P.lse_resp = lse_part + (size_t)d.num_shards * rows_all;
   P.status = status_dev;
   P.R = R;
   P.Hq = Hq;
   P.Hkv = Hkv;
   P.g = Hq / Hkv;
-  P.S = d.num_shards;
+  P.S = parts;
   P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 127) / 128;
   P.nq_tiles = packed ? 1 : P.g * P.tiles_per_head;
@@ -587,9 +603,10 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.ablate = prm->flags & LS_FLAG_ABLATE_MASK;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * 1.4426950408889634f;
-  const int64_t grid = (int64_t)Hkv * (d.num_shards + 1) * P.nq_tiles;
+  const int64_t grid = (int64_t)Hkv * (parts + 1) * P.nq_tiles;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (mla) return ls::launch_fwd<576, 256, 2>(P, grid, cs);
-  if (d.dim_k == 128) return ls::launch_fwd<128, 128, 1>(P, grid, cs);
-  return ls::launch_fwd<256, 256, 1>(P, grid, cs);
+  st = mla ? ls::launch_fwd<576, 256, 2>(P, grid, cs)
+           : d.dim_k == 128 ? ls::launch_fwd<128, 128, 1>(P, grid, cs) : ls::launch_fwd<256, 256, 1>(P, grid, cs);
+  if (st != LS_OK || fine == 1) return st;
+  return ls::group_merge(d.num_shards, fine, rows_all, d.dim_v, fine_o, fine_lse, o_part, lse_part, cs);
 }

@@ -37,12 +37,21 @@ struct ls_pages {
   // per shard: position (in its page list) of the global last logical page, or -1
   std::vector<int32_t> shard_tail_slot;       // [S]
 
+  // Kernel-side plan: every shard is cut into `fine` contiguous sub-shards so that one
+  // (KV head, sub-shard) stream of K and V fits comfortably in L2 while the CTAs that share it
+  // drift apart.  The device arrays below describe the S * fine sub-shards; the kernels treat
+  // them as S * fine partials and the host folds them back into the S the caller asked for.
+  int32_t fine;
+  std::vector<int32_t> fine_page_offset;      // [S * fine + 1]
+  std::vector<int64_t> fine_tokens;           // [S * fine]
+  std::vector<int32_t> fine_tail_slot;        // [S * fine]
+
   bool on_device;
   int device;
   int32_t* d_shard_phys_pages;   // [Np]
-  int32_t* d_shard_page_offset;  // [S+1]
-  int32_t* d_shard_tail_slot;    // [S]
-  int64_t* d_shard_tokens;       // [S]
+  int32_t* d_shard_page_offset;  // [S * fine + 1]  (sub-shards)
+  int32_t* d_shard_tail_slot;    // [S * fine]
+  int64_t* d_shard_tokens;       // [S * fine]
   int32_t* d_page_table;         // [Np]
   ls::PoolMaps k_maps, v_maps;
 };
@@ -89,6 +98,10 @@ ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int
 ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
                     void* dk_resp, void* dv_resp, int32_t* status_dev, cudaStream_t cs);
+
+// Folds `fine` consecutive sub-shard partials into each of `groups` shard partials.
+ls_status_t group_merge(int groups, int fine, int64_t rows, int dv, const float* in_o, const float* in_lse,
+                        float* out_o, float* out_lse, cudaStream_t st);
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -3,6 +3,7 @@
 // Eq. glm-tr-zigzag-pages), upload of the plan, TMA descriptors of the page pool, and
 // the integrity checksum used between replays.
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 #include <new>
 
@@ -205,6 +206,37 @@ extern "C" ls_status_t ls_prefix_pages_build(const ls_pages_desc_t* d, const int
     h->shard_tokens[s] = tokens;
   }
 
+  // sub-shards for the kernels: aim at <= 32 MB of K+V per (KV head, sub-shard)
+  {
+    int64_t max_tokens = 0;
+    for (int s = 0; s < S; ++s) max_tokens = std::max(max_tokens, h->shard_tokens[s]);
+    const int64_t bytes_per_tok = (int64_t)(d->dim_k + (d->v_aliases_k ? 0 : d->dim_v)) * 2;
+    int64_t fine = (max_tokens * bytes_per_tok + (32ll << 20) - 1) / (32ll << 20);
+    if (const char* e = getenv("LS_SUBSPLIT")) fine = atoi(e);
+    fine = std::max<int64_t>(1, std::min<int64_t>(fine, 16));
+    h->fine = (int32_t)fine;
+    h->fine_page_offset.assign(S * fine + 1, 0);
+    h->fine_tokens.assign(S * fine, 0);
+    h->fine_tail_slot.assign(S * fine, -1);
+    std::vector<int64_t> cut;
+    for (int s = 0; s < S; ++s) {
+      const int64_t lo = h->shard_page_offset[s], n = h->shard_page_offset[s + 1] - lo;
+      ls::even_chunks(n, fine, cut);
+      for (int64_t f = 0; f < fine; ++f) {
+        const int64_t i = s * fine + f;
+        h->fine_page_offset[i] = (int32_t)(lo + cut[f]);
+        h->fine_page_offset[i + 1] = (int32_t)(lo + cut[f + 1]);
+        int64_t tokens = (cut[f + 1] - cut[f]) * pg;
+        const int32_t tail = h->shard_tail_slot[s];
+        if (tail >= cut[f] && tail < cut[f + 1]) {
+          tokens -= pg - h->last_valid;
+          h->fine_tail_slot[i] = (int32_t)(tail - cut[f]);
+        }
+        h->fine_tokens[i] = tokens;
+      }
+    }
+  }
+
   if (d->k_pool == nullptr) {   // host-only plan
     *out = h;
     return LS_OK;
@@ -245,11 +277,10 @@ extern "C" ls_status_t ls_prefix_pages_build(const ls_pages_desc_t* d, const int
   }
 
   cudaError_t e = cudaGetDevice(&h->device);
-  std::vector<int32_t> off32(h->shard_page_offset.begin(), h->shard_page_offset.end());
   if (e == cudaSuccess) e = ls::upload(&h->d_shard_phys_pages, h->shard_phys_pages);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_page_offset, off32);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_tail_slot, h->shard_tail_slot);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_tokens, h->shard_tokens);
+  if (e == cudaSuccess) e = ls::upload(&h->d_shard_page_offset, h->fine_page_offset);
+  if (e == cudaSuccess) e = ls::upload(&h->d_shard_tail_slot, h->fine_tail_slot);
+  if (e == cudaSuccess) e = ls::upload(&h->d_shard_tokens, h->fine_tokens);
   if (e == cudaSuccess) e = ls::upload(&h->d_page_table, h->page_table);
   if (e != cudaSuccess) {
     ls::free_device(h);

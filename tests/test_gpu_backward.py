@@ -96,3 +96,18 @@ def test_backward_split_count_does_not_change_dq():
     torch.cuda.synchronize()
     for o in outs[1:]:
         assert (o[0].float() - outs[0][0].float()).abs().max() < 2e-3
+
+
+@pytest.mark.parametrize("fine", [2, 3, 5])
+def test_sub_split_shards_forward_and_backward(fine, monkeypatch):
+    # shards are cut into sub-shards for the kernels (a locality measure for long prefixes) and folded
+    # back into the S partials of the ABI; force it on small cases, including sub-shards left empty
+    monkeypatch.setenv("LS_SUBSPLIT", str(fine))
+    for cfg in (small("sub_pg64", P=64 * 13 + 7, page_size=64, num_shards=4, R=130),
+                small("sub_pg256", P=256 * 9 + 100, page_size=256, num_shards=2, R=200, Hq=6, Hkv=2),
+                small("sub_d128", Dk=128, Dv=128, P=128 * 11, page_size=128, num_shards=3, R=96, Hq=8, Hkv=2),
+                small("sub_mla", Dk=576, Dv=512, v_aliases_k=True, Hq=4, Hkv=1, P=64 * 9 + 3, page_size=64,
+                      num_shards=2, R=70)):
+        case = parity.Case(cfg)
+        fw = parity.check_forward(case, per_shard=True)
+        parity.check_backward(case, fw)
