@@ -28,6 +28,10 @@ from paper_2607_14952_b200 import workloads as W  # noqa: E402
 METRIC = "replay_attn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dQ kernel, from the one-pass ncu
+# capture summarised in profiles/dram_traffic_p2m.md (full-size workload, no scaling needed).
+DQ_KERNEL_DRAM_BYTES = {"p2m": 16482.4e6 + 6519.2e6}
+
 
 def algorithmic_flops(cfg):
     """Forward 2(Dk+Dv) per visible (query, key) pair; backward 2(2Dk+Dv) on a prefix key (the
@@ -130,13 +134,16 @@ def run_cuda(args):
     lse = torch.empty((cfg.R, cfg.Hq), dtype=torch.float32, device=dev)
     ws = torch.empty(B.ls_replay_attn_workspace_bytes(pages, cfg.R, cfg.Hq, cfg.scale, B.LS_WORKSPACE_BWD),
                      dtype=torch.uint8, device=dev)
+    fwd_ws_bytes = B.ls_replay_attn_workspace_bytes(pages, cfg.R, cfg.Hq, cfg.scale, B.LS_WORKSPACE_FWD)
+    fwd_ws = torch.empty(fwd_ws_bytes, dtype=torch.uint8, device=dev) if fwd_ws_bytes else None
     dq = torch.empty((cfg.R, cfg.Hq, cfg.Dk), dtype=torch.bfloat16, device=dev)
     dk = torch.empty((cfg.R, cfg.Hkv, cfg.Dk), dtype=torch.bfloat16, device=dev)
     dv = torch.empty((cfg.R, cfg.Hkv, cfg.Dv), dtype=torch.bfloat16, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
     def step(q, kr, vr, d_o):
-        B.ls_replay_attn_fwd(pages, q, kr, vr, cfg.scale, o_part=o_part, lse_part=lse_part, status=status)
+        B.ls_replay_attn_fwd(pages, q, kr, vr, cfg.scale, o_part=o_part, lse_part=lse_part, status=status,
+                             workspace=fwd_ws)
         B.ls_lse_merge(o_part, lse_part, o_bf16=o_bf16, o_f32=o_f32, lse=lse)
         B.ls_replay_attn_bwd(pages, q, kr, vr, o_f32, lse, d_o, cfg.scale, workspace=ws, dq=dq, dk_resp=dk,
                              dv_resp=dv, status=status)
@@ -228,11 +235,13 @@ def run_cuda(args):
         "clocks": clocks,
         "e2e": {"value": world * step_flops / (e2e_ms / args.steps * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": (7 + (1 if fwd_ws is not None else 0)) * args.steps,
         "roofline": {"bound": "tensor", "kernel": "bwd_kernel<D,DQ> (query-gradient pass)",
                      "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
                      "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
-                     "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ], "traffic": None,
+                     "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
+                     "traffic": DQ_KERNEL_DRAM_BYTES.get(cfg.name),
+                     "algorithmic_flops_per_launch": dq_f,
                      "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peak,
                                     "ms_per_launch": k_ms[B.LS_KERNEL_FWD]},
                      "whole_step_frac": value / world / peak,
