@@ -23,6 +23,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2607_14952_b200 import replicas  # noqa: E402
 from paper_2607_14952_b200 import workloads as W  # noqa: E402
 
 METRIC = "replay_attn_fwd_bwd_tflops"
@@ -126,7 +127,7 @@ def run_cuda(args):
                                     v_aliases_k=cfg.v_aliases_k)
     S = cfg.num_shards
     n_members = max(1, min(cfg.G, 4))
-    members = [W.make_member(cfg, (m + rank * n_members), dev) for m in range(n_members)]
+    members = [W.make_member(cfg, m, dev) for m in replicas.member_ids(rank, n_members)]
     o_part = torch.empty((S + 1, cfg.R, cfg.Hq, cfg.Dv), dtype=torch.float32, device=dev)
     lse_part = torch.empty((S + 1, cfg.R, cfg.Hq), dtype=torch.float32, device=dev)
     o_bf16 = torch.empty((cfg.R, cfg.Hq, cfg.Dv), dtype=torch.bfloat16, device=dev)
@@ -176,10 +177,7 @@ def run_cuda(args):
     clocks = sampler.stop() if rank == 0 else None
     ms = sum(a.elapsed_time(b) for a, b in ev)
     k_ms = {k: sum(a.elapsed_time(b) for a, b in kev[k]) / args.steps for k in kev}
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = replicas.max_over_ranks(ms, dev, world)
     if int(status.item()) != 0:
         raise RuntimeError("device status %d" % int(status.item()))
 
@@ -207,10 +205,7 @@ def run_cuda(args):
     e1.record()
     barrier()
     e2e_wall = time.perf_counter() - t0
-    te = torch.tensor([max(e0.elapsed_time(e1), e2e_wall * 1e3)], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(te, op=torch.distributed.ReduceOp.MAX)
-    e2e_ms = float(te.item())
+    e2e_ms = replicas.max_over_ranks(max(e0.elapsed_time(e1), e2e_wall * 1e3), dev, world)
 
     if rank != 0:
         if world > 1:
@@ -218,7 +213,7 @@ def run_cuda(args):
         return
     peaks = measured_peaks()
     ms_per_step = ms_total / args.steps
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = replicas.aggregate_throughput(step_flops, args.steps, world, ms_total) / 1e12
     dq_tflops = dq_f / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e12
     fwd_tflops = fwd_f / (k_ms[B.LS_KERNEL_FWD] * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
