@@ -288,9 +288,13 @@ def _oracle_rows(one, kp, vp, table, q, kr, vr, d_o, rows):
 def cpu_baseline(cfg, seconds_target=15.0, inputs=None):
     """The fp64 oracle as it stands, timed on this machine's host cores on a bounded row sample."""
     inp = inputs or _cpu_sample_inputs(cfg)
-    dt, fl = _oracle_rows(*inp, rows=4)
-    rows = int(max(4, min(256, seconds_target / max(dt / 4, 1e-6))))
+    rows = 4
     dt, fl = _oracle_rows(*inp, rows=rows)
+    for _ in range(3):                        # grow the sample until it costs about the target time
+        if dt >= 0.6 * seconds_target or rows >= 256:
+            break
+        rows = int(max(rows + 1, min(256, rows * seconds_target / max(dt, 1e-6))))
+        dt, fl = _oracle_rows(*inp, rows=rows)
     return {"value": fl / dt / 1e12, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
             "sample": "%d (row, head) pairs of one KV head of %s, forward + backward over all %d visible keys, "
                       "%.1f s" % (rows, cfg.name, cfg.P + cfg.R, dt)}
