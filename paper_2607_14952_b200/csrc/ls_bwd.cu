@@ -623,7 +623,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
               tma_load_5d_pair(dst, m, &full[slot], 0, tk & pg_mask, 2 * c, kvh, (small_pages && rank) ? pb : pa);
             }
           } else {
-            const int grp = 2 * c + (int)rank;
+            // D = 256: one 256-wide MMA covers both chunks, so this CTA owns channels [128 rank, +128)
+            // and chunk c is its c-th 64-channel group; D = 128: the single chunk's half `rank`
+            const int grp = (C::NC == 2) ? 2 * (int)rank + c : (int)rank;
             if (is_resp) {
               tma_load_5d_pair(dst, &p.rk_m, &full[slot], 0, tok, grp, kvh, 0);
             } else if (!small_pages) {
@@ -673,6 +675,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
       constexpr uint32_t hi = sdesc_hi(1024);
       const uint32_t a1_lo = sdesc_lo(smem_u32(a1_smem), 16), a2_lo = sdesc_lo(smem_u32(a2_smem), 16);
       const uint32_t ring_lo = sdesc_lo(smem_u32(ring), 16);
+      constexpr uint32_t idesc_acc2 = make_idesc(256, 256, 0, 1);
+      const uint32_t ring2_lo = sdesc_lo(smem_u32(ring), kDq2Chunk);   // MN-major, two 64-channel groups one slot apart
       uint32_t slot = 0, phase = 0;
       bool ok = mbar_wait(a_full, 0, abort_flag);
       auto advance = [&]() {
@@ -714,19 +718,35 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
           ok = ok && LS_BTWAIT(tw1, mbar_wait(&e_full[qd], i & 1, abort_flag));
           if (!ok) return;
           tc_fence_after();
+          if (qd == 0) {
 #pragma unroll
-          for (int c = 0; c < C::NC; ++c) {
-            if (qd == 0) {
+            for (int c = 0; c < C::NC; ++c) {
               ok = ok && LS_BTWAIT(tw2, mbar_wait(&full[cs[c]], cph[c], abort_flag));
               if (!ok) return;
-              tc_fence_after();
             }
-            const uint32_t b_lo = ring_lo + cs[c] * (kDq2Chunk >> 4);
+            tc_fence_after();
+          }
+          if (C::NC == 2) {
+            // D = 256: the two 64-channel groups sit in adjacent slots (6 chunks per tile in a ring
+            // of 6 keeps them at slots 4 and 5): one 256-wide MMA per 16 keys
+            const uint32_t b_lo = ring2_lo + cs[0] * (kDq2Chunk >> 4);
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk)
-              mma_ts_pair(tmem_acc + c * 128, tmem_s + (2 * qd + kk) * 8,
-                          sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi), idesc_acc, (i | qd | kk) != 0);
-            if (qd == 3) mma_commit_pair(&empty[cs[c]]);
+              mma_ts_pair(tmem_acc, tmem_s + (2 * qd + kk) * 8, sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi),
+                          idesc_acc2, (i | qd | kk) != 0);
+          } else {
+#pragma unroll
+            for (int c = 0; c < C::NC; ++c) {
+              const uint32_t b_lo = ring_lo + cs[c] * (kDq2Chunk >> 4);
+#pragma unroll
+              for (int kk = 0; kk < 2; ++kk)
+                mma_ts_pair(tmem_acc + c * 128, tmem_s + (2 * qd + kk) * 8,
+                            sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi), idesc_acc, (i | qd | kk) != 0);
+            }
+          }
+          if (qd == 3) {
+#pragma unroll
+            for (int c = 0; c < C::NC; ++c) mma_commit_pair(&empty[cs[c]]);
           }
         }
         if (i == n_tiles - 1) mma_commit_pair(acc_final);
