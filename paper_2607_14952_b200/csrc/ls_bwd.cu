@@ -46,6 +46,7 @@ struct BwdParams {
   //   *_m: 128 columns x 64 channels (box 64 x 128 x 1, or 64 x 64 x 1 on 64-token pages) for ACC
   CUtensorMap pk_s, pk_s_tail, pv_s, pv_s_tail, pk_m, pk_m_tail;   // prefix pool
   CUtensorMap rk_s, rv_s, rk_m;                                     // response K, V, K
+  CUtensorMap pv_m, pv_m_tail, rv_m;   // V as 128 columns x 64 channels (256-key tile variant)
   const int32_t* shard_phys_pages;
   const int32_t* shard_page_offset;
   const int32_t* shard_tail_slot;
@@ -916,6 +917,388 @@ static ls_status_t launch_bwd(const BwdParams& prm, int grid, cudaStream_t st) {
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------
+// dQ pass on CTA pairs with 256-key tiles (D = 256).  With N = 256 every MMA runs at the math
+// rate (the resident operand is re-read from shared memory half as often per key).  TMEM has
+// room for the accumulator and ONE 256-column score buffer, so a tile goes S -> p (kept in
+// registers, 128 per thread, two threads per row) -> T into the same buffer -> E = p (T - Delta)
+// in four 64-key quarters -> dQ += E K per quarter.
+// Chunks of 16 KB per CTA: K or V as (this CTA's 128 keys x 64 channels) for S / T, and K as
+// (64 keys x this CTA's 128 channels) for the accumulate.
+// ---------------------------------------------------------------------------------
+constexpr int kDq3Threads = 320;        // producer warp, MMA warp, 8 elementwise warps (2 threads per row)
+
+struct Dq3Cfg {
+  static constexpr int D = 256;
+  static constexpr int SLABS = 4;
+  static constexpr int RING = 6;
+  static constexpr int A_BYTES = 2 * SLABS * 16384;
+  static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * kDq2Chunk + 512;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
+    bwd_dq3_kernel(const __grid_constant__ BwdParams p) {
+  using C = Dq3Cfg;
+  constexpr int D = 256;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a1_smem = smem;
+  uint8_t* a2_smem = smem + C::SLABS * 16384;
+  uint8_t* ring = smem + C::A_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kDq2Chunk);
+  uint64_t* a_full = bars;               // (even CTA) both CTAs' resident operands landed
+  uint64_t* full = bars + 1;             // (even CTA) both halves of a chunk landed
+  uint64_t* empty = full + C::RING;      // (each CTA) chunk consumed
+  uint64_t* s_full = empty + C::RING;    // (each CTA) S in TMEM
+  uint64_t* s_read = s_full + 1;         // (even CTA) every row thread of both CTAs has pulled S: 16 warp arrivals
+  uint64_t* t_full = s_read + 1;         // (each CTA) T in TMEM
+  uint64_t* e_full = t_full + 1;         // [4] (even CTA) quarter of E in both CTAs' TMEM: 16 warp arrivals
+  uint64_t* acc_final = e_full + 4;      // (each CTA)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  constexpr bool kTimedMode = true;
+  long long tw0 = 0, tw1 = 0, tw2 = 0;
+  (void)tw0; (void)tw1; (void)tw2; (void)kTimedMode;
+  const long long t_kernel0 = clock64();
+  (void)t_kernel0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+
+  const int npairs = (p.nq_tiles + 1) / 2;
+  int idx = blockIdx.x >> 1;
+  const int pairi = idx % npairs;
+  idx /= npairs;
+  const int part = idx % (p.S + 1);
+  const int kvh = idx / (p.S + 1);
+  const bool is_resp = (part == p.S);
+  auto tile_of = [&](int qt, int& hh, int& r0) {
+    if (qt < p.nq_tiles) {
+      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      r0 = (qt % p.tiles_per_head) * 128;
+    } else {
+      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      r0 = p.tiles_per_head * 128;
+    }
+  };
+  int h, row0, h_o, row0_o;
+  tile_of(2 * pairi + (int)rank, h, row0);
+  tile_of(2 * pairi + 1 - (int)rank, h_o, row0_o);
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, max(row0, row0_o) + 128);
+  } else {
+    tokens = p.shard_tokens[part];
+    page_off = p.shard_page_offset[part];
+    n_pages = p.shard_page_offset[part + 1] - page_off;
+    tail_slot = p.shard_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 255) / 256);
+
+  if (threadIdx.x == 0) {
+    mbar_init(a_full, 1);
+    for (int i = 0; i < C::RING; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    mbar_init(s_full, 1);
+    mbar_init(s_read, 16);
+    mbar_init(t_full, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 16);
+    mbar_init(acc_final, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_holder, 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const uint32_t tmem_acc = tmem_base;
+  const uint32_t tmem_st = tmem_base + D;      // S, then T, then E (bf16) over its first 128 columns
+
+  if (warp == 0) {
+    // =========================================================== producer (one thread per CTA)
+    if (lane == 0 && n_tiles > 0) {
+      const int a_rows = p.packed ? p.g * p.R : 128;
+      if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * a_rows * 128);
+      for (int c = 0; c < C::SLABS; ++c) {
+        tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
+        tma_load_5d_pair(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, h, 0);
+      }
+      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int pg_mask = (1 << p.pg_shift) - 1;
+      const bool small_pages = !is_resp && p.pg_shift == 6;
+      auto page_at = [&](int tok) -> int {       // physical page holding key `tok` of this partial
+        if (is_resp) return 0;
+        const int ps = tok >> p.pg_shift;
+        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
+      };
+      uint32_t slot = 0, phase = 0, issued = 0;
+      bool ok = true;
+      auto acquire = [&]() -> uint8_t* {
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
+        if (ok && leader) mbar_arrive_expect_tx(&full[slot], 2 * kDq2Chunk);
+        return ring + slot * kDq2Chunk;
+      };
+      auto advance = [&]() {
+        ++issued;
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      // pq[j]: page of keys [256 i + 64 j, +64) of the tile being loaded
+      auto load_tile = [&](int i, const int* pq) {
+        const int tk = i * 256 + (int)rank * 128;          // this CTA's 128 keys for S and T
+        for (int which = 0; which < 2; ++which) {
+          for (int g = 0; g < 4; ++g) {
+            uint8_t* dst = acquire();
+            if (ok) {
+              if (is_resp) {
+                tma_load_5d_pair(dst, which ? &p.rv_m : &p.rk_m, &full[slot], 0, tk, g, kvh, 0);
+              } else if (!small_pages) {
+                const bool tail = (tk >> p.pg_shift) == tail_slot;
+                const CUtensorMap* m = which ? (tail ? &p.pv_m_tail : &p.pv_m) : (tail ? &p.pk_m_tail : &p.pk_m);
+                tma_load_5d_pair(dst, m, &full[slot], 0, tk & pg_mask, g, kvh, pq[2 * rank]);
+              } else {
+                const int sa = tk >> 6;
+                const CUtensorMap* ma = which ? (sa == tail_slot ? &p.pv_m_tail : &p.pv_m)
+                                              : (sa == tail_slot ? &p.pk_m_tail : &p.pk_m);
+                const CUtensorMap* mb = which ? (sa + 1 == tail_slot ? &p.pv_m_tail : &p.pv_m)
+                                              : (sa + 1 == tail_slot ? &p.pk_m_tail : &p.pk_m);
+                tma_load_5d_pair(dst, ma, &full[slot], 0, 0, g, kvh, pq[2 * rank]);
+                tma_load_5d_pair(dst + 8192, mb, &full[slot], 0, 0, g, kvh, pq[2 * rank + 1]);
+              }
+            }
+            advance();
+          }
+        }
+        for (int j = 0; j < 4; ++j) {                       // K for the accumulate: 64 keys x this CTA's 128 channels
+          uint8_t* dst = acquire();
+          if (ok) {
+            const int tq = i * 256 + j * 64;
+            if (is_resp) {
+              tma_load_5d_pair(dst, &p.rk_s, &full[slot], 0, tq, 2 * (int)rank, kvh, 0);
+            } else {
+              const bool tail = (tq >> p.pg_shift) == tail_slot;
+              tma_load_5d_pair(dst, tail ? &p.pk_s_tail : &p.pk_s, &full[slot], 0, tq & pg_mask, 2 * (int)rank, kvh,
+                               pq[j]);
+            }
+          }
+          advance();
+        }
+      };
+      int pq0[4], pq1[4];
+      for (int j = 0; j < 4; ++j) pq0[j] = page_at(j * 64);
+      for (int i = 0; i < n_tiles; ++i) {
+        for (int j = 0; j < 4; ++j) pq1[j] = (i + 1 < n_tiles) ? page_at((i + 1) * 256 + j * 64) : 0;   // next tile
+        load_tile(i, pq0);
+        for (int j = 0; j < 4; ++j) pq0[j] = pq1[j];
+      }
+      LS_BTDUMP(0, tw0);
+      LS_BTDUMP(1, clock64() - t_kernel0);
+      if (*abort_flag && leader) {
+        for (uint32_t s2 = 0; s2 < (uint32_t)C::RING && s2 < issued; ++s2) {
+          const uint32_t last = ((issued - 1 - s2) / C::RING) * C::RING + s2;
+          const uint64_t t_start = globaltimer_ns();
+          while (!mbar_try_wait(&full[s2], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer (one thread of the even CTA)
+    if (leader && lane == 0 && n_tiles > 0) {
+      constexpr uint32_t idesc_st = make_idesc(256, 256, 0, 0);
+      constexpr uint32_t idesc_acc = make_idesc(256, 256, 0, 1);
+      constexpr uint32_t hi = sdesc_hi(1024);
+      const uint32_t a1_lo = sdesc_lo(smem_u32(a1_smem), 16), a2_lo = sdesc_lo(smem_u32(a2_smem), 16);
+      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major 128 keys x 64 channels
+      const uint32_t ring_m_lo = sdesc_lo(smem_u32(ring), 8192);     // MN-major 64 keys x 2 groups of 64 channels
+      uint32_t slot = 0, phase = 0;
+      bool ok = mbar_wait(a_full, 0, abort_flag);
+      auto advance = [&]() {
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      for (int i = 0; i < n_tiles && ok; ++i) {
+#pragma unroll
+        for (int op = 0; op < 2; ++op) {
+          if (op == 1) {                     // T overwrites S: every row thread must have pulled its S first
+            ok = ok && LS_BTWAIT(tw1, mbar_wait(s_read, i & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+          }
+          const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            ok = ok && LS_BTWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t b_lo = ring_k_lo + slot * (kDq2Chunk >> 4);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              mma_ss_pair(tmem_st, sdesc(a_lo + ((g * 16384 + k * 32) >> 4), hi), sdesc(b_lo + ((k * 32) >> 4), hi),
+                          idesc_st, (g | k) != 0);
+            mma_commit_pair(&empty[slot]);
+            advance();
+          }
+          if (!ok) break;
+          mma_commit_pair(op == 0 ? s_full : t_full);
+        }
+        if (!ok) break;
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          ok = ok && LS_BTWAIT(tw2, mbar_wait(&e_full[qd], i & 1, abort_flag));
+          ok = ok && LS_BTWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t b_lo = ring_m_lo + slot * (kDq2Chunk >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            mma_ts_pair(tmem_acc, tmem_st + (4 * qd + kk) * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi), idesc_acc,
+                        (i | qd | kk) != 0);
+          mma_commit_pair(&empty[slot]);
+          advance();
+        }
+        if (ok && i == n_tiles - 1) mma_commit_pair(acc_final);
+      }
+      LS_BTDUMP(8, tw0);
+      LS_BTDUMP(9, tw1);
+      LS_BTDUMP(10, tw2);
+      LS_BTDUMP(11, clock64() - t_kernel0);
+    }
+  } else {
+    // =========================================================== elementwise + epilogue (both CTAs)
+    const int quad = warp & 3;
+    const int sub = (warp - 2) >> 2;                // which 32 of every 64-column quarter this thread owns (2 threads per row)
+    const int row = quad * 32 + lane;
+    const int r_idx = p.packed ? row0 + row % p.R : row0 + row;
+    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
+    const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+    const bool row_ok = r_idx < p.R && (!p.packed || row < p.g * p.R);
+    float* dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + hr) * D;
+    if (n_tiles == 0) {
+      if (row_ok)
+        for (int c = sub * (D / 2); c < (sub + 1) * (D / 2); c += 4)
+          *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+      const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
+      const float lse2_row = p.lse[ri] * kLog2e;
+      const float delta_row = p.delta[ri];
+      const int64_t lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
+      const uint32_t s_read_remote = mapa_u32(smem_u32(s_read), 0);
+      uint32_t e_remote[4];
+#pragma unroll
+      for (int qd = 0; qd < 4; ++qd) e_remote[qd] = mapa_u32(smem_u32(&e_full[qd]), 0);
+      bool ok = true;
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const int key0 = i * 256;
+        const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 255 > lim);
+        ok = LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        // p = exp(s - LSE) for this thread's 4 x 32 columns: all four TMEM loads in flight at once,
+        // p kept as packed bf16 pairs (64 registers) until T is ready
+        uint32_t sr[128];
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tmem_ld32(tmem_st + lane_sel + 64 * qd + 32 * sub, sr + 32 * qd);
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tc_wait_ld32(sr + 32 * qd);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(s_read_remote);    // this warp no longer needs S: T may overwrite it
+        uint32_t pp[64];
+#pragma unroll
+        for (int j = 0; j < 128; j += 2) {
+          float e0 = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
+          float e1 = ex2(fmaf(__uint_as_float(sr[j + 1]), p.scale_log2, -lse2_row));
+          if (edge) {
+            const int64_t col = (int64_t)key0 + 64 * (j >> 5) + 32 * sub + (j & 31);
+            if (col > lim) e0 = 0.f;
+            if (col + 1 > lim) e1 = 0.f;
+          }
+          pp[j >> 1] = pack_bf16(e0, e1);
+        }
+        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t tr[2][32];
+        tmem_ld32(tmem_st + lane_sel + 32 * sub, tr[0]);
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          tc_wait_ld32(tr[qd & 1]);
+          if (qd < 3) tmem_ld32(tmem_st + lane_sel + 64 * (qd + 1) + 32 * sub, tr[(qd + 1) & 1]);   // in flight meanwhile
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const uint32_t pw = pp[16 * qd + (j >> 1)];
+            pk[j >> 1] = pack_bf16(__uint_as_float(pw << 16) * (__uint_as_float(tr[qd & 1][j]) - delta_row),
+                                   __uint_as_float(pw & 0xffff0000u) * (__uint_as_float(tr[qd & 1][j + 1]) - delta_row));
+          }
+          // E (bf16 pairs) of quarter q goes to columns [32 q, 32 q + 32) of the buffer: T columns that
+          // this quarter or an earlier one has read -- by either thread of the row, hence the barrier
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          tmem_st16(tmem_st + lane_sel + 32 * qd + 16 * sub, pk);
+          tc_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(e_remote[qd]);
+        }
+      }
+      if (threadIdx.x == 64) {
+        LS_BTDUMP(16, tw0);
+        LS_BTDUMP(17, tw1);
+        LS_BTDUMP(18, clock64() - t_kernel0);
+      }
+      if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = sub * (D / 2); c < (sub + 1) * (D / 2); c += 32) {
+          uint32_t o[32];
+          tmem_ld32(tmem_acc + lane_sel + c, o);
+          tc_wait_ld32(o);
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(dq_dst + c + j) =
+                  make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
+                              __uint_as_float(o[j + 3]));
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+}
+
+static ls_status_t launch_dq3(const BwdParams& prm, int64_t grid, cudaStream_t st) {
+  static bool configured = false;
+  if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
+  if (!configured) {
+    if (cudaFuncSetAttribute(bwd_dq3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Dq3Cfg::SMEM_BYTES) !=
+        cudaSuccess)
+      return LS_ERR_CUDA;
+    configured = true;
+  }
+  profile_begin(LS_KERNEL_BWD_DQ, st);
+  bwd_dq3_kernel<<<(int)grid, kDq3Threads, Dq3Cfg::SMEM_BYTES, st>>>(prm);
+  profile_end(LS_KERNEL_BWD_DQ, st);
+  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
 template <int D>
 static ls_status_t launch_dq2(const BwdParams& prm, int64_t grid, cudaStream_t st) {
   using C = Dq2Cfg<D>;
@@ -1037,8 +1420,13 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m, h, 0, mbox, 1, false);
     if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m_tail, h, 0, mbox, 1, true);
     if (st != LS_OK) return st;
+    if (st == LS_OK) st = dense_map(&P.rv_m, v_resp, Hkv, 128, 1);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_m, h, 1, mbox, 1, false);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_m_tail, h, 1, mbox, 1, true);
+    if (st != LS_OK) return st;
     const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
-    st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq2<256>(P, grid2, cs);
+    const bool wide = D == 256 && !(pair_env && pair_env[0] == '2');     // LS_BWD_PAIR=2: 128-key pair kernel
+    st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : wide ? ls::launch_dq3(P, grid2, cs) : ls::launch_dq2<256>(P, grid2, cs);
   } else {
     st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DQ>(P, (int)grid_dq, cs)
                     : ls::launch_bwd<256, ls::MODE_DQ>(P, (int)grid_dq, cs);

@@ -32,6 +32,8 @@ struct FwdParams {
   CUtensorMap k_map, k_tail_map;   // pool K: box 64 x 128 x KSLABS (pages >= 128 tokens) or 64 x 64 x 1
   CUtensorMap v_map, v_tail_map;   // pool V: box 64 x 64 tokens x DV/64 groups
   CUtensorMap kr_map, vr_map;      // response K (64 x 128 x KSLABS) and V (64 x 64 x DV/64)
+  // CTA-pair variant (D = 256): every box is 64 channels x 64 tokens x 2 groups (16 KB)
+  CUtensorMap pk2, pk2_tail, pv2, pv2_tail, rk2, rv2;
   const int32_t* shard_phys_pages;
   const int32_t* shard_page_offset;
   const int32_t* shard_tail_slot;
@@ -498,6 +500,362 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
 }
 
+// ---------------------------------------------------------------------------------
+// Forward on CTA pairs (cta_group::2), head dim 256.  Two neighbouring SMs take two Q tiles of
+// the same (KV head, partial) and stream the keys once between them: for S each CTA loads 64
+// of the 128 keys of a tile, for P V each loads 128 of the 256 value channels, so shared-memory
+// writes and L2 reads halve and the ring covers two tiles.  One thread of the even CTA issues
+// all MMAs (256 rows); completions are multicast to both CTAs' barriers; the odd CTA's softmax
+// warps report P to the even CTA's barrier.  Chunks are 16 KB: 64 tokens x 128 channels.
+// ---------------------------------------------------------------------------------
+struct Fwd2Cfg {
+  static constexpr int D = 256;
+  static constexpr int CHUNK = 16384;
+  static constexpr int RING = 8;
+  static constexpr int Q_BYTES = 4 * 16384;
+  static constexpr int SMEM_BYTES = 1024 + Q_BYTES + RING * CHUNK + 512;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
+    fwd2_kernel(const __grid_constant__ FwdParams p) {
+  using C = Fwd2Cfg;
+  constexpr int DV = 256;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_smem = smem;
+  uint8_t* ring = smem + C::Q_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * C::CHUNK);
+  uint64_t* q_full = bars;              // (even CTA) both CTAs' Q tiles landed
+  uint64_t* full = bars + 1;            // (even CTA) both halves of a chunk landed
+  uint64_t* empty = full + C::RING;     // (each CTA)
+  uint64_t* s_full = empty + C::RING;   // [2] (each CTA)
+  uint64_t* p_full = s_full + 2;        // [2] (even CTA) P of both CTAs in TMEM: 8 warp arrivals
+  uint64_t* pv_done = p_full + 2;       // (each CTA) one phase per tile
+  uint64_t* o_final = pv_done + 1;      // (each CTA)
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(o_final + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+
+  // ---- work item of the pair, and this CTA's Q tile
+  const int npairs = (p.nq_tiles + 1) / 2;
+  int idx = blockIdx.x >> 1;
+  const int pairi = idx % npairs;
+  idx /= npairs;
+  const int part = idx % (p.S + 1);
+  const int kvh = idx / (p.S + 1);
+  const bool is_resp = (part == p.S);
+  auto tile_of = [&](int qt, int& hh, int& r0) {
+    if (qt < p.nq_tiles) {
+      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      r0 = (qt % p.tiles_per_head) * 128;
+    } else {                                 // odd tile count: the pair's second CTA works on zero rows
+      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
+    }
+  };
+  int h, t0, h_o, t0_o;
+  tile_of(2 * pairi + (int)rank, h, t0);
+  tile_of(2 * pairi + 1 - (int)rank, h_o, t0_o);
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, max(t0, t0_o) + 128);          // both CTAs walk the longer causal range
+  } else {
+    tokens = p.shard_tokens[part];
+    page_off = p.shard_page_offset[part];
+    n_pages = p.shard_page_offset[part + 1] - page_off;
+    tail_slot = p.shard_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 127) / 128);
+
+  if (threadIdx.x == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < C::RING; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    mbar_init(&s_full[0], 1);
+    mbar_init(&s_full[1], 1);
+    mbar_init(&p_full[0], 8);
+    mbar_init(&p_full[1], 8);
+    mbar_init(pv_done, 1);
+    mbar_init(o_final, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_holder, 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                      // both CTAs' barriers exist before any remote signal
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const uint32_t tmem_o = tmem_base;
+  const uint32_t tmem_s0 = tmem_base + DV;
+
+  if (warp == 0) {
+    // =========================================================== producer (one thread per CTA)
+    if (lane == 0 && n_tiles > 0) {
+      if (leader) mbar_arrive_expect_tx(q_full, 2 * p.q_bytes);
+      for (int c = 0; c < 4; ++c) tma_load_5d_pair(q_smem + c * 16384, &p.q_map, q_full, 0, t0, c, h, 0);
+      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int pg_mask = (1 << p.pg_shift) - 1;
+      auto page_at = [&](int tok) -> int {
+        if (is_resp) return 0;
+        const int ps = tok >> p.pg_shift;
+        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
+      };
+      uint32_t slot = 0, phase = 0, issued = 0;
+      bool ok = true;
+      // one chunk: 64 tokens starting at `tok` x channel groups [grp, grp + 2) of K (which = 0) or V
+      auto load = [&](int which, int tok, int grp, int page) {
+        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
+        if (ok) {
+          if (leader) mbar_arrive_expect_tx(&full[slot], 2 * C::CHUNK);
+          uint8_t* dst = ring + slot * C::CHUNK;
+          if (is_resp) {
+            tma_load_5d_pair(dst, which ? &p.rv2 : &p.rk2, &full[slot], 0, tok, grp, kvh, 0);
+          } else {
+            const bool tail = (tok >> p.pg_shift) == tail_slot;
+            const CUtensorMap* m = which ? (tail ? &p.pv2_tail : &p.pv2) : (tail ? &p.pk2_tail : &p.pk2);
+            tma_load_5d_pair(dst, m, &full[slot], 0, tok & pg_mask, grp, kvh, page);
+          }
+        }
+        ++issued;
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      // K of tile i for S: this CTA's 64 keys, two chunks of 128 channels.
+      // V of tile i for P V: both 64-key halves, this CTA's 128 channels.
+      auto load_k = [&](int i, int pa, int pb) {
+        const int tok = i * 128 + (int)rank * 64;
+        const int pg = rank ? pb : pa;
+        load(0, tok, 0, pg);
+        load(0, tok, 2, pg);
+      };
+      auto load_v = [&](int i, int pa, int pb) {
+        load(1, i * 128, 2 * (int)rank, pa);
+        load(1, i * 128 + 64, 2 * (int)rank, pb);
+      };
+      // pages of the two 64-key halves of tile i (equal unless the pages hold 64 tokens)
+      int pa0 = page_at(0), pb0 = page_at(64), pa1 = page_at(128), pb1 = page_at(192);
+      load_k(0, pa0, pb0);
+      for (int i = 0; i < n_tiles; ++i) {
+        const int pa2 = (i + 2 < n_tiles) ? page_at((i + 2) * 128) : 0;        // used next round
+        const int pb2 = (i + 2 < n_tiles) ? page_at((i + 2) * 128 + 64) : 0;
+        if (i + 1 < n_tiles) load_k(i + 1, pa1, pb1);
+        load_v(i, pa0, pb0);
+        pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
+      }
+      if (*abort_flag && leader) {   // aborted: wait (bounded) for the copies credited to this CTA's barriers
+        for (uint32_t s2 = 0; s2 < (uint32_t)C::RING && s2 < issued; ++s2) {
+          const uint32_t last = ((issued - 1 - s2) / C::RING) * C::RING + s2;
+          const uint64_t t_start = globaltimer_ns();
+          while (!mbar_try_wait(&full[s2], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer (one thread of the even CTA)
+    if (leader && lane == 0 && n_tiles > 0) {
+      constexpr uint32_t idesc_s = make_idesc(256, 128, 0, 0);
+      constexpr uint32_t idesc_pv = make_idesc(256, 256, 0, 1);
+      constexpr uint32_t hi = sdesc_hi(1024);
+      const uint32_t q_lo = sdesc_lo(smem_u32(q_smem), 16);
+      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major: 2 slabs of 64 keys x 64 channels
+      const uint32_t ring_v_lo = sdesc_lo(smem_u32(ring), 8192);     // MN-major: 2 groups of 64 channels x 64 keys
+      uint32_t slot = 0, phase = 0;
+      bool ok = mbar_wait(q_full, 0, abort_flag);
+      auto advance = [&]() {
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      auto issue_s = [&](int tile) {
+        const uint32_t d = tmem_s0 + (tile & 1) * 128;
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
+          const uint32_t b_lo = ring_k_lo + slot * (C::CHUNK >> 4);
+#pragma unroll
+          for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              mma_ss_pair(d, sdesc(q_lo + (((2 * c + s2) * 16384 + k * 32) >> 4), hi),
+                          sdesc(b_lo + ((s2 * 8192 + k * 32) >> 4), hi), idesc_s, (c | s2 | k) != 0);
+          mma_commit_pair(&empty[slot]);
+          advance();
+        }
+        mma_commit_pair(&s_full[tile & 1]);
+      };
+      auto issue_pv = [&](int tile) {
+        const uint32_t a_base = tmem_s0 + (tile & 1) * 128;   // P over the S columns
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
+          const uint32_t b_lo = ring_v_lo + slot * (C::CHUNK >> 4);
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            mma_ts_pair(tmem_o, a_base + (r * 4 + kk) * 8, sdesc(b_lo + ((kk * 2048) >> 4), hi), idesc_pv,
+                        (tile | r | kk) != 0);
+          mma_commit_pair(&empty[slot]);
+          advance();
+        }
+        mma_commit_pair(pv_done);
+        if (tile == n_tiles - 1) mma_commit_pair(o_final);
+      };
+      if (ok) issue_s(0);
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        if (i + 1 < n_tiles) issue_s(i + 1);
+        ok = ok && mbar_wait(&p_full[i & 1], (i >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        issue_pv(i);
+      }
+    }
+  } else {
+    // =========================================================== softmax + epilogue (both CTAs)
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const int t = p.packed ? t0 + row % p.R : t0 + row;
+    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
+    const bool row_ok = t < p.R && (!p.packed || row < p.g * p.R);
+    const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+    const size_t out_row = ((size_t)(is_resp ? 0 : part) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
+    float* o_dst = (is_resp ? p.o_resp : p.o_part) + out_row * p.dv_total;
+    float* lse_dst = (is_resp ? p.lse_resp : p.lse_part) + out_row;
+    if (n_tiles == 0) {
+      if (row_ok) {
+        for (int c = 0; c < DV; c += 4) *reinterpret_cast<float4*>(o_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+        *lse_dst = -INFINITY;
+      }
+    } else {
+      const int64_t lim = is_resp ? (int64_t)min(t, p.R - 1) : tokens - 1;
+      float m_ref = -INFINITY, l = 0.f;
+      const float thresh = kRescaleLog2 / p.scale_log2;
+      const uint32_t p_remote[2] = {mapa_u32(smem_u32(&p_full[0]), 0), mapa_u32(smem_u32(&p_full[1]), 0)};
+      bool ok = true;
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        const uint32_t ts = tmem_s0 + (i & 1) * 128 + lane_sel;
+        ok = mbar_wait(&s_full[i & 1], (i >> 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sr[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(ts + c * 32, sr + c * 32);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tc_wait_ld32(sr + c * 32);
+        float* s = reinterpret_cast<float*>(sr);
+        const int key0 = i * 128;
+        if (__any_sync(0xffffffffu, (int64_t)key0 + 127 > lim)) {
+#pragma unroll
+          for (int j = 0; j < 128; ++j)
+            if ((int64_t)key0 + j > lim) s[j] = -INFINITY;
+        }
+        float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
+#pragma unroll
+        for (int j = 4; j < 128; j += 4) {
+          mx0 = fmaxf(mx0, s[j]);
+          mx1 = fmaxf(mx1, s[j + 1]);
+          mx2 = fmaxf(mx2, s[j + 2]);
+          mx3 = fmaxf(mx3, s[j + 3]);
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        if (i == 0) {
+          m_ref = (mx == -INFINITY) ? 0.f : mx;
+        } else if (__any_sync(0xffffffffu, mx > m_ref + thresh)) {
+          // rare: raise the reference maximum and rescale the running sum and O (this CTA's rows)
+          ok = mbar_wait(pv_done, (i - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const float m_new = fmaxf(m_ref, mx);
+          const float f = ex2((m_ref - m_new) * p.scale_log2);
+          m_ref = m_new;
+          l *= f;
+#pragma unroll 1
+          for (int c = 0; c < DV; c += 32) {
+            uint32_t o[32];
+            tmem_ld32(tmem_o + lane_sel + c, o);
+            tc_wait_ld32(o);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * f);
+            tmem_st32(tmem_o + lane_sel + c, o);
+          }
+          tc_wait_st();
+        }
+        const float neg_m = -m_ref * p.scale_log2;
+        uint32_t pk[64];
+        float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 128; j += 2) {
+          const float p0 = ex2(fmaf(s[j], p.scale_log2, neg_m));
+          const float p1 = ex2(fmaf(s[j + 1], p.scale_log2, neg_m));
+          l0 += p0;
+          l1 += p1;
+          pk[j >> 1] = pack_bf16(p0, p1);
+        }
+        l += l0 + l1;
+        tmem_st32(ts, pk);
+        tmem_st32(ts + 32, pk + 32);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(p_remote[i & 1]);   // one arrival per warp, at the even CTA
+      }
+      if (ok) ok = mbar_wait(o_final, 0, abort_flag);
+      if (ok) {
+        tc_fence_after();
+        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
+#pragma unroll 1
+        for (int c = 0; c < DV; c += 32) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + lane_sel + c, o);
+          tc_wait_ld32(o);
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(o_dst + c + j) =
+                  make_float4(__uint_as_float(o[j]) * inv_l, __uint_as_float(o[j + 1]) * inv_l,
+                              __uint_as_float(o[j + 2]) * inv_l, __uint_as_float(o[j + 3]) * inv_l);
+          }
+        }
+        if (row_ok) *lse_dst = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();          // neither CTA leaves while the other may still touch its shared memory
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+}
+
+static ls_status_t launch_fwd2(const FwdParams& prm, int64_t grid, cudaStream_t st) {
+  static bool configured = false;
+  if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
+  if (!configured) {
+    if (cudaFuncSetAttribute(fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd2Cfg::SMEM_BYTES) !=
+        cudaSuccess)
+      return LS_ERR_CUDA;
+    configured = true;
+  }
+  profile_begin(LS_KERNEL_FWD, st);
+  fwd2_kernel<<<(int)grid, kFwdThreads, Fwd2Cfg::SMEM_BYTES, st>>>(prm);
+  profile_end(LS_KERNEL_FWD, st);
+  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
 template <int DK, int DVT, int NDV>
 static ls_status_t launch_fwd(const FwdParams& prm, int64_t grid, cudaStream_t st) {
   using C = FwdCfg<DK, DVT>;
@@ -605,8 +963,21 @@ extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_par
   P.scale_log2 = prm->scale * 1.4426950408889634f;
   const int64_t grid = (int64_t)Hkv * (parts + 1) * P.nq_tiles;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  st = mla ? ls::launch_fwd<576, 256, 2>(P, grid, cs)
-           : d.dim_k == 128 ? ls::launch_fwd<128, 128, 1>(P, grid, cs) : ls::launch_fwd<256, 256, 1>(P, grid, cs);
+  const char* pair_env = getenv("LS_FWD_PAIR");
+  if (d.dim_k == 256 && !(pair_env && pair_env[0] == '0')) {
+    st = ls::encode_map5(&P.rk2, k_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
+    if (st == LS_OK)
+      st = ls::encode_map5(&P.rv2, v_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk2, h, 0, 64, 2, false);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk2_tail, h, 0, 64, 2, true);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv2, h, 1, 64, 2, false);
+    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv2_tail, h, 1, 64, 2, true);
+    if (st != LS_OK) return st;
+    st = ls::launch_fwd2(P, (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2, cs);
+  } else {
+    st = mla ? ls::launch_fwd<576, 256, 2>(P, grid, cs)
+             : d.dim_k == 128 ? ls::launch_fwd<128, 128, 1>(P, grid, cs) : ls::launch_fwd<256, 256, 1>(P, grid, cs);
+  }
   if (st != LS_OK || fine == 1) return st;
   return ls::group_merge(d.num_shards, fine, rows_all, d.dim_v, fine_o, fine_lse, o_part, lse_part, cs);
 }
