@@ -232,6 +232,15 @@ typedef enum {
 } ls_kernel_t;
 ls_status_t ls_profile_arm_events(int kernel, void* start_event, void* stop_event);
 
+/*
+ * Self-test of the bounded device-side wait (the paper has no counterpart).  Launches one
+ * small CTA whose thread waits, with the library's own wait routine and a budget of
+ * `budget_ns` nanoseconds, on a barrier that nothing ever completes.  The wait must give up,
+ * the kernel must exit normally and LS_ERR_TIMEOUT must appear in *status_dev (device int32,
+ * zeroed by the caller).  Nothing traps, faults or spins without bound.
+ */
+ls_status_t ls_selftest_bounded_wait(int32_t* status_dev, uint64_t budget_ns, void* stream);
+
 const char* ls_status_string(ls_status_t status);
 
 #ifdef __cplusplus

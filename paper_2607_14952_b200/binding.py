@@ -68,6 +68,8 @@ def lib():
         L.ls_replay_attn_bwd_static.restype = C.c_int
         L.ls_replay_attn_bwd_static_capacity.argtypes = []
         L.ls_replay_attn_bwd_static_capacity.restype = C.c_size_t
+        L.ls_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp]
+        L.ls_selftest_bounded_wait.restype = C.c_int
         L.ls_profile_arm_events.argtypes = [C.c_int, vp, vp]
         L.ls_profile_arm_events.restype = C.c_int
         L.ls_status_string.argtypes = [C.c_int]
@@ -252,3 +254,8 @@ def ls_profile_arm_events(kernel, start_event, stop_event):
     a = None if start_event is None else C.c_void_p(start_event.cuda_event)
     b = None if stop_event is None else C.c_void_p(stop_event.cuda_event)
     _check(lib().ls_profile_arm_events(kernel, a, b), "ls_profile_arm_events")
+
+
+def ls_selftest_bounded_wait(status, budget_ns):
+    """Runs the bounded-wait self test; `status` is a zeroed int32 CUDA tensor."""
+    _check(lib().ls_selftest_bounded_wait(_ptr(status), int(budget_ns), _stream()), "ls_selftest_bounded_wait")

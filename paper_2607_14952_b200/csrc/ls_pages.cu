@@ -8,6 +8,7 @@
 #include <new>
 
 #include "ls_internal.h"
+#include "ls_sm100.cuh"
 
 namespace ls {
 
@@ -380,6 +381,32 @@ extern "C" ls_status_t ls_profile_arm_events(int kernel, void* start_event, void
   ls::g_profile[kernel].start = static_cast<cudaEvent_t>(start_event);
   ls::g_profile[kernel].stop = static_cast<cudaEvent_t>(stop_event);
   return LS_OK;
+}
+
+namespace ls {
+// One thread waits on a barrier that nobody arrives at; the bounded wait gives up after
+// budget_ns and the CTA reports LS_ERR_TIMEOUT exactly as the attention kernels would.
+__global__ void selftest_wait_kernel(int32_t* status, uint64_t budget_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const bool done = mbar_wait_budget(&bar, 0, &abort_flag, budget_ns, 1000);
+    if (!done && abort_flag && status) atomicExch(status, (int)LS_ERR_TIMEOUT);
+  }
+  __syncthreads();
+}
+}  // namespace ls
+
+extern "C" ls_status_t ls_selftest_bounded_wait(int32_t* status_dev, uint64_t budget_ns, void* stream) {
+  if (!status_dev || budget_ns == 0 || budget_ns > 1000000000ull) return LS_ERR_INVALID_ARG;
+  ls::selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status_dev, budget_ns);
+  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
 extern "C" const char* ls_status_string(ls_status_t s) {

@@ -69,17 +69,21 @@ constexpr uint64_t kWaitBudgetNs = 2000000000ull;   // 2 s
 constexpr uint32_t kWaitHintNs = 200000u;           // one parked poll lasts at most 0.2 ms
 
 // Returns true when the phase with the given parity completed; false on abort/time-out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
+__device__ __forceinline__ bool mbar_wait_budget(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                 uint64_t budget_ns, uint32_t hint_ns) {
+  if (mbar_try_wait(bar, parity, hint_ns)) return true;
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
-    if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
+    if (mbar_try_wait(bar, parity, hint_ns)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > kWaitBudgetNs) {
+    if (globaltimer_ns() - t0 > budget_ns) {
       *abort_flag = 1;
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetNs, kWaitHintNs);
 }
 
 // ------------------------------------------------------------------ TMA

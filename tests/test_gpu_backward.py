@@ -111,3 +111,17 @@ def test_sub_split_shards_forward_and_backward(fine, monkeypatch):
         case = parity.Case(cfg)
         fw = parity.check_forward(case, per_shard=True)
         parity.check_backward(case, fw)
+
+
+@pytest.mark.parametrize("fwd_pair,bwd_pair", [("0", "0"), ("0", "2"), ("1", "2")])
+def test_alternative_kernels_stay_correct(fwd_pair, bwd_pair, monkeypatch):
+    # head dim 256 defaults to the CTA-pair forward and the 256-key-tile pair dQ kernel; the
+    # single-CTA forward / dQ kernels and the 128-key-tile pair kernel remain selectable
+    monkeypatch.setenv("LS_FWD_PAIR", fwd_pair)
+    monkeypatch.setenv("LS_BWD_PAIR", bwd_pair)
+    for cfg in (small("alt_basic", P=2048 + 300, page_size=256, num_shards=3, R=200, Hq=6, Hkv=2),
+                small("alt_pg64", P=64 * 13 + 7, page_size=64, num_shards=4, R=130),
+                small("alt_short", P=3000, page_size=128, num_shards=5, R=5, Hq=6, Hkv=2)):
+        case = parity.Case(cfg)
+        fw = parity.check_forward(case, per_shard=True)
+        parity.check_backward(case, fw)

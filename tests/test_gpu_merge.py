@@ -40,3 +40,17 @@ def test_merge_all_empty_and_dominant_partial():
     assert torch.isinf(lse[:4]).all() and (lse[:4] < 0).all() and (o_f32[:4] == 0).all()
     assert torch.allclose(lse[4:], torch.full_like(lse[4:], 64.0)) and torch.allclose(o_f32[4:], torch.full_like(o_f32[4:], 3.0))
     assert torch.isfinite(o_f32).all()
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    # a barrier that nothing completes: the wait must run out (2 ms budget), the kernel must return,
+    # the status word must say LS_ERR_TIMEOUT and the context must stay usable
+    import time
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = time.perf_counter()
+    B.ls_selftest_bounded_wait(status, 2_000_000)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0
+    assert int(status.item()) == B.LS_ERR_TIMEOUT
+    x = torch.ones(4, device="cuda") * 2                      # the context still works
+    assert float(x.sum()) == 8.0
