@@ -31,7 +31,7 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dQ kernel, from the one-pass ncu
 # capture summarised in profiles/dram_traffic_p2m.md (full-size workload, no scaling needed).
-DQ_KERNEL_DRAM_BYTES = {"p2m": 16482.4e6 + 6519.2e6}
+DQ_KERNEL_DRAM_BYTES = {"p2m": 16650.2e6 + 6615.7e6}
 
 
 def algorithmic_flops(cfg):
@@ -231,7 +231,7 @@ def run_cuda(args):
         "e2e": {"value": world * step_flops / (e2e_ms / args.steps * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": (7 + (1 if fwd_ws is not None else 0)) * args.steps,
-        "roofline": {"bound": "tensor", "kernel": "bwd_kernel<D,DQ> (query-gradient pass)",
+        "roofline": {"bound": "tensor", "kernel": "bwd_dq3_kernel (query-gradient pass, CTA pairs)",
                      "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
                      "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
                      "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
