@@ -153,6 +153,11 @@ size_t ls_replay_attn_workspace_bytes(const ls_pages_t* pages, const ls_attn_par
  * An empty partial has lse = -inf and o = 0.
  *  q [R,Hq,dim_k] bf16; k_resp [R,Hkv,dim_k], v_resp [R,Hkv,dim_v] bf16
  *  o_part [(S+1),R,Hq,dim_v] fp32; lse_part [(S+1),R,Hq] fp32
+ *  workspace: ls_replay_attn_workspace_bytes(.., LS_WORKSPACE_FWD) bytes of device memory,
+ *  16-byte aligned; 0 (workspace may be NULL) unless the plan splits a shard into
+ *  cache-sized sub-shards, whose partials are held there and merged per shard with the same
+ *  Eq. qwen-lse-parts arithmetic before the call returns its (S+1) partials.  A workspace
+ *  that is too small gives LS_ERR_WORKSPACE before any launch.
  */
 ls_status_t ls_replay_attn_fwd(const ls_pages_t* pages, const ls_attn_params_t* prm,
                                const void* q, const void* k_resp, const void* v_resp,
