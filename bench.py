@@ -31,6 +31,9 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dQ kernel, from the one-pass ncu
 # capture summarised in profiles/dram_traffic_p2m.md (full-size workload, no scaling needed).
+DQ_KERNEL_NAME = {(256, 256): "bwd_dq3_kernel (query-gradient pass, CTA pairs)",
+                  (128, 128): "bwd_dq2_kernel<128> (query-gradient pass, CTA pairs)",
+                  (576, 512): "bwd_mla_dq_kernel (query-gradient pass, 576/512 shape)"}
 DQ_KERNEL_DRAM_BYTES = {"p2m": 16650.2e6 + 6615.7e6}
 
 
@@ -231,7 +234,7 @@ def run_cuda(args):
         "e2e": {"value": world * step_flops / (e2e_ms / args.steps * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": (7 + (1 if fwd_ws is not None else 0)) * args.steps,
-        "roofline": {"bound": "tensor", "kernel": "bwd_dq3_kernel (query-gradient pass, CTA pairs)",
+        "roofline": {"bound": "tensor", "kernel": DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv), "query-gradient pass"),
                      "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
                      "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
                      "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
