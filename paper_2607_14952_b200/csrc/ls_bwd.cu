@@ -1342,15 +1342,18 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   const int64_t rows = (int64_t)R * Hq;
   float* dq_part = static_cast<float*>(workspace);
   const int parts = d.num_shards * h->fine;        // sub-shards; the kernels see `parts` prefix partials
-  float* delta = dq_part + (size_t)(parts + 1) * rows * D;
+  const bool mla_fast = mla && ls::mla_dq_fast(h);
+  float* delta = dq_part + (size_t)(mla_fast ? 1 : parts + 1) * rows * D;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
   ls::delta_kernel<<<(int)((rows + 7) / 8), 256, 0, cs>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows,
                                                         d.dim_v, delta);
 
   if (mla) {
-    ls_status_t ms = ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_part, dk_resp, dv_resp, status_dev, cs);
+    ls_status_t ms =
+        ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_part, dk_resp, dv_resp, mla_fast, status_dev, cs);
     if (ms != LS_OK) return ms;
+    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_part, dq, status_dev, cs);
     const int64_t n4m = rows * D / 4;
     ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4m + 255) / 256, 148 * 16), 256, 0, cs>>>(
         dq_part, parts + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));

@@ -41,6 +41,7 @@ struct MlaBwdParams {
   __nv_bfloat16* out;      // dk_resp [R, Hkv, 576] or dv_resp [R, Hkv, 512]
   int32_t* status;
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles;   // tiles of 64 rows
+  int part_first, part_count;   // mode DQ: partials [part_first, part_first + part_count) are computed
   float scale, scale_log2;
 };
 
@@ -86,8 +87,8 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
   if (MODE == MLA_DQ) {
     const int qtile = idx % p.nq_tiles;
     idx /= p.nq_tiles;
-    part = idx % (p.S + 1);
-    kvh = idx / (p.S + 1);
+    part = p.part_first + idx % p.part_count;
+    kvh = idx / p.part_count;
     h = kvh * p.g + qtile / p.tiles_per_head;
     row0 = (qtile % p.tiles_per_head) * 64;
     is_resp = (part == p.S);
@@ -273,7 +274,7 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
     const bool row_ok = r_idx < p.R;
     float* dq_dst = nullptr;
     if (MODE == MLA_DQ)
-      dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + h) * kD1 + pass * NACC * 64;
+      dq_dst = p.dq_part + (((size_t)(part - p.part_first) * p.R + min(r_idx, p.R - 1)) * p.Hq + h) * kD1 + pass * NACC * 64;
     if (n_tiles == 0) {
       if (MODE == MLA_DQ && row_ok)
         for (int c = 0; c < NACC * 64; c += 4) *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -404,7 +405,7 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
 }
 
 template <int MODE>
-static ls_status_t launch_mla(const MlaBwdParams& prm, int64_t grid, cudaStream_t st) {
+static ls_status_t launch_mla(const MlaBwdParams& prm, int64_t grid, cudaStream_t st, bool timed = true) {
   static bool configured = false;
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   if (!configured) {
@@ -414,16 +415,17 @@ static ls_status_t launch_mla(const MlaBwdParams& prm, int64_t grid, cudaStream_
     configured = true;
   }
   constexpr int which = MODE == MLA_DQ ? LS_KERNEL_BWD_DQ : MODE == MLA_DK ? LS_KERNEL_BWD_DK : LS_KERNEL_BWD_DV;
-  profile_begin(which, st);
+  if (timed) profile_begin(which, st);
   bwd_mla_kernel<MODE><<<(int)grid, kMlaThreads, kMlaSmem, st>>>(prm);
-  profile_end(which, st);
+  if (timed) profile_end(which, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
-// dq_part (fp32, unscaled) and dk_resp / dv_resp (bf16) of the 576/512 shape.
+// dq_part (fp32, unscaled; only the response block's partial, at index 0, when dq_resp_only)
+// and dk_resp / dv_resp (bf16) of the 576/512 shape.
 ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
-                    void* dk_resp, void* dv_resp, int32_t* status_dev, cudaStream_t cs) {
+                    void* dk_resp, void* dv_resp, bool dq_resp_only, int32_t* status_dev, cudaStream_t cs) {
   const ls_pages_desc_t& d = h->desc;
   const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads;
   auto dense_map = [&](CUtensorMap* m, const void* base, int heads, int dim) {
@@ -447,6 +449,8 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
   P.tiles_per_head = (R + 63) / 64;
   P.nq_tiles = P.g * P.tiles_per_head;
+  P.part_first = dq_resp_only ? P.S : 0;
+  P.part_count = dq_resp_only ? 1 : P.S + 1;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * kLog2eMla;
 
@@ -460,7 +464,7 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   if (st == LS_OK) st = encode_pool_map5(&P.bv_tail, h, 1, 64, 1, true);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
-  st = launch_mla<MLA_DQ>(P, (int64_t)Hkv * (d.num_shards * h->fine + 1) * P.nq_tiles * 3, cs);
+  st = launch_mla<MLA_DQ>(P, (int64_t)Hkv * P.part_count * P.nq_tiles * 3, cs, !dq_resp_only);
   if (st != LS_OK) return st;
 
   st = dense_map(&P.a1_map, k_resp, Hkv, kD1);

@@ -881,7 +881,9 @@ extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_a
   const size_t parts = (size_t)h->desc.num_shards * h->fine;      // sub-shard partials
   // forward: sub-shard partials (O and LSE) when shards are sub-split, else nothing
   if (which == LS_WORKSPACE_FWD) return h->fine > 1 ? parts * rows * (h->desc.dim_v + 1) * sizeof(float) : 0;
-  // backward: per-partial dQ (fp32) + Delta (fp32)
+  // backward: per-partial dQ (fp32) + Delta (fp32); the aliased 576/512 path sums the prefix
+  // partials in its accumulator and keeps only the response block's partial
+  if (ls::mla_dq_fast(h)) return rows * h->desc.dim_k * sizeof(float) + rows * sizeof(float);
   return (parts + 1) * rows * h->desc.dim_k * sizeof(float) + rows * sizeof(float);
 }
 

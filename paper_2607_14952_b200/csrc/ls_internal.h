@@ -94,10 +94,19 @@ ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int
                              bool tail);
 
 // Backward of the shared-latent 576/512 shape (ls_bwd_mla.cu): fills dq_part (fp32, unscaled,
-// [(S+1), R, Hq, 576]) and the bf16 dk_resp / dv_resp.
+// [(S+1), R, Hq, 576]; with dq_resp_only just the response block's partial, [R, Hq, 576]) and
+// the bf16 dk_resp / dv_resp.
 ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
-                    void* dk_resp, void* dv_resp, int32_t* status_dev, cudaStream_t cs);
+                    void* dk_resp, void* dv_resp, bool dq_resp_only, int32_t* status_dev, cudaStream_t cs);
+
+// Prefix part of dQ for the 576/512 shape when V aliases K (ls_bwd_mla_dq.cu): every CTA walks
+// all partials, adds dq_resp (fp32, unscaled, [R, Hq, 576]) and writes the final bf16 dQ.
+ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
+                       const float* lse, const float* delta, const float* dq_resp, void* dq, int32_t* status_dev,
+                       cudaStream_t cs);
+// True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix, LS_MLA_DQ != 0).
+bool mla_dq_fast(const ls_pages* h);
 
 // Folds `fine` consecutive sub-shard partials into each of `groups` shard partials.
 ls_status_t group_merge(int groups, int fine, int64_t rows, int dv, const float* in_o, const float* in_lse,

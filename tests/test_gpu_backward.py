@@ -125,3 +125,18 @@ def test_alternative_kernels_stay_correct(fwd_pair, bwd_pair, monkeypatch):
         case = parity.Case(cfg)
         fw = parity.check_forward(case, per_shard=True)
         parity.check_backward(case, fw)
+
+
+@pytest.mark.parametrize("mla_dq", ["0", "1"])
+def test_shared_latent_dq_paths(mla_dq, monkeypatch):
+    # 576/512 pools whose V aliases K take the transposed dQ kernel that walks every partial in
+    # one accumulator (LS_MLA_DQ=1, the default); the per-partial kernel stays selectable.  Cases: ragged tail page, several heads per
+    # latent, more than one row tile per head, a response longer than one key tile.
+    monkeypatch.setenv("LS_MLA_DQ", mla_dq)
+    for cfg in (small("mla_t_pg64", Dk=576, Dv=512, v_aliases_k=True, Hq=8, Hkv=1, P=64 * 37 + 21, page_size=64,
+                      num_shards=5, R=150),
+                small("mla_t_pg512", Dk=576, Dv=512, v_aliases_k=True, Hq=2, Hkv=1, P=512 * 5 + 300, page_size=512,
+                      num_shards=3, R=64)):
+        case = parity.Case(cfg)
+        fw = parity.check_forward(case, per_shard=True)
+        parity.check_backward(case, fw)
