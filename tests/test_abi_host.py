@@ -103,3 +103,21 @@ def test_error_paths_before_any_launch():
     pages = bld(page_table=np.array([3, 0, 2, 1]), num_phys_pages=6)          # pool larger than Np is fine
     assert B.ls_prefix_pages_export(pages)["page_table"].tolist() == [3, 0, 2, 1]
     assert B.lib().ls_status_string(B.LS_ERR_TIMEOUT) != b"unknown status"
+
+
+def test_backward_workspace_sizes(monkeypatch):
+    # per-partial fp32 dQ sums + Delta in general; the aliased 576/512 shape sums the prefix
+    # partials in its accumulator and keeps only the response block's partial
+    R, Hq = 96, 8
+    rows = R * Hq
+    plain = B.ls_prefix_pages_build(256 * 12, 256, 3, 2, 256, 256, 12)
+    assert B.ls_replay_attn_workspace_bytes(plain, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == (3 + 1) * rows * 256 * 4 + rows * 4
+    assert B.ls_replay_attn_workspace_bytes(plain, R, Hq, 0.0625, B.LS_WORKSPACE_FWD) == 0
+    mla = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=True)
+    monkeypatch.delenv("LS_MLA_DQ", raising=False)
+    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == rows * 576 * 4 + rows * 4
+    monkeypatch.setenv("LS_MLA_DQ", "0")
+    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == (4 + 1) * rows * 576 * 4 + rows * 4
+    monkeypatch.delenv("LS_MLA_DQ")
+    empty = B.ls_prefix_pages_build(0, 64, 1, 1, 576, 512, 1, v_aliases_k=True)
+    assert B.ls_replay_attn_workspace_bytes(empty, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == (1 + 1) * rows * 576 * 4 + rows * 4
