@@ -18,15 +18,18 @@
  *    outputs are fully contiguous in the stated shape.  All bases 16-byte aligned.
  *  - The caller owns every buffer, including the page pool and the workspaces.
  *    The library owns only the opaque ls_pages_t handle and its small metadata
- *    arrays, and never writes the pool.
+ *    arrays.  It never writes a pool page that the prefix maps; the only pool pages
+ *    it writes are the unmapped ones a caller hands to ls_suffix_pages_append.
  *  - All compute calls enqueue work on `stream` (a cudaStream_t passed as
  *    void*, NULL = default stream) and return without synchronising.  They
  *    allocate nothing.
  *  - Every call returns an ls_status_t; nothing aborts or throws across the ABI.
  *    Argument, shape, alignment and page-table validation happen on the host
  *    before any launch.  Conditions found on the device (a bounded wait that ran
- *    out) are written to `status_dev` (one int32, nullable, must be zeroed by
- *    the caller) and never trap.
+ *    out, a non-finite merged log-normaliser) are written to `status_dev` (one
+ *    int32, nullable, must be zeroed by the caller) and never trap.
+ *  - A handle belongs to the device that was current in ls_prefix_pages_build; a
+ *    compute call made with another device current returns LS_ERR_STALE.
  *  - GQA: query head h uses KV head h / (num_q_heads / num_kv_heads).
  *  - Response query t sits at global position P + t; it sees every prefix
  *    position and the response positions j <= t.
@@ -54,10 +57,10 @@ typedef enum {
   LS_ERR_UNSUPPORTED_SHAPE = -3,
   LS_ERR_ALIGNMENT = -4,
   LS_ERR_WORKSPACE = -5,
-  LS_ERR_STALE = -6,
+  LS_ERR_STALE = -6,       /* handle of another device, or its suffix changed since the caller looked */
   LS_ERR_CUDA = -7,
-  LS_ERR_TIMEOUT = -8,
-  LS_ERR_NONFINITE = -9
+  LS_ERR_TIMEOUT = -8,     /* device side: a bounded wait ran out */
+  LS_ERR_NONFINITE = -9    /* device side: a merged log-normaliser is NaN or +inf */
 } ls_status_t;
 
 typedef enum {
@@ -79,7 +82,10 @@ typedef struct {
   int32_t dim_v;
   int32_t v_aliases_k;     /* 1: V is the first dim_v channels of the K page (shared latent);
                               v_pool may then be NULL */
-  int32_t reserved;
+  int32_t stream_budget_kib; /* 0 = default (32768).  Upper bound, in KiB, for the K+V bytes of one
+                              (KV head, key range) stream that many CTAs read together: a shard above
+                              it is walked as up to 16 consecutive sub-ranges, which keeps the stream
+                              in L2.  Results do not depend on it beyond fp32 summation order. */
   int64_t num_phys_pages;  /* pool capacity, >= ceil(P / page_size) */
   const void* k_pool;      /* [num_phys_pages, page_size, num_kv_heads, dim_k] bf16, or NULL */
   const void* v_pool;      /* [num_phys_pages, page_size, num_kv_heads, dim_v] bf16, or NULL */
@@ -125,24 +131,23 @@ ls_status_t ls_prefix_pages_checksum(const ls_pages_t* pages, uint64_t* scratch_
 ls_status_t ls_prefix_pages_destroy(ls_pages_t* pages);
 
 typedef struct {
-  int32_t R;             /* response tokens, >= 1 */
+  int32_t R;             /* response tokens of this call (a whole response, or one block of it), >= 1 */
   int32_t num_q_heads;   /* Hq */
   float scale;           /* softmax scale, e.g. 1/sqrt(dim_k) */
   int32_t flags;         /* 0, or LS_FLAG_* bits */
+  uint64_t generation;   /* 0 = not checked; otherwise the value of ls_pages_generation() the caller
+                            planned this call against: a handle whose suffix changed since then
+                            (append / pop) makes the call return LS_ERR_STALE before any launch */
 } ls_attn_params_t;
 
-/* Diagnostic switches for profiling the kernel pipelines: they skip one stage (operand
- * loads, tensor-core instructions, or the per-row arithmetic) while keeping every barrier
- * hand-off, so the cost of the remaining stages can be timed.  Outputs are meaningless
- * when any of them is set. */
-#define LS_FLAG_ABLATE_LOADS   (1 << 16)
-#define LS_FLAG_ABLATE_MMA     (1 << 17)
-#define LS_FLAG_ABLATE_SOFTMAX (1 << 18)
-#define LS_FLAG_ABLATE_MASK    (7 << 16)
+/* Backward only: add the retained suffix gradient pages of the block that was popped last
+ * (the one being replayed) to dk_resp / dv_resp.  See ls_suffix_pages_append. */
+#define LS_FLAG_ADD_SUFFIX_GRAD (1 << 0)
 
-enum { LS_WORKSPACE_FWD = 0, LS_WORKSPACE_BWD = 1 };
+enum { LS_WORKSPACE_FWD = 0, LS_WORKSPACE_BWD = 1, LS_WORKSPACE_FWD_MERGED = 2 };
 
-/* Bytes of caller-provided scratch needed by the forward (0) or the backward. */
+/* Bytes of caller-provided scratch needed by ls_replay_attn_fwd (0), ls_replay_attn_bwd (1) or
+ * ls_replay_attn_fwd_merged (2).  Depends on the handle and on prm->R, prm->num_q_heads only. */
 size_t ls_replay_attn_workspace_bytes(const ls_pages_t* pages, const ls_attn_params_t* prm, int which);
 
 /*
@@ -154,10 +159,13 @@ size_t ls_replay_attn_workspace_bytes(const ls_pages_t* pages, const ls_attn_par
  *  q [R,Hq,dim_k] bf16; k_resp [R,Hkv,dim_k], v_resp [R,Hkv,dim_v] bf16
  *  o_part [(S+1),R,Hq,dim_v] fp32; lse_part [(S+1),R,Hq] fp32
  *  workspace: ls_replay_attn_workspace_bytes(.., LS_WORKSPACE_FWD) bytes of device memory,
- *  16-byte aligned; 0 (workspace may be NULL) unless the plan splits a shard into
- *  cache-sized sub-shards, whose partials are held there and merged per shard with the same
- *  Eq. qwen-lse-parts arithmetic before the call returns its (S+1) partials.  A workspace
- *  that is too small gives LS_ERR_WORKSPACE before any launch.
+ *  16-byte aligned: 0 (workspace may be NULL) unless a shard is walked as several
+ *  sub-ranges (stream_budget_kib), in which case it holds a few KB of hand-over counters:
+ *  the CTAs of consecutive sub-ranges fold their results into the shard's partial in a
+ *  fixed order with the Eq. qwen-lse-parts arithmetic, so the caller still receives (S+1)
+ *  partials and no per-sub-range partial ever exists in memory.  A workspace that is too
+ *  small gives LS_ERR_WORKSPACE before any launch.
+ * The handle must have no suffix blocks (LS_ERR_INVALID_ARG): use ls_replay_attn_fwd_merged.
  */
 ls_status_t ls_replay_attn_fwd(const ls_pages_t* pages, const ls_attn_params_t* prm,
                                const void* q, const void* k_resp, const void* v_resp,
@@ -172,20 +180,52 @@ ls_status_t ls_replay_attn_fwd(const ls_pages_t* pages, const ls_attn_params_t* 
  *  o_part [num_parts, rows, dim_v] fp32; lse_part [num_parts, rows] fp32
  *  o_bf16 [rows, dim_v] bf16 (nullable); o_f32 [rows, dim_v] fp32 (nullable; the backward
  *  consumes it); lse [rows] fp32.
+ * A merged l that is NaN or +inf (only possible from non-finite inputs) is still written,
+ * and LS_ERR_NONFINITE goes to *status_dev (nullable).
  */
 ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim_v,
                          const float* o_part, const float* lse_part,
-                         void* o_bf16, float* o_f32, float* lse, void* stream);
+                         void* o_bf16, float* o_f32, float* lse, int32_t* status_dev, void* stream);
+
+/*
+ * Replay forward with the merge folded in: the composed output of Eq. qwen-global-attn and
+ * its log-normaliser, without the per-shard partials ever reaching memory.  This is the
+ * form of the score-only passes of a group member (old and reference scoring keep no
+ * per-shard state, Sec. "Four-Block Response Replay") and of every block of a blockwise
+ * replay.  The partials are the response block, every prefix shard (sub-range by
+ * sub-range) and every appended suffix block; the CTAs that own a row tile fold them into
+ * o_f32 / lse in that fixed order with the pairwise form of Eq. qwen-lse-parts
+ * (m = max(l, l_r); a = e^{l-m} + e^{l_r-m}; o = (e^{l-m} o + e^{l_r-m} o_r)/a; l = m + log a),
+ * so the result is bit-reproducible; the last one also writes o_bf16.
+ *  Response query t sits at global position P + T + t (T = suffix tokens) and sees all P
+ *  prefix positions, all T suffix positions and the response positions j <= t.
+ *  q [R,Hq,dim_k], k_resp [R,Hkv,dim_k], v_resp [R,Hkv,dim_v] bf16
+ *  o_bf16 [R,Hq,dim_v] bf16 (nullable); o_f32 [R,Hq,dim_v] fp32 (required: it is the running
+ *  value; the backward consumes it); lse [R,Hq] fp32.
+ *  workspace: ls_replay_attn_workspace_bytes(.., LS_WORKSPACE_FWD_MERGED) bytes (hand-over
+ *  counters; for the 576/512 shape also a second running l of R*Hq floats).
+ */
+ls_status_t ls_replay_attn_fwd_merged(const ls_pages_t* pages, const ls_attn_params_t* prm,
+                                      const void* q, const void* k_resp, const void* v_resp,
+                                      void* o_bf16, float* o_f32, float* lse,
+                                      void* workspace, size_t workspace_bytes,
+                                      int32_t* status_dev, void* stream);
 
 /*
  * Replay backward with the prefix detached (Sec. "Lazy Gradient Pages"):
  *   Delta = dO.O; p_tj = exp(s_tj - LSE); ds_tj = p_tj (dO_th.v_j - Delta)
- *   dQ_th = scale * sum_j ds_tj k_j over prefix and response keys; per-shard
- *           contributions are summed on the device (Eq. qwen-dq-reduce)
+ *   dQ_th = scale * sum_j ds_tj k_j over prefix, suffix and response keys; the per-shard
+ *           contributions are summed on the device in a fixed order (Eq. qwen-dq-reduce)
  *   dK_resp_j = scale * sum_{t>=j,h in group} ds_tj q_th;  dV_resp_j = sum p_tj dO_th
- * Prefix pages get no gradient and are not written.
- *  o_f32 [R,Hq,dim_v], lse [R,Hq] from ls_lse_merge; d_o [R,Hq,dim_v] bf16
- *  dq [R,Hq,dim_k], dk_resp [R,Hkv,dim_k], dv_resp [R,Hkv,dim_v] bf16
+ * Prefix pages get no gradient and are not written.  With suffix blocks on the handle
+ * (blockwise replay) the keys of every suffix block additionally receive
+ *   dk_grad[key] += scale * sum_{t,h in group} ds_t,key q_th,  dv_grad[key] += sum p_t,key dO_th
+ * in the fp32 gradient pages given to ls_suffix_pages_reserve, and LS_FLAG_ADD_SUFFIX_GRAD
+ * adds the gradient pages of the block popped last to dk_resp / dv_resp.
+ *  o_f32 [R,Hq,dim_v], lse [R,Hq] from ls_lse_merge / ls_replay_attn_fwd_merged;
+ *  d_o [R,Hq,dim_v] bf16; dq [R,Hq,dim_k], dk_resp [R,Hkv,dim_k], dv_resp [R,Hkv,dim_v] bf16
+ *  workspace: ls_replay_attn_workspace_bytes(.., LS_WORKSPACE_BWD) bytes, 16-byte aligned: one
+ *  fp32 running dQ of R*Hq*dim_k, Delta and the hand-over counters.
  */
 ls_status_t ls_replay_attn_bwd(const ls_pages_t* pages, const ls_attn_params_t* prm,
                                const void* q, const void* k_resp, const void* v_resp,
@@ -195,23 +235,59 @@ ls_status_t ls_replay_attn_bwd(const ls_pages_t* pages, const ls_attn_params_t* 
                                int32_t* status_dev, void* stream);
 
 /*
+ * Response suffix as temporary pages behind the resident prefix (Sec. "Four-Block Response
+ * Replay": a no-grad suffix pass appends each block's KV pages, the policy pass walks the
+ * blocks in reverse and pops them; Sec. "Lazy Gradient Pages": K/V gradient pages are kept
+ * for the response suffix only; Sec. "LongStraw: Long-Context Execution Design": append/pop
+ * transactions with a version check at every replay boundary; Sec. "State Inventory and
+ * Ownership": branches may append suffix pages but cannot mutate the shared prefix).
+ *
+ * ls_suffix_pages_reserve: call once before the first append.  max_blocks, max_pages bound
+ * the suffix; dk_grad [max_pages, page_size, Hkv, dim_k] and dv_grad [.., dim_v] are the
+ * caller-owned fp32 gradient pages, indexed by suffix page SLOT (the s-th page appended and
+ * not yet popped has slot s), or both NULL for forward-only use.  Allocates the handle's
+ * (small) device metadata for that capacity; no later suffix call allocates.
+ *
+ * ls_suffix_pages_append: copies n_tokens of k_block [n,Hkv,dim_k] / v_block [n,Hkv,dim_v]
+ * (bf16, device) into ceil(n/page_size) pool pages phys_pages[] (host array), which must be
+ * distinct, inside the pool and mapped neither by the prefix nor by the suffix
+ * (LS_ERR_BAD_PAGE_TABLE); the unused tail of the last page is zero-filled and the block's
+ * gradient pages are zeroed.  With v_aliases_k, v_block is ignored.  Every block starts on a
+ * fresh page.  Enqueued on `stream`; later attention calls on the same stream see the block.
+ *
+ * ls_suffix_pages_pop: unmaps the last block (its pool pages are the caller's again; its
+ * gradient pages keep their contents for LS_FLAG_ADD_SUFFIX_GRAD).  Host-only.
+ *
+ * Each append / pop increments ls_pages_generation (1 after build).
+ * Supported for head dims 128 and 256 (LS_ERR_UNSUPPORTED_SHAPE for 576/512).
+ */
+ls_status_t ls_suffix_pages_reserve(ls_pages_t* pages, int32_t max_blocks, int32_t max_pages,
+                                    float* dk_grad, float* dv_grad);
+ls_status_t ls_suffix_pages_append(ls_pages_t* pages, int32_t n_tokens, const int32_t* phys_pages,
+                                   const void* k_block, const void* v_block, void* stream);
+ls_status_t ls_suffix_pages_pop(ls_pages_t* pages);
+uint64_t ls_pages_generation(const ls_pages_t* pages);
+int64_t ls_suffix_pages_tokens(const ls_pages_t* pages);
+
+/*
  * ls_replay_attn_bwd for callers that cannot hand over scratch memory (the paper has no
  * counterpart; this is a packaging variant, the arithmetic and the outputs are those of
  * ls_replay_attn_bwd).  A replay scheduler that has sized the page pool to fill the GPU, or
  * code running under a framework whose allocator already owns all device memory, has
  * nowhere to take a workspace from at backward time: a late cudaMalloc there can fail or
  * stall the whole device.  This call therefore allocates nothing, in the library or in
- * CUDA: the per-partial dQ sums and Delta go to a fixed array of LS_STATIC_SCRATCH_BYTES
- * that is part of the library's device image, so every GPU that loads the library holds
- * that much memory until the process exits.
+ * CUDA: Delta, the hand-over counters and the fp32 running dQ go to a fixed array of
+ * LS_STATIC_SCRATCH_BYTES that is part of the library's device image, so every GPU that
+ * loads the library holds that much memory until the process exits.
  *  - Shapes whose backward workspace (ls_replay_attn_workspace_bytes) exceeds
  *    LS_STATIC_SCRATCH_BYTES are rejected with LS_ERR_WORKSPACE before any launch.
  *  - The first call on each device looks up the array's device address (the device must be
  *    current); make that first call before starting any stream capture.
  *  - All calls on a device share the one array, which keeps the previous call's contents.
- *    Nothing needs clearing (every word that is read is written first by the same call),
- *    but two calls whose kernels overlap on the GPU (different streams) race on it:
- *    serialise them.
+ *    The call clears what must start at zero (the hand-over counters, by a memset on
+ *    `stream`); every other word is written before it is read.  Two calls whose kernels
+ *    overlap on the GPU (different streams) race on the array: serialise them.
+ *  - The handle must belong to the current device (LS_ERR_STALE otherwise).
  * Arguments and errors otherwise as ls_replay_attn_bwd.
  */
 #define LS_STATIC_SCRATCH_BYTES (32u << 20)

@@ -18,21 +18,23 @@ LS_OK = 0
 LS_ERR_INVALID_ARG, LS_ERR_BAD_PAGE_TABLE, LS_ERR_UNSUPPORTED_SHAPE, LS_ERR_ALIGNMENT = -1, -2, -3, -4
 LS_ERR_WORKSPACE, LS_ERR_STALE, LS_ERR_CUDA, LS_ERR_TIMEOUT, LS_ERR_NONFINITE = -5, -6, -7, -8, -9
 LS_SHARD_CONTIGUOUS, LS_SHARD_CYCLIC, LS_SHARD_ZIGZAG = 0, 1, 2
-LS_WORKSPACE_FWD, LS_WORKSPACE_BWD = 0, 1
+LS_WORKSPACE_FWD, LS_WORKSPACE_BWD, LS_WORKSPACE_FWD_MERGED = 0, 1, 2
+LS_FLAG_ADD_SUFFIX_GRAD = 1
 LS_KERNEL_FWD, LS_KERNEL_BWD_DQ, LS_KERNEL_BWD_DK, LS_KERNEL_BWD_DV = 0, 1, 2, 3
 
 
 class ls_pages_desc_t(C.Structure):
     _fields_ = [("prefix_len", C.c_int64), ("page_size", C.c_int32), ("num_shards", C.c_int32),
                 ("shard_policy", C.c_int32), ("num_kv_heads", C.c_int32), ("dim_k", C.c_int32),
-                ("dim_v", C.c_int32), ("v_aliases_k", C.c_int32), ("reserved", C.c_int32),
+                ("dim_v", C.c_int32), ("v_aliases_k", C.c_int32), ("stream_budget_kib", C.c_int32),
                 ("num_phys_pages", C.c_int64), ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
                 ("k_stride_page", C.c_int64), ("k_stride_tok", C.c_int64), ("k_stride_head", C.c_int64),
                 ("v_stride_page", C.c_int64), ("v_stride_tok", C.c_int64), ("v_stride_head", C.c_int64)]
 
 
 class ls_attn_params_t(C.Structure):
-    _fields_ = [("R", C.c_int32), ("num_q_heads", C.c_int32), ("scale", C.c_float), ("flags", C.c_int32)]
+    _fields_ = [("R", C.c_int32), ("num_q_heads", C.c_int32), ("scale", C.c_float), ("flags", C.c_int32),
+                ("generation", C.c_uint64)]
 
 
 class LsError(RuntimeError):
@@ -60,7 +62,16 @@ def lib():
         L.ls_replay_attn_workspace_bytes.argtypes = [vp, C.POINTER(ls_attn_params_t), C.c_int]
         L.ls_replay_attn_workspace_bytes.restype = C.c_size_t
         L.ls_replay_attn_fwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
-        L.ls_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp]
+        L.ls_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.ls_replay_attn_fwd_merged.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, C.c_size_t,
+                                                vp, vp]
+        L.ls_suffix_pages_reserve.argtypes = [vp, i32, i32, vp, vp]
+        L.ls_suffix_pages_append.argtypes = [vp, i32, vp, vp, vp, vp]
+        L.ls_suffix_pages_pop.argtypes = [vp]
+        L.ls_pages_generation.argtypes = [vp]
+        L.ls_pages_generation.restype = C.c_uint64
+        L.ls_suffix_pages_tokens.argtypes = [vp]
+        L.ls_suffix_pages_tokens.restype = C.c_int64
         L.ls_replay_attn_bwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                          C.c_size_t, vp, vp]
         L.ls_replay_attn_bwd_static.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, vp, vp,
@@ -75,7 +86,9 @@ def lib():
         L.ls_status_string.argtypes = [C.c_int]
         L.ls_status_string.restype = C.c_char_p
         for f in ("ls_prefix_pages_build", "ls_prefix_pages_export", "ls_prefix_pages_checksum",
-                  "ls_prefix_pages_destroy", "ls_replay_attn_fwd", "ls_lse_merge", "ls_replay_attn_bwd"):
+                  "ls_prefix_pages_destroy", "ls_replay_attn_fwd", "ls_lse_merge", "ls_replay_attn_bwd",
+                  "ls_replay_attn_fwd_merged", "ls_suffix_pages_reserve", "ls_suffix_pages_append",
+                  "ls_suffix_pages_pop"):
             getattr(L, f).restype = C.c_int
         _LIB = L
     return _LIB
@@ -115,13 +128,14 @@ class Pages:
 
 def ls_prefix_pages_build(prefix_len, page_size, num_shards, num_kv_heads, dim_k, dim_v, num_phys_pages,
                           page_table=None, k_pool=None, v_pool=None, shard_policy=LS_SHARD_CONTIGUOUS,
-                          v_aliases_k=False):
+                          v_aliases_k=False, stream_budget_kib=0):
     """k_pool/v_pool: bf16 CUDA tensors [num_phys_pages, page_size, num_kv_heads, dim] (last dim dense) or
     None for a host-only plan.  page_table: int32 numpy array or None (identity)."""
     d = ls_pages_desc_t()
     d.prefix_len, d.page_size, d.num_shards, d.shard_policy = prefix_len, page_size, num_shards, shard_policy
     d.num_kv_heads, d.dim_k, d.dim_v, d.v_aliases_k = num_kv_heads, dim_k, dim_v, int(bool(v_aliases_k))
     d.num_phys_pages = num_phys_pages
+    d.stream_budget_kib = stream_budget_kib
     if k_pool is not None:
         assert k_pool.dtype == torch.bfloat16 and k_pool.stride(-1) == 1
         d.k_pool = k_pool.data_ptr()
@@ -161,8 +175,8 @@ def ls_prefix_pages_checksum(pages):
     return int(out.value)
 
 
-def _params(R, Hq, scale, flags=0):
-    return ls_attn_params_t(R, Hq, float(scale), flags)
+def _params(R, Hq, scale, flags=0, generation=0):
+    return ls_attn_params_t(R, Hq, float(scale), flags, generation)
 
 
 def ls_replay_attn_workspace_bytes(pages, R, Hq, scale, which):
@@ -171,7 +185,7 @@ def ls_replay_attn_workspace_bytes(pages, R, Hq, scale, which):
 
 
 def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=None, status=None, flags=0,
-                       workspace=None):
+                       workspace=None, generation=0):
     """Returns (o_part [(S+1),R,Hq,Dv] fp32, lse_part [(S+1),R,Hq] fp32)."""
     R, Hq, _ = q.shape
     S, Dv = pages.desc.num_shards, pages.desc.dim_v
@@ -179,7 +193,7 @@ def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=No
         o_part = torch.empty((S + 1, R, Hq, Dv), dtype=torch.float32, device=q.device)
     if lse_part is None:
         lse_part = torch.empty((S + 1, R, Hq), dtype=torch.float32, device=q.device)
-    prm = _params(R, Hq, scale, flags)
+    prm = _params(R, Hq, scale, flags, generation)
     if workspace is None:
         nbytes = ls_replay_attn_workspace_bytes(pages, R, Hq, scale, LS_WORKSPACE_FWD)
         if nbytes:
@@ -191,7 +205,7 @@ def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=No
     return o_part, lse_part
 
 
-def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=True, want_f32=True):
+def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=True, want_f32=True, status=None):
     """o_part [parts, ..., Dv] fp32, lse_part [parts, ...] fp32 -> (o_bf16, o_f32, lse)."""
     parts, dv = o_part.shape[0], o_part.shape[-1]
     rows = lse_part[0].numel()
@@ -203,13 +217,61 @@ def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=
     if lse is None:
         lse = torch.empty(shape[:-1], dtype=torch.float32, device=o_part.device)
     st = lib().ls_lse_merge(parts, rows, dv, _ptr(o_part), _ptr(lse_part), _ptr(o_bf16), _ptr(o_f32), _ptr(lse),
-                            _stream())
+                            _ptr(status), _stream())
     _check(st, "ls_lse_merge")
     return o_bf16, o_f32, lse
 
 
+def ls_replay_attn_fwd_merged(pages, q, k_resp, v_resp, scale, o_bf16=None, o_f32=None, lse=None, status=None,
+                              workspace=None, want_bf16=True, generation=0):
+    """Forward with the merge folded in: returns (o_bf16 [R,Hq,Dv] or None, o_f32, lse [R,Hq])."""
+    R, Hq, _ = q.shape
+    Dv = pages.desc.dim_v
+    if o_bf16 is None and want_bf16:
+        o_bf16 = torch.empty((R, Hq, Dv), dtype=torch.bfloat16, device=q.device)
+    if o_f32 is None:
+        o_f32 = torch.empty((R, Hq, Dv), dtype=torch.float32, device=q.device)
+    if lse is None:
+        lse = torch.empty((R, Hq), dtype=torch.float32, device=q.device)
+    prm = _params(R, Hq, scale, 0, generation)
+    if workspace is None:
+        nbytes = ls_replay_attn_workspace_bytes(pages, R, Hq, scale, LS_WORKSPACE_FWD_MERGED)
+        workspace = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=q.device)
+    st = lib().ls_replay_attn_fwd_merged(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp),
+                                         _ptr(o_bf16), _ptr(o_f32), _ptr(lse), _ptr(workspace), workspace.numel(),
+                                         _ptr(status), _stream())
+    _check(st, "ls_replay_attn_fwd_merged")
+    return o_bf16, o_f32, lse
+
+
+def ls_suffix_pages_reserve(pages, max_blocks, max_pages, dk_grad=None, dv_grad=None):
+    """dk_grad / dv_grad: fp32 CUDA tensors [max_pages, page_size, Hkv, Dk|Dv] or None (forward only)."""
+    _check(lib().ls_suffix_pages_reserve(pages.handle, max_blocks, max_pages, _ptr(dk_grad), _ptr(dv_grad)),
+           "ls_suffix_pages_reserve")
+    pages.grad_pages = (dk_grad, dv_grad)
+
+
+def ls_suffix_pages_append(pages, phys_pages, k_block, v_block=None):
+    """Appends one block of response K/V ([n,Hkv,D] bf16) into the given free pool pages."""
+    ids = np.ascontiguousarray(phys_pages, dtype=np.int32)
+    _check(lib().ls_suffix_pages_append(pages.handle, k_block.shape[0], ids.ctypes.data_as(C.c_void_p), _ptr(k_block),
+                                        _ptr(v_block), _stream()), "ls_suffix_pages_append")
+
+
+def ls_suffix_pages_pop(pages):
+    _check(lib().ls_suffix_pages_pop(pages.handle), "ls_suffix_pages_pop")
+
+
+def ls_pages_generation(pages):
+    return int(lib().ls_pages_generation(pages.handle))
+
+
+def ls_suffix_pages_tokens(pages):
+    return int(lib().ls_suffix_pages_tokens(pages.handle))
+
+
 def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspace=None, dq=None, dk_resp=None,
-                       dv_resp=None, status=None, flags=0):
+                       dv_resp=None, status=None, flags=0, generation=0):
     """Returns (dq, dk_resp, dv_resp) in bf16."""
     R, Hq, _ = q.shape
     if workspace is None:
@@ -221,7 +283,7 @@ def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspa
         dk_resp = torch.empty_like(k_resp)
     if dv_resp is None:
         dv_resp = torch.empty_like(v_resp)
-    prm = _params(R, Hq, scale, flags)
+    prm = _params(R, Hq, scale, flags, generation)
     st = lib().ls_replay_attn_bwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_f32),
                                   _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk_resp), _ptr(dv_resp), _ptr(workspace),
                                   workspace.numel(), _ptr(status), _stream())

@@ -2,30 +2,27 @@
 // for sm_100a.
 //
 //   Delta_th = dO_th . O_th;  p_tj = exp(s_tj - LSE_th);  ds_tj = p_tj (dO_th . v_j - Delta_th)
-//   dQ_th = scale * sum_j ds_tj k_j      (prefix and response keys; per-partial sums reduced here)
-//   dK_j  = scale * sum_{t>=j,h} ds_tj q_th,   dV_j = sum_{t>=j,h} p_tj dO_th   (response keys only)
+//   dQ_th = scale * sum_j ds_tj k_j      (prefix, suffix and response keys)
+//   dK_j  = scale * sum_{t,h} ds_tj q_th,   dV_j = sum_{t,h} p_tj dO_th   (response and suffix keys only)
 //
-// One row-stationary kernel serves all three gradients.  A CTA keeps 128 "rows" resident in
-// shared memory (operands A1, A2) and streams 128-wide "column" tiles through a small ring of
-// chunks (128 columns x 128 channels each):
-//     S = A1 B1^T,  T = A2 B2^T      (tcgen05.mma 128x128x16, operands in shared memory)
-//     E = f(S, T)                     (one thread per row; bf16, written over S in TMEM,
-//                                      in four 32-column quarters, each with its own barrier)
-//     ACC += E B3                     (E read from TMEM, B3 MN-major from shared memory; the
-//                                      MMAs of a quarter start as soon as that quarter is ready)
-//   mode DQ: rows = 128 queries of one head, columns = keys of one partial (prefix shard
-//            through the page table, or the causal response block); A1 = Q, A2 = dO,
-//            B1 = B3 = K, B2 = V; E = p (T - Delta_row).  The prefix needs no dK/dV, so this
-//            three-GEMM form is all the prefix ever costs.
-//   mode DK: rows = 128 response keys, columns = queries (t >= j) of every head of the group;
-//            A1 = K_resp, A2 = V_resp, B1 = B3 = Q, B2 = dO; E = p (T - Delta_col).
-//   mode DV: as DK without T; B3 = dO; E = p.
-// The 128-wide tile halves how often the resident operand is re-read from shared memory per
-// key (a 64-wide S/T MMA is bound by that re-read, not by the tensor pipe).  It leaves TMEM
-// room for one S and one T buffer only: ACC [0, D), S [D, D+128), T [D+128, D+256).
+// All kernels are row-stationary: a CTA keeps 128 "rows" resident in shared memory (operands
+// A1, A2) and streams "column" tiles through a small ring of chunks:
+//     S = A1 B1^T,  T = A2 B2^T      (tcgen05.mma, operands in shared memory)
+//     E = f(S, T)                     (row threads; bf16, written over S in TMEM, quarter by quarter)
+//     ACC += E B3                     (E read from TMEM, B3 MN-major from shared memory)
+//   dQ pass (bwd_dq3_kernel for head dim 256, bwd_dq2_kernel for 128; CTA pairs): rows = queries
+//            of one head, columns = keys of one part (prefix sub-shard or suffix block through
+//            the page table, or the causal response block); A1 = Q, A2 = dO, B1 = B3 = K,
+//            B2 = V; E = p (T - Delta_row).  The prefix needs no dK/dV, so this three-GEMM form
+//            is all the prefix ever costs.  The parts of one row tile are summed in a fixed
+//            order through one fp32 running dQ (ordered hand-over between CTAs); the last part
+//            writes the scaled bf16 result.
+//   dK / dV pass (bwd_kv_kernel): rows = 128 keys -- of the response block (columns = queries
+//            t >= j of every head of the group) or of a suffix block read through its pages
+//            (columns = every query); A1 = K, A2 = V, B1 = B3 = Q, B2 = dO; E = p (T - Delta_col)
+//            for dK, E = p with B3 = dO for dV.
 #include <cuda_bf16.h>
 
-#include <cstdlib>
 #include <mutex>
 
 #include "ls_internal.h"
@@ -33,37 +30,42 @@
 
 namespace ls {
 
-enum { MODE_DQ = 0, MODE_DK = 1, MODE_DV = 2 };
+enum { MODE_DK = 1, MODE_DV = 2 };
 
 struct BwdParams {
   CUtensorMap a1_map, a2_map;                 // stationary rows: box 64 x 128 tokens x 1 group
-  // streamed chunks of 128 columns x 128 channels: box 64 x 128 tokens x 2 groups, or, when the
-  // pages hold 64 tokens, 64 x 64 x 1 (four boxes per chunk)
-  CUtensorMap bk_map, bk_tail, bv_map, bv_tail;   // prefix pool K and V (mode DQ)
-  CUtensorMap b1r_map, b2r_map, b3r_map;          // dense sources: response K/V/K (DQ) or Q/dO/(Q|dO) (DK, DV)
-  // CTA-pair variant of the dQ pass: each CTA loads half of every streamed operand.
-  //   *_s: 64 columns x 128 channels (box 64 x 64 tokens x 2 groups) for S and T
-  //   *_m: 128 columns x 64 channels (box 64 x 128 x 1, or 64 x 64 x 1 on 64-token pages) for ACC
-  CUtensorMap pk_s, pk_s_tail, pv_s, pv_s_tail, pk_m, pk_m_tail;   // prefix pool
+  CUtensorMap b1r_map, b2r_map, b3r_map;      // dK / dV pass: Q / dO / (Q | dO) as 128 columns x 128 channels
+  // dQ pass on CTA pairs: each CTA loads half of every streamed operand.
+  //   *_s: 64 columns x 128 channels (box 64 x 64 tokens x 2 groups)
+  //   *_m: 128 columns x 64 channels (box 64 x 128 x 1, or 64 x 64 x 1 on 64-token pages)
+  CUtensorMap pk_s, pk_s_tail, pv_s, pv_s_tail, pk_m, pk_m_tail;   // pool
   CUtensorMap rk_s, rv_s, rk_m;                                     // response K, V, K
   CUtensorMap pv_m, pv_m_tail, rv_m;   // V as 128 columns x 64 channels (256-key tile variant)
-  const int32_t* shard_phys_pages;
-  const int32_t* shard_page_offset;
-  const int32_t* shard_tail_slot;
-  const int64_t* shard_tokens;
+  const int32_t* part_pages;
+  const int32_t* part_page_offset;
+  const int32_t* part_tail_slot;
+  const int64_t* part_tokens;
   const float* lse;      // [R, Hq]
   const float* delta;    // [R, Hq]
-  float* dq_part;        // [(S+1), R, Hq, D] fp32, unscaled (mode DQ)
-  __nv_bfloat16* out;    // dk_resp or dv_resp [R, Hkv, D] (modes DK, DV)
+  float* dq_acc;         // [R, Hq, D] fp32 running sum over parts, unscaled (dQ pass)
+  __nv_bfloat16* dq;     // [R, Hq, D] final result, written by the last part of every chain
+  int* ctl;              // hand-over control words (dQ pass)
+  __nv_bfloat16* out;    // dk_resp or dv_resp [R, Hkv, D] (dK / dV pass over the response block)
+  float* grad;           // dK / dV pass: fp32 gradient pages [slot, page, Hkv, D]; accumulated into (suffix
+                         // keys) or added to `out` (response keys, when not NULL)
   int32_t* status;
-  int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
-  int packed;    // pair dQ pass only: one Q tile holds every (head, token) row of a KV group
+  long long* timing;     // diagnostic builds only
+  int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  int packed;    // dQ pass: one Q tile holds every (head, token) row of a KV group
+  // dK / dV pass: keys of a suffix block (1) read through pages [key_page_off, ..) of part_pages,
+  // key_tokens of them, first gradient slot grad_slot0; or the response block (0)
+  int keys_paged, key_page_off, key_tokens, grad_slot0;
   float scale, scale_log2;
 };
 
 #ifdef LS_TIMING
 #define LS_BTWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
-#define LS_BTDUMP(slot, val) do { if (kTimedMode && blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
+#define LS_BTDUMP(slot, val) do { if (blockIdx.x == 0 && p.timing) p.timing[(slot)] = (val); } while (0)
 #else
 #define LS_BTWAIT(acc, expr) (expr)
 #define LS_BTDUMP(slot, val) do { } while (0)
@@ -82,8 +84,11 @@ struct BwdCfg {
   static constexpr int SMEM_BYTES = 1024 + A_BYTES + RING * kBwdChunk + 512;
 };
 
+// dK / dV of 128 keys: the 128-wide column tile halves how often the resident operand is
+// re-read from shared memory per column (a 64-wide S/T MMA is bound by that re-read, not by the
+// tensor pipe).  TMEM: ACC [0, D), S [D, D+128), T [D+128, D+256).
 template <int D, int MODE>
-__global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_constant__ BwdParams p) {
+__global__ void __launch_bounds__(kBwdThreads, 1) bwd_kv_kernel(const __grid_constant__ BwdParams p) {
   using C = BwdCfg<D>;
   constexpr bool HAS_T = (MODE != MODE_DV);
   extern __shared__ uint8_t smem_raw[];
@@ -103,44 +108,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr bool kTimedMode = (MODE == MODE_DQ);
-  long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
-  (void)tw0; (void)tw1; (void)tw2; (void)kTimedMode;
-  const long long t_kernel = clock64();
-  (void)t_kernel;
 
-  // ---- work item
-  int part = 0, kvh, h = 0, row0;          // row0: first query (DQ) or first key (DK, DV) of the tile
-  bool is_resp = true;
-  int64_t tokens = 0;
-  int page_off = 0, n_pages = 0, tail_slot = -1;
-  int n_tiles;
-  int tt_min = 0, n_tt = 0;                // DK/DV: first 128-query tile and tiles per head
-  if (MODE == MODE_DQ) {
-    int idx = blockIdx.x;
-    const int qtile = idx % p.nq_tiles;
-    idx /= p.nq_tiles;
-    part = idx % (p.S + 1);
-    kvh = idx / (p.S + 1);
-    h = kvh * p.g + qtile / p.tiles_per_head;
-    row0 = (qtile % p.tiles_per_head) * 128;
-    is_resp = (part == p.S);
-    if (is_resp) {
-      tokens = min(p.R, row0 + 128);
-    } else {
-      tokens = p.shard_tokens[part];
-      page_off = p.shard_page_offset[part];
-      n_pages = p.shard_page_offset[part + 1] - page_off;
-      tail_slot = p.shard_tail_slot[part];
-    }
-    n_tiles = (int)((tokens + 127) / 128);
-  } else {
-    kvh = blockIdx.x / p.tiles_per_head;
-    row0 = (blockIdx.x % p.tiles_per_head) * 128;
-    tt_min = row0 / 128;
-    n_tt = p.tiles_per_head - tt_min;
-    n_tiles = p.g * n_tt;
-  }
+  // ---- work item: 128 keys of one KV head; columns = (head of the group, 128-query tile)
+  const int key_tiles = p.keys_paged ? (p.key_tokens + 127) / 128 : p.tiles_per_head;
+  const int kvh = blockIdx.x / key_tiles;
+  const int row0 = (blockIdx.x % key_tiles) * 128;      // first key of the tile
+  const int tt_min = p.keys_paged ? 0 : row0 / 128;     // response keys are seen by queries t >= j only
+  const int n_tt = p.tiles_per_head - tt_min;
+  const int n_tiles = p.g * n_tt;
+  const int n_keys = p.keys_paged ? p.key_tokens : p.R;
 
   if (threadIdx.x == 0) {
     mbar_init(a_full, 1);
@@ -171,75 +147,54 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     // =========================================================== producer (one thread)
     if (lane == 0 && n_tiles > 0) {
       mbar_arrive_expect_tx(a_full, (HAS_T ? 2 : 1) * C::SLABS * 16384);
-      const int a_head = (MODE == MODE_DQ) ? h : kvh;
-      for (int c = 0; c < C::SLABS; ++c) {
-        tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, a_head, 0);
-        if (HAS_T) tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, a_head, 0);
+      if (!p.keys_paged) {
+        for (int c = 0; c < C::SLABS; ++c) {
+          tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, kvh, 0);
+          if (HAS_T) tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, kvh, 0);
+        }
+      } else {
+        // keys of a suffix block through its pages: one 128-token box, or two 64-token pages
+        const int32_t* pages = p.part_pages + p.key_page_off;
+        const int n_pages = (p.key_tokens + (1 << p.pg_shift) - 1) >> p.pg_shift;
+        const int pg_mask = (1 << p.pg_shift) - 1;
+        const int boxes = p.pg_shift == 6 ? 2 : 1;
+        for (int b = 0; b < boxes; ++b) {
+          const int tok = row0 + b * 64;
+          const int ps = tok >> p.pg_shift;
+          const int page = ps < n_pages ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: zeros
+          for (int c = 0; c < C::SLABS; ++c) {
+            tma_load_5d(a1_smem + c * 16384 + b * 8192, &p.a1_map, a_full, 0, tok & pg_mask, c, kvh, page);
+            if (HAS_T) tma_load_5d(a2_smem + c * 16384 + b * 8192, &p.a2_map, a_full, 0, tok & pg_mask, c, kvh, page);
+          }
+        }
       }
-      const int32_t* pages = p.shard_phys_pages + page_off;
-      const int pg_mask = (1 << p.pg_shift) - 1;
-      const bool dense = (MODE != MODE_DQ) || is_resp;
-      const bool small_pages = !dense && p.pg_shift == 6;   // a 128-key tile spans two 64-token pages
-      auto fetch = [&](int ps) -> int {      // physical page of the shard's page slot (prefix shards only)
-        if (dense) return 0;
-        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
-      };
       uint32_t slot = 0, phase = 0, issued = 0;
       bool ok = true;
       // one chunk: 128 columns x channels [128 c, 128 c + 128) of source `which` (0: B1, 1: B2, 2: B3)
-      auto load = [&](int which, int i, int c, int pa, int pb) {
-        ok = ok && LS_BTWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
+      auto load = [&](int which, int i, int c) {
+        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
         if (ok) {
           mbar_arrive_expect_tx(&full[slot], kBwdChunk);
           uint8_t* dst = ring + slot * kBwdChunk;
-          if (MODE == MODE_DQ) {
-            const int tok = i * 128;
-            if (is_resp) {
-              tma_load_5d(dst, which == 1 ? &p.b2r_map : &p.b1r_map, &full[slot], 0, tok, 2 * c, kvh, 0);
-            } else if (!small_pages) {
-              const bool tail = (tok >> p.pg_shift) == tail_slot;
-              const CUtensorMap* m = which == 1 ? (tail ? &p.bv_tail : &p.bv_map) : (tail ? &p.bk_tail : &p.bk_map);
-              tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 2 * c, kvh, pa);
-            } else {
-              const int sa = tok >> 6;
-              const CUtensorMap* ma = which == 1 ? (sa == tail_slot ? &p.bv_tail : &p.bv_map)
-                                                 : (sa == tail_slot ? &p.bk_tail : &p.bk_map);
-              const CUtensorMap* mb = which == 1 ? (sa + 1 == tail_slot ? &p.bv_tail : &p.bv_map)
-                                                 : (sa + 1 == tail_slot ? &p.bk_tail : &p.bk_map);
-              for (int s = 0; s < 2; ++s) {
-                tma_load_5d(dst + s * 16384, ma, &full[slot], 0, 0, 2 * c + s, kvh, pa);
-                tma_load_5d(dst + s * 16384 + 8192, mb, &full[slot], 0, 0, 2 * c + s, kvh, pb);
-              }
-            }
-          } else {
-            const int hh = kvh * p.g + i / n_tt;
-            const int tq = (tt_min + i % n_tt) * 128;
-            const CUtensorMap* m = which == 0 ? &p.b1r_map : which == 1 ? &p.b2r_map : &p.b3r_map;
-            tma_load_5d(dst, m, &full[slot], 0, tq, 2 * c, hh, 0);
-          }
+          const int hh = kvh * p.g + i / n_tt;
+          const int tq = (tt_min + i % n_tt) * 128;
+          const CUtensorMap* m = which == 0 ? &p.b1r_map : which == 1 ? &p.b2r_map : &p.b3r_map;
+          tma_load_5d(dst, m, &full[slot], 0, tq, 2 * c, hh, 0);
         }
         ++issued;
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
-      auto load_st = [&](int i, int pa, int pb) {
-        for (int c = 0; c < C::NC; ++c) load(0, i, c, pa, pb);
+      auto load_st = [&](int i) {
+        for (int c = 0; c < C::NC; ++c) load(0, i, c);
         if (HAS_T)
-          for (int c = 0; c < C::NC; ++c) load(1, i, c, pa, pb);
+          for (int c = 0; c < C::NC; ++c) load(1, i, c);
       };
       // chunk order = consumption order: ST(0) [M(i) ST(i+1)] ...
-      const int sh = small_pages ? 1 : (p.pg_shift - 7);            // page slot of tile i = (128 i) >> pg_shift
-      auto slot_of = [&](int i) { return small_pages ? 2 * i : (i >> sh); };
-      int pa0 = fetch(slot_of(0)), pb0 = small_pages ? fetch(1) : pa0;         // pages of tile i
-      int pa1 = fetch(slot_of(1)), pb1 = small_pages ? fetch(3) : pa1;         // pages of tile i + 1
-      load_st(0, pa0, pb0);
+      load_st(0);
       for (int i = 0; i < n_tiles; ++i) {
-        const int pa2 = fetch(slot_of(i + 2)), pb2 = small_pages ? fetch(2 * i + 5) : pa2;   // used next round
-        for (int c = 0; c < C::NC; ++c) load(2, i, c, pa0, pb0);
-        if (i + 1 < n_tiles) load_st(i + 1, pa1, pb1);
-        pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
+        for (int c = 0; c < C::NC; ++c) load(2, i, c);
+        if (i + 1 < n_tiles) load_st(i + 1);
       }
-      LS_BTDUMP(0, tw0);
-      LS_BTDUMP(1, clock64() - t_kernel);
       if (*abort_flag) {   // aborted: wait (bounded) for the copies already started
         for (uint32_t s = 0; s < (uint32_t)C::RING && s < issued; ++s) {
           const uint32_t last = ((issued - 1 - s) / C::RING) * C::RING + s;
@@ -270,7 +225,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
           const uint32_t d = op == 0 ? tmem_s : tmem_t;
 #pragma unroll
           for (int c = 0; c < C::NC; ++c) {
-            ok = ok && LS_BTWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
+            ok = ok && mbar_wait(&full[slot], phase, abort_flag);
             if (!ok) return;
             tc_fence_after();
             const uint32_t b_lo = ring_k_lo + slot * (kBwdChunk >> 4);
@@ -298,13 +253,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         }
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-          ok = ok && LS_BTWAIT(tw1, mbar_wait(&e_full[qd], i & 1, abort_flag));
+          ok = ok && mbar_wait(&e_full[qd], i & 1, abort_flag);
           if (!ok) return;
           tc_fence_after();
 #pragma unroll
           for (int c = 0; c < C::NC; ++c) {
             if (qd == 0) {
-              ok = ok && LS_BTWAIT(tw2, mbar_wait(&full[cs[c]], cph[c], abort_flag));
+              ok = ok && mbar_wait(&full[cs[c]], cph[c], abort_flag);
               if (!ok) return;
               tc_fence_after();
             }
@@ -323,10 +278,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
         issue_acc(i);
         if (ok && i + 1 < n_tiles) issue_st(i + 1);
       }
-      LS_BTDUMP(8, tw0);
-      LS_BTDUMP(9, tw1);
-      LS_BTDUMP(10, tw2);
-      LS_BTDUMP(11, clock64() - t_kernel);
     }
   } else {
     // =========================================================== elementwise + epilogue
@@ -335,138 +286,122 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;
-    const int r_idx = row0 + row;                 // query t (DQ) or key j (DK, DV)
+    const int r_idx = row0 + row;                 // key j
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const bool row_ok = r_idx < p.R;
-    float* dq_dst = nullptr;
-    if (MODE == MODE_DQ) dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + h) * D;
-    if (n_tiles == 0) {
-      if (MODE == MODE_DQ && row_ok)
-        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 4)
-          *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-    } else {
-      float lse2_row = 0.f, delta_row = 0.f;
-      int64_t lim = 0;
-      if (MODE == MODE_DQ) {
-        const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + h;
-        lse2_row = p.lse[ri] * kLog2e;
-        delta_row = p.delta[ri];
-        lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
+    const bool row_ok = r_idx < n_keys;
+    bool ok = true;
+    for (int i = 0; i < n_tiles; ++i) {
+      // per-column constants: lane L holds columns L + 32 q of the tile
+      float cl[4] = {0.f, 0.f, 0.f, 0.f}, cd[4] = {0.f, 0.f, 0.f, 0.f};
+      const int hh = kvh * p.g + i / n_tt;
+      const int tq0 = (tt_min + i % n_tt) * 128;
+#pragma unroll
+      for (int qd = 0; qd < 4; ++qd) {
+        const int tc = min(tq0 + 32 * qd + lane, p.R - 1);
+        cl[qd] = __ldg(p.lse + (size_t)tc * p.Hq + hh) * kLog2e;
+        if (MODE == MODE_DK) cd[qd] = __ldg(p.delta + (size_t)tc * p.Hq + hh);
       }
-      bool ok = true;
-      for (int i = 0; i < n_tiles && ok; ++i) {
-        // per-column constants (DK, DV): lane L holds columns L + 32 q of the tile
-        float cl[4] = {0.f, 0.f, 0.f, 0.f}, cd[4] = {0.f, 0.f, 0.f, 0.f};
-        int tq0 = 0;
-        if (MODE != MODE_DQ) {
-          const int hh = kvh * p.g + i / n_tt;
-          tq0 = (tt_min + i % n_tt) * 128;
+      // column t is visible to key row j when j <= t < R (response keys) or t < R (suffix keys)
+      const bool edge = (!p.keys_paged && tq0 < row0 + 127) || (tq0 + 127 >= p.R);
+      const int t_min = p.keys_paged ? 0 : r_idx;
+      // ---- p = exp(s - LSE) for this thread's 4 x 16 columns, as soon as S is complete
+      // (the T MMAs are still running)
+      ok = ok && mbar_wait(s_full, i & 1, abort_flag);
+      tc_fence_after();
+      float pr[64];
 #pragma unroll
-          for (int qd = 0; qd < 4; ++qd) {
-            const int tc = min(tq0 + 32 * qd + lane, p.R - 1);
-            cl[qd] = __ldg(p.lse + (size_t)tc * p.Hq + hh) * kLog2e;
-            if (MODE == MODE_DK) cd[qd] = __ldg(p.delta + (size_t)tc * p.Hq + hh);
+      for (int qd = 0; qd < 4; ++qd) {
+        uint32_t sr[16];
+        tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr);
+        tc_wait_ld16(sr);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float l0 = __shfl_sync(0xffffffffu, cl[qd], 16 * half + j);
+          float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -l0));
+          if (edge) {
+            const int ta = tq0 + 32 * qd + 16 * half + j;
+            if (ta < t_min || ta >= p.R) e = 0.f;
           }
-        }
-        const int key0 = i * 128;
-        const bool edge = (MODE == MODE_DQ) ? __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim)
-                                            : ((tq0 < row0 + 127) || (tq0 + 127 >= p.R));
-        // ---- p = exp(s - LSE) for this thread's 4 x 16 columns, as soon as S is complete
-        // (the T MMAs are still running)
-        ok = LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        float pr[64];
-#pragma unroll
-        for (int qd = 0; qd < 4; ++qd) {
-          uint32_t sr[16];
-          tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr);
-          tc_wait_ld16(sr);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int col = 32 * qd + 16 * half + j;
-            float e;
-            if (MODE == MODE_DQ) {
-              e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
-              if (edge && (int64_t)key0 + col > lim) e = 0.f;
-            } else {
-              const float l0 = __shfl_sync(0xffffffffu, cl[qd], 16 * half + j);
-              e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -l0));
-              if (edge) {                      // column t is visible to key row j when j <= t < R
-                const int ta = tq0 + col;
-                if (ta < r_idx || ta >= p.R) e = 0.f;
-              }
-            }
-            pr[16 * qd + j] = e;
-          }
-        }
-        // E overwrites S columns that the row's other thread reads: all 256 threads must be done
-        // reading S before anyone writes (named barrier 1; the T MMAs normally still run here)
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        // ---- E = p (T - Delta), quarter by quarter, once T is complete
-        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int qd = 0; qd < 4; ++qd) {
-          uint32_t pk[8];
-          if (HAS_T) {
-            uint32_t tr[16];
-            tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr);
-            tc_wait_ld16(tr);
-#pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-              float d0 = delta_row, d1 = delta_row;
-              if (MODE == MODE_DK) {
-                d0 = __shfl_sync(0xffffffffu, cd[qd], 16 * half + j);
-                d1 = __shfl_sync(0xffffffffu, cd[qd], 16 * half + j + 1);
-              }
-              pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[j]) - d0),
-                                     pr[16 * qd + j + 1] * (__uint_as_float(tr[j + 1]) - d1));
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 16; j += 2) pk[j >> 1] = pack_bf16(pr[16 * qd + j], pr[16 * qd + j + 1]);
-          }
-          // quarter q of E (bf16 pairs) lands in columns [16 q, 16 q + 16) of the S region, whose
-          // fp32 contents every thread has already pulled into registers
-          tmem_st8(tmem_s + lane_sel + 16 * qd + 8 * half, pk);
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(&e_full[qd]);
+          pr[16 * qd + j] = e;
         }
       }
-      if (threadIdx.x == 64) {
-        LS_BTDUMP(16, tw0);
-        LS_BTDUMP(18, clock64() - t_kernel);
+      // E overwrites S columns that the row's other thread reads: all 256 threads must be done
+      // reading S before anyone writes (named barrier 1; the T MMAs normally still run here).
+      // The barrier also carries the vote on whether any wait gave up: the threads leave the
+      // loop together or not at all.
+      ok = bar_and(1, 256, ok);
+      if (!ok) break;
+      // ---- E = p (T - Delta), quarter by quarter, once T is complete
+      ok = mbar_wait(t_full, i & 1, abort_flag);     // a failure here is voted on in the next round
+      tc_fence_after();
+#pragma unroll
+      for (int qd = 0; qd < 4; ++qd) {
+        uint32_t pk[8];
+        if (HAS_T) {
+          uint32_t tr[16];
+          tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr);
+          tc_wait_ld16(tr);
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const float d0 = __shfl_sync(0xffffffffu, cd[qd], 16 * half + j);
+            const float d1 = __shfl_sync(0xffffffffu, cd[qd], 16 * half + j + 1);
+            pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[j]) - d0),
+                                   pr[16 * qd + j + 1] * (__uint_as_float(tr[j + 1]) - d1));
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) pk[j >> 1] = pack_bf16(pr[16 * qd + j], pr[16 * qd + j + 1]);
+        }
+        // quarter q of E (bf16 pairs) lands in columns [16 q, 16 q + 16) of the S region, whose
+        // fp32 contents every thread has already pulled into registers
+        tmem_st8(tmem_s + lane_sel + 16 * qd + 8 * half, pk);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(&e_full[qd]);
       }
-      if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        const float out_scale = (MODE == MODE_DK) ? p.scale : 1.0f;
+    }
+    if (n_tiles > 0 && ok) ok = mbar_wait(acc_final, 0, abort_flag);
+    if (n_tiles > 0 && ok) {
+      tc_fence_after();
+      const float out_scale = (MODE == MODE_DK) ? p.scale : 1.0f;
+      // gradient page row of this key: pages are indexed by suffix slot
+      float* grow = nullptr;
+      if (p.grad) {
+        const int pg = 1 << p.pg_shift;
+        const int kk = min(r_idx, n_keys - 1);
+        grow = p.grad + ((((size_t)p.grad_slot0 + (kk >> p.pg_shift)) * pg + (kk & (pg - 1))) * p.Hkv + kvh) * D;
+      }
 #pragma unroll 1
-        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 32) {
-          uint32_t o[32];
-          tmem_ld32(tmem_acc + lane_sel + c, o);
-          tc_wait_ld32(o);
-          if (row_ok) {
-            if (MODE == MODE_DQ) {
+      for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 32) {
+        uint32_t o[32];
+        tmem_ld32(tmem_acc + lane_sel + c, o);
+        tc_wait_ld32(o);
+        if (row_ok) {
+          float v[32];
 #pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dq_dst + c + j) =
-                    make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
-                                __uint_as_float(o[j + 3]));
-            } else {
-              __nv_bfloat16* dst = p.out + ((size_t)r_idx * p.Hkv + kvh) * D + c;
+          for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(o[j]) * out_scale;
+          if (grow) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 v;
-                v.x = pack_bf16(__uint_as_float(o[j]) * out_scale, __uint_as_float(o[j + 1]) * out_scale);
-                v.y = pack_bf16(__uint_as_float(o[j + 2]) * out_scale, __uint_as_float(o[j + 3]) * out_scale);
-                v.z = pack_bf16(__uint_as_float(o[j + 4]) * out_scale, __uint_as_float(o[j + 5]) * out_scale);
-                v.w = pack_bf16(__uint_as_float(o[j + 6]) * out_scale, __uint_as_float(o[j + 7]) * out_scale);
-                *reinterpret_cast<uint4*>(dst + j) = v;
-              }
+            for (int j = 0; j < 32; j += 4) {
+              const float4 gv = *reinterpret_cast<const float4*>(grow + c + j);
+              v[j] += gv.x; v[j + 1] += gv.y; v[j + 2] += gv.z; v[j + 3] += gv.w;
+            }
+          }
+          if (p.keys_paged) {
+            // suffix keys: the sum stays in the fp32 gradient page (this CTA alone owns these rows)
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(grow + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+          } else {
+            __nv_bfloat16* dst = p.out + ((size_t)r_idx * p.Hkv + kvh) * D + c;
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              uint4 w;
+              w.x = pack_bf16(v[j], v[j + 1]);
+              w.y = pack_bf16(v[j + 2], v[j + 3]);
+              w.z = pack_bf16(v[j + 4], v[j + 5]);
+              w.w = pack_bf16(v[j + 6], v[j + 7]);
+              *reinterpret_cast<uint4*>(dst + j) = w;
             }
           }
         }
@@ -481,6 +416,70 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_kernel(const __grid_consta
     tmem_dealloc(tmem_base, 512);
   }
   if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+}
+
+// Row-thread wait of the dQ kernels: returns the warp's common answer.
+__device__ __forceinline__ bool bwd_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
+
+// Work item of the dQ pass: link 0 is the causal response block, links 1.. are the prefix
+// sub-shards and then the suffix blocks; the links of one row tile are summed in that order.
+struct DqItem {
+  int kvh, link, part, pairi;
+  bool is_resp;
+};
+__device__ __forceinline__ DqItem dq_item(const BwdParams& p, int idx, int npairs) {
+  DqItem it;
+  it.pairi = idx % npairs;
+  idx /= npairs;
+  it.link = idx % (p.parts + 1);
+  it.kvh = idx / (p.parts + 1);
+  it.is_resp = it.link == 0;
+  it.part = it.is_resp ? p.parts : it.link - 1;
+  return it;
+}
+
+// One row thread's share of the dQ epilogue: NCOL accumulator columns of its row are added
+// to the running fp32 sum (fold), stored as the first term, or -- last link -- scaled and
+// written as bf16.  An empty part in the middle of a chain leaves the sum untouched.
+template <int NCOL>
+__device__ __forceinline__ void dq_store_row(uint32_t tmem_row, bool have_acc, bool fold, bool last, float scale,
+                                             float* acc_dst, __nv_bfloat16* dq_dst, bool row_ok) {
+  if (!have_acc && fold && !last) return;
+#pragma unroll 1
+  for (int c = 0; c < NCOL; c += 32) {
+    uint32_t o[32];
+    if (have_acc) {
+      tmem_ld32(tmem_row + c, o);
+      tc_wait_ld32(o);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[j] = 0u;
+    }
+    if (row_ok) {
+      float4 run[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        run[j] = fold ? __ldcg(reinterpret_cast<const float4*>(acc_dst + c) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float4 v;
+        v.x = run[j].x + __uint_as_float(o[4 * j]);
+        v.y = run[j].y + __uint_as_float(o[4 * j + 1]);
+        v.z = run[j].z + __uint_as_float(o[4 * j + 2]);
+        v.w = run[j].w + __uint_as_float(o[4 * j + 3]);
+        if (last) {
+          uint2 pk;
+          pk.x = pack_bf16(v.x * scale, v.y * scale);
+          pk.y = pack_bf16(v.z * scale, v.w * scale);
+          *(reinterpret_cast<uint2*>(dq_dst + c) + j) = pk;
+        } else {
+          *(reinterpret_cast<float4*>(acc_dst + c) + j) = v;
+        }
+      }
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------
@@ -521,47 +520,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   uint64_t* acc_final = e_full + 4;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* work_idx = const_cast<int*>(abort_flag) + 1;   // (even CTA) the pair's work item
 
-  constexpr bool kTimedMode = true;
   long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
-  (void)tw0; (void)tw1; (void)tw2; (void)kTimedMode;
+  (void)tw0; (void)tw1; (void)tw2;
   const long long t_kernel0 = clock64();
   (void)t_kernel0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
-
-  // ---- work item of the pair, and this CTA's Q tile
-  const int npairs = (p.nq_tiles + 1) / 2;
-  int idx = blockIdx.x >> 1;
-  const int pairi = idx % npairs;
-  idx /= npairs;
-  const int part = idx % (p.S + 1);
-  const int kvh = idx / (p.S + 1);
-  const bool is_resp = (part == p.S);
-  auto tile_of = [&](int qt, int& hh, int& r0) {
-    if (qt < p.nq_tiles) {
-      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
-      r0 = (qt % p.tiles_per_head) * 128;
-    } else {                                 // odd tile count: the pair's second CTA works on zero rows
-      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
-      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
-    }
-  };
-  int h, row0, h_o, row0_o;
-  tile_of(2 * pairi + (int)rank, h, row0);
-  tile_of(2 * pairi + 1 - (int)rank, h_o, row0_o);
-  int64_t tokens;
-  int page_off = 0, n_pages = 0, tail_slot = -1;
-  if (is_resp) {
-    tokens = min(p.R, max(row0, row0_o) + 128);      // both CTAs walk the longer causal range
-  } else {
-    tokens = p.shard_tokens[part];
-    page_off = p.shard_page_offset[part];
-    n_pages = p.shard_page_offset[part + 1] - page_off;
-    tail_slot = p.shard_tail_slot[part];
-  }
-  const int n_tiles = (int)((tokens + 127) / 128);
 
   if (threadIdx.x == 0) {
     mbar_init(a_full, 1);
@@ -574,6 +541,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
     for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 16);
     mbar_init(acc_final, 1);
     *abort_flag = 0;
+    // work items are handed out in launch order of the pairs that ask (see chain_wait)
+    if (leader) *work_idx = atomicAdd(p.ctl, 1);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -589,6 +558,36 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   const uint32_t tmem_s = tmem_base + D;
   const uint32_t tmem_t = tmem_base + D + 128;
 
+  // ---- work item of the pair, and this CTA's Q tile
+  const int npairs = (p.nq_tiles + 1) / 2;
+  const DqItem it = dq_item(p, (int)ld_shared_cluster_u32(mapa_u32(smem_u32(work_idx), 0)), npairs);
+  const int pairi = it.pairi, part = it.part, kvh = it.kvh;
+  const bool is_resp = it.is_resp;
+  auto tile_of = [&](int qt, int& hh, int& r0) {
+    if (qt < p.nq_tiles) {
+      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      r0 = (qt % p.tiles_per_head) * 128;
+    } else {                                 // odd tile count: the pair's second CTA works on zero rows
+      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
+    }
+  };
+  const int qtile = 2 * pairi + (int)rank;
+  int h, row0, h_o, row0_o;
+  tile_of(qtile, h, row0);
+  tile_of(2 * pairi + 1 - (int)rank, h_o, row0_o);
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, max(row0, row0_o) + 128);      // both CTAs walk the longer causal range
+  } else {
+    tokens = p.part_tokens[part];
+    page_off = p.part_page_offset[part];
+    n_pages = p.part_page_offset[part + 1] - page_off;
+    tail_slot = p.part_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 127) / 128);
+
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
@@ -598,7 +597,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
         tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
         tma_load_5d_pair(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, h, 0);
       }
-      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
       const bool small_pages = !is_resp && p.pg_shift == 6;
       auto fetch = [&](int ps) -> int {
@@ -771,26 +770,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
     const int r_idx = p.packed ? row0 + row % p.R : row0 + row;
     const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const bool row_ok = r_idx < p.R && (!p.packed || row < p.g * p.R);
-    float* dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + hr) * D;
-    if (n_tiles == 0) {
-      if (row_ok)
-        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 4)
-          *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-    } else {
-      const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
+    const bool tile_ok = qtile < p.nq_tiles;
+    const bool row_ok = tile_ok && r_idx < p.R && (!p.packed || row < p.g * p.R);
+    const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
+    bool ok = true;
+    if (n_tiles > 0) {
       const float lse2_row = p.lse[ri] * kLog2e;
       const float delta_row = p.delta[ri];
       const int64_t lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
       uint32_t e_remote[4];
 #pragma unroll
       for (int qd = 0; qd < 4; ++qd) e_remote[qd] = mapa_u32(smem_u32(&e_full[qd]), 0);
-      bool ok = true;
-      for (int i = 0; i < n_tiles && ok; ++i) {
+      for (int i = 0; i < n_tiles; ++i) {
         const int key0 = i * 128;
         const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim);
-        ok = LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
-        if (!ok) break;
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
         tc_fence_after();
         float pr[64];
 #pragma unroll
@@ -805,9 +799,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
             pr[16 * qd + j] = e;
           }
         }
-        asm volatile("bar.sync 1, 256;" ::: "memory");   // all S reads of this CTA done before any E write
-        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
+        // all S reads of this CTA done before any E write; the barrier also carries the vote on
+        // whether any wait gave up, so the row threads leave the loop together or not at all
+        ok = bar_and(1, 256, ok);
         if (!ok) break;
+        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));   // a failure here is voted on in the next round
         tc_fence_after();
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
@@ -830,23 +826,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
         LS_BTDUMP(17, tw1);
         LS_BTDUMP(18, clock64() - t_kernel0);
       }
-      if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-#pragma unroll 1
-        for (int c = half * (D / 2); c < (half + 1) * (D / 2); c += 32) {
-          uint32_t o[32];
-          tmem_ld32(tmem_acc + lane_sel + c, o);
-          tc_wait_ld32(o);
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(dq_dst + c + j) =
-                  make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
-                              __uint_as_float(o[j + 3]));
-          }
-        }
-      }
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) ok = bwd_wait_warp(acc_final, 0, abort_flag);
+      if (ok) tc_fence_after();
+    }
+    // ---- epilogue: add this part's sum to the running dQ of the row tile, in link order
+    const bool fold = it.link > 0, last = it.link == p.parts;
+    int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + min(qtile, p.nq_tiles - 1);
+    if (tile_ok) {
+      if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
+      if (ok)
+        dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, fold, last, p.scale,
+                            p.dq_acc + ri * D + half * (D / 2), p.dq + ri * D + half * (D / 2), row_ok);
+      const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
+      if (row == 0 && half == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
 
@@ -857,7 +850,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
   }
-  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+    st_relaxed_gpu(p.ctl + 1, 1);    // ends every other chain wait of this launch
+  }
 }
 
 // Delta[t,h] = sum_d dO[t,h,d] * O[t,h,d], one warp per row.
@@ -901,19 +897,15 @@ __global__ void dq_reduce_kernel(const float* __restrict__ dq_part, int parts, i
 }
 
 template <int D, int MODE>
-static ls_status_t launch_bwd(const BwdParams& prm, int grid, cudaStream_t st) {
+static ls_status_t launch_kv(const BwdParams& prm, int grid, cudaStream_t st, bool timed) {
   using C = BwdCfg<D>;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(bwd_kernel<D, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
-        cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
-  constexpr int which = MODE == MODE_DQ ? LS_KERNEL_BWD_DQ : MODE == MODE_DK ? LS_KERNEL_BWD_DK : LS_KERNEL_BWD_DV;
-  profile_begin(which, st);
-  bwd_kernel<D, MODE><<<grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
-  profile_end(which, st);
+  static bool configured[64] = {};
+  const ls_status_t cs = configure_smem(bwd_kv_kernel<D, MODE>, C::SMEM_BYTES, configured);
+  if (cs != LS_OK) return cs;
+  constexpr int which = MODE == MODE_DK ? LS_KERNEL_BWD_DK : LS_KERNEL_BWD_DV;
+  if (timed) profile_begin(which, st);
+  bwd_kv_kernel<D, MODE><<<grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
+  if (timed) profile_end(which, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
@@ -956,46 +948,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   uint64_t* acc_final = e_full + 4;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* work_idx = const_cast<int*>(abort_flag) + 1;   // (even CTA) the pair's work item
 
-  constexpr bool kTimedMode = true;
   long long tw0 = 0, tw1 = 0, tw2 = 0;
-  (void)tw0; (void)tw1; (void)tw2; (void)kTimedMode;
+  (void)tw0; (void)tw1; (void)tw2;
   const long long t_kernel0 = clock64();
   (void)t_kernel0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
-
-  const int npairs = (p.nq_tiles + 1) / 2;
-  int idx = blockIdx.x >> 1;
-  const int pairi = idx % npairs;
-  idx /= npairs;
-  const int part = idx % (p.S + 1);
-  const int kvh = idx / (p.S + 1);
-  const bool is_resp = (part == p.S);
-  auto tile_of = [&](int qt, int& hh, int& r0) {
-    if (qt < p.nq_tiles) {
-      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
-      r0 = (qt % p.tiles_per_head) * 128;
-    } else {
-      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
-      r0 = p.tiles_per_head * 128;
-    }
-  };
-  int h, row0, h_o, row0_o;
-  tile_of(2 * pairi + (int)rank, h, row0);
-  tile_of(2 * pairi + 1 - (int)rank, h_o, row0_o);
-  int64_t tokens;
-  int page_off = 0, n_pages = 0, tail_slot = -1;
-  if (is_resp) {
-    tokens = min(p.R, max(row0, row0_o) + 128);
-  } else {
-    tokens = p.shard_tokens[part];
-    page_off = p.shard_page_offset[part];
-    n_pages = p.shard_page_offset[part + 1] - page_off;
-    tail_slot = p.shard_tail_slot[part];
-  }
-  const int n_tiles = (int)((tokens + 255) / 256);
 
   if (threadIdx.x == 0) {
     mbar_init(a_full, 1);
@@ -1009,6 +970,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
     for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 16);
     mbar_init(acc_final, 1);
     *abort_flag = 0;
+    // work items are handed out in launch order of the pairs that ask (see chain_wait)
+    if (leader) *work_idx = atomicAdd(p.ctl, 1);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -1023,6 +986,35 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   const uint32_t tmem_acc = tmem_base;
   const uint32_t tmem_st = tmem_base + D;      // S, then T, then E (bf16) over its first 128 columns
 
+  const int npairs = (p.nq_tiles + 1) / 2;
+  const DqItem it = dq_item(p, (int)ld_shared_cluster_u32(mapa_u32(smem_u32(work_idx), 0)), npairs);
+  const int pairi = it.pairi, part = it.part, kvh = it.kvh;
+  const bool is_resp = it.is_resp;
+  auto tile_of = [&](int qt, int& hh, int& r0) {
+    if (qt < p.nq_tiles) {
+      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      r0 = (qt % p.tiles_per_head) * 128;
+    } else {
+      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      r0 = p.tiles_per_head * 128;
+    }
+  };
+  const int qtile = 2 * pairi + (int)rank;
+  int h, row0, h_o, row0_o;
+  tile_of(qtile, h, row0);
+  tile_of(2 * pairi + 1 - (int)rank, h_o, row0_o);
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, max(row0, row0_o) + 128);
+  } else {
+    tokens = p.part_tokens[part];
+    page_off = p.part_page_offset[part];
+    n_pages = p.part_page_offset[part + 1] - page_off;
+    tail_slot = p.part_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 255) / 256);
+
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
@@ -1032,7 +1024,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
         tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
         tma_load_5d_pair(a2_smem + c * 16384, &p.a2_map, a_full, 0, row0, c, h, 0);
       }
-      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
       const bool small_pages = !is_resp && p.pg_shift == 6;
       auto page_at = [&](int tok) -> int {       // physical page holding key `tok` of this partial
@@ -1179,14 +1171,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
     const int r_idx = p.packed ? row0 + row % p.R : row0 + row;
     const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const bool row_ok = r_idx < p.R && (!p.packed || row < p.g * p.R);
-    float* dq_dst = p.dq_part + (((size_t)part * p.R + min(r_idx, p.R - 1)) * p.Hq + hr) * D;
-    if (n_tiles == 0) {
-      if (row_ok)
-        for (int c = sub * (D / 2); c < (sub + 1) * (D / 2); c += 4)
-          *reinterpret_cast<float4*>(dq_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-    } else {
-      const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
+    const bool tile_ok = qtile < p.nq_tiles;
+    const bool row_ok = tile_ok && r_idx < p.R && (!p.packed || row < p.g * p.R);
+    const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
+    bool ok = true;
+    if (n_tiles > 0) {
       const float lse2_row = p.lse[ri] * kLog2e;
       const float delta_row = p.delta[ri];
       const int64_t lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
@@ -1194,12 +1183,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
       uint32_t e_remote[4];
 #pragma unroll
       for (int qd = 0; qd < 4; ++qd) e_remote[qd] = mapa_u32(smem_u32(&e_full[qd]), 0);
-      bool ok = true;
-      for (int i = 0; i < n_tiles && ok; ++i) {
+      for (int i = 0; i < n_tiles; ++i) {
         const int key0 = i * 256;
         const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 255 > lim);
-        ok = LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
-        if (!ok) break;
+        // No thread leaves this loop on its own: a wait that gave up is remembered in `ok` and put
+        // to the vote at the first named barrier of the tile, where all 256 leave together.
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
         tc_fence_after();
         // p = exp(s - LSE) for this thread's 4 x 32 columns: all four TMEM loads in flight at once,
         // p kept as packed bf16 pairs (64 registers) until T is ready
@@ -1223,8 +1212,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
           }
           pp[j >> 1] = pack_bf16(e0, e1);
         }
-        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
-        if (!ok) break;
+        ok = ok && LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
         tc_fence_after();
         uint32_t tr[2][32];
         tmem_ld32(tmem_st + lane_sel + 32 * sub, tr[0]);
@@ -1241,36 +1229,38 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
           }
           // E (bf16 pairs) of quarter q goes to columns [32 q, 32 q + 32) of the buffer: T columns that
           // this quarter or an earlier one has read -- by either thread of the row, hence the barrier
-          asm volatile("bar.sync 1, 256;" ::: "memory");
+          if (qd == 0) {
+            ok = bar_and(1, 256, ok);
+            if (!ok) break;
+          } else {
+            bar_sync(1, 256);
+          }
           tmem_st16(tmem_st + lane_sel + 32 * qd + 16 * sub, pk);
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(e_remote[qd]);
         }
+        if (!ok) break;          // (uniform: decided by the vote above)
       }
       if (threadIdx.x == 64) {
         LS_BTDUMP(16, tw0);
         LS_BTDUMP(17, tw1);
         LS_BTDUMP(18, clock64() - t_kernel0);
       }
-      if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-#pragma unroll 1
-        for (int c = sub * (D / 2); c < (sub + 1) * (D / 2); c += 32) {
-          uint32_t o[32];
-          tmem_ld32(tmem_acc + lane_sel + c, o);
-          tc_wait_ld32(o);
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(dq_dst + c + j) =
-                  make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
-                              __uint_as_float(o[j + 3]));
-          }
-        }
-      }
+      if (ok) ok = bwd_wait_warp(acc_final, 0, abort_flag);
+      if (ok) tc_fence_after();
+    }
+    // ---- epilogue: add this part's sum to the running dQ of the row tile, in link order
+    const bool fold = it.link > 0, last = it.link == p.parts;
+    int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + min(qtile, p.nq_tiles - 1);
+    if (tile_ok) {
+      if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
+      if (ok)
+        dq_store_row<D / 2>(tmem_acc + lane_sel + sub * (D / 2), n_tiles > 0, fold, last, p.scale,
+                            p.dq_acc + ri * D + sub * (D / 2), p.dq + ri * D + sub * (D / 2), row_ok);
+      const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
+      if (row == 0 && sub == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
 
@@ -1281,18 +1271,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
   }
-  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+    st_relaxed_gpu(p.ctl + 1, 1);    // ends every other chain wait of this launch
+  }
 }
 
 static ls_status_t launch_dq3(const BwdParams& prm, int64_t grid, cudaStream_t st) {
-  static bool configured = false;
+  static bool configured[64] = {};
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  if (!configured) {
-    if (cudaFuncSetAttribute(bwd_dq3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Dq3Cfg::SMEM_BYTES) !=
-        cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
+  const ls_status_t cs = configure_smem(bwd_dq3_kernel, Dq3Cfg::SMEM_BYTES, configured);
+  if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_BWD_DQ, st);
   bwd_dq3_kernel<<<(int)grid, kDq3Threads, Dq3Cfg::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_BWD_DQ, st);
@@ -1302,14 +1291,10 @@ static ls_status_t launch_dq3(const BwdParams& prm, int64_t grid, cudaStream_t s
 template <int D>
 static ls_status_t launch_dq2(const BwdParams& prm, int64_t grid, cudaStream_t st) {
   using C = Dq2Cfg<D>;
-  static bool configured = false;
+  static bool configured[64] = {};
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  if (!configured) {
-    if (cudaFuncSetAttribute(bwd_dq2_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
-        cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
+  const ls_status_t cs = configure_smem(bwd_dq2_kernel<D>, C::SMEM_BYTES, configured);
+  if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_BWD_DQ, st);
   bwd_dq2_kernel<D><<<(int)grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_BWD_DQ, st);
@@ -1323,40 +1308,46 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
                                           const float* lse, const void* d_o, void* dq, void* dk_resp,
                                           void* dv_resp, void* workspace, size_t workspace_bytes,
                                           int32_t* status_dev, void* stream) {
-  if (!h || !prm || !q || !k_resp || !v_resp || !o_f32 || !lse || !d_o || !dq || !dk_resp || !dv_resp)
-    return LS_ERR_INVALID_ARG;
-  if (!h->on_device) return LS_ERR_INVALID_ARG;
+  ls_status_t st = ls::check_handle(h, prm);
+  if (st != LS_OK) return st;
+  if (!q || !k_resp || !v_resp || !o_f32 || !lse || !d_o || !dq || !dk_resp || !dv_resp) return LS_ERR_INVALID_ARG;
   const ls_pages_desc_t& d = h->desc;
   if (prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % d.num_kv_heads != 0) return LS_ERR_INVALID_ARG;
   if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;
   const bool mla = d.dim_k == 576 && d.dim_v == 512;
-  if (!((d.dim_k == 128 && d.dim_v == 128) || (d.dim_k == 256 && d.dim_v == 256) || mla))
-    return LS_ERR_UNSUPPORTED_SHAPE;
   const void* ptrs[] = {q, k_resp, v_resp, o_f32, d_o, dq, dk_resp, dv_resp, workspace};
   for (const void* ptr : ptrs)
     if (!ls::aligned16(ptr)) return LS_ERR_ALIGNMENT;
   const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_BWD);
   if (!workspace || workspace_bytes < need) return LS_ERR_WORKSPACE;
+  const bool add_grad = (prm->flags & LS_FLAG_ADD_SUFFIX_GRAD) != 0;
+  if ((add_grad || !h->suffix_blocks.empty()) && (mla || !h->dk_grad)) return LS_ERR_INVALID_ARG;
 
   const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads, D = d.dim_k;
+  const int g = Hq / Hkv;
+  const int tiles_per_head = (R + 127) / 128;
   const int64_t rows = (int64_t)R * Hq;
-  float* dq_part = static_cast<float*>(workspace);
-  const int parts = d.num_shards * h->fine;        // sub-shards; the kernels see `parts` prefix partials
-  const bool mla_fast = mla && ls::mla_dq_fast(h);
-  float* delta = dq_part + (size_t)(mla_fast ? 1 : parts + 1) * rows * D;
+  // workspace: Delta | hand-over control words | fp32 running dQ (one per partial for the generic 576/512 path)
+  float* delta = static_cast<float*>(workspace);
+  const size_t delta_bytes = ((size_t)rows * sizeof(float) + 15) & ~(size_t)15;
+  int* ctl = reinterpret_cast<int*>(static_cast<char*>(workspace) + delta_bytes);
+  const size_t ctl_bytes = ((size_t)(ls::kChainHeaderInts + (int64_t)Hkv * g * tiles_per_head) * sizeof(int) + 15) & ~(size_t)15;
+  float* dq_acc = reinterpret_cast<float*>(reinterpret_cast<char*>(ctl) + ctl_bytes);
+  const int parts = h->num_parts();
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
   ls::delta_kernel<<<(int)((rows + 7) / 8), 256, 0, cs>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows,
                                                         d.dim_v, delta);
 
   if (mla) {
+    const bool mla_fast = ls::mla_dq_fast(h);
     ls_status_t ms =
-        ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_part, dk_resp, dv_resp, mla_fast, status_dev, cs);
+        ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_acc, dk_resp, dv_resp, mla_fast, status_dev, cs);
     if (ms != LS_OK) return ms;
-    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_part, dq, status_dev, cs);
+    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_acc, dq, status_dev, cs);
     const int64_t n4m = rows * D / 4;
     ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4m + 255) / 256, 148 * 16), 256, 0, cs>>>(
-        dq_part, parts + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));
+        dq_acc, parts + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));
     return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
   }
 
@@ -1364,102 +1355,116 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     return ls::encode_map5(m, base, D, R, heads, 1, (int64_t)heads * D, D, (int64_t)R * heads * D, box_tok, groups);
   };
   const bool small_pages = d.page_size == 64;
-  const int pbox = small_pages ? 64 : 128, pgroups = small_pages ? 1 : 2;   // pool boxes
+  const int mbox = small_pages ? 64 : 128;
   ls::BwdParams P;
-  P.shard_phys_pages = h->d_shard_phys_pages;
-  P.shard_page_offset = h->d_shard_page_offset;
-  P.shard_tail_slot = h->d_shard_tail_slot;
-  P.shard_tokens = h->d_shard_tokens;
+  P.part_pages = h->d_part_pages;
+  P.part_page_offset = h->d_part_page_offset;
+  P.part_tail_slot = h->d_part_tail_slot;
+  P.part_tokens = h->d_part_tokens;
   P.lse = lse;
   P.delta = delta;
-  P.dq_part = dq_part;
+  P.dq_acc = dq_acc;
+  P.dq = static_cast<__nv_bfloat16*>(dq);
+  P.ctl = ctl;
   P.out = nullptr;
+  P.grad = nullptr;
   P.status = status_dev;
+  P.timing = ls::g_timing_buffer;
   P.R = R;
   P.Hq = Hq;
   P.Hkv = Hkv;
-  P.g = Hq / Hkv;
-  P.S = parts;
-  P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
-  P.tiles_per_head = (R + 127) / 128;
-  P.nq_tiles = P.g * P.tiles_per_head;
+  P.g = g;
+  P.parts = parts;
+  P.pg_shift = ls::pg_shift_of(d.page_size);
+  P.tiles_per_head = tiles_per_head;
+  P.nq_tiles = g * tiles_per_head;
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
+  P.keys_paged = P.key_page_off = P.key_tokens = P.grad_slot0 = 0;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * ls::kLog2e;
 
-  // ---- dQ: rows = queries, columns = keys of every partial
-  ls_status_t st = dense_map(&P.a1_map, q, Hq, 128, 1);
-  if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128, 1);
-  if (st == LS_OK) st = dense_map(&P.b1r_map, k_resp, Hkv, 128, 2);
-  if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 128, 2);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_map, h, 0, pbox, pgroups, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bk_tail, h, 0, pbox, pgroups, true);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_map, h, 1, pbox, pgroups, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.bv_tail, h, 1, pbox, pgroups, true);
-  if (st != LS_OK) return st;
-  P.b3r_map = P.b1r_map;
-  const int64_t grid_dq = (int64_t)Hkv * (parts + 1) * P.nq_tiles;
-  if (grid_dq > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  const char* pair_env = getenv("LS_BWD_PAIR");
-  const bool use_pairs = !(pair_env && pair_env[0] == '0');
+  // ---- dQ: rows = queries, columns = keys of every part, summed through the running dQ
   P.packed = 0;
-  if (use_pairs) {
-    const int g = Hq / Hkv;
-    if (g > 1 && g * R <= 128) {           // short response: all rows of a KV group in one Q tile
-      P.packed = 1;
-      P.nq_tiles = 1;
-      st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, R, g);
-      if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, R, g);
-      if (st != LS_OK) return st;
-    }
-    const int mbox = small_pages ? 64 : 128;
-    st = dense_map(&P.rk_s, k_resp, Hkv, 64, 2);
-    if (st == LS_OK) st = dense_map(&P.rv_s, v_resp, Hkv, 64, 2);
-    if (st == LS_OK) st = dense_map(&P.rk_m, k_resp, Hkv, 128, 1);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_s, h, 0, 64, 2, false);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_s_tail, h, 0, 64, 2, true);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_s, h, 1, 64, 2, false);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_s_tail, h, 1, 64, 2, true);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m, h, 0, mbox, 1, false);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk_m_tail, h, 0, mbox, 1, true);
-    if (st != LS_OK) return st;
-    if (st == LS_OK) st = dense_map(&P.rv_m, v_resp, Hkv, 128, 1);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_m, h, 1, mbox, 1, false);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv_m_tail, h, 1, mbox, 1, true);
-    if (st != LS_OK) return st;
-    const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
-    const bool wide = D == 256 && !(pair_env && pair_env[0] == '2');     // LS_BWD_PAIR=2: 128-key pair kernel
-    st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : wide ? ls::launch_dq3(P, grid2, cs) : ls::launch_dq2<256>(P, grid2, cs);
+  if (g > 1 && g * R <= 128) {           // short response: all rows of a KV group in one Q tile
+    P.packed = 1;
+    P.nq_tiles = 1;
+    st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, R, g);
+    if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, R, g);
   } else {
-    st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DQ>(P, (int)grid_dq, cs)
-                    : ls::launch_bwd<256, ls::MODE_DQ>(P, (int)grid_dq, cs);
+    st = dense_map(&P.a1_map, q, Hq, 128, 1);
+    if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128, 1);
   }
+  if (st == LS_OK) st = dense_map(&P.rk_s, k_resp, Hkv, 64, 2);
+  if (st == LS_OK) st = dense_map(&P.rv_s, v_resp, Hkv, 64, 2);
+  if (st == LS_OK) st = dense_map(&P.rk_m, k_resp, Hkv, 128, 1);
+  if (st == LS_OK) st = dense_map(&P.rv_m, v_resp, Hkv, 128, 1);
+  if (st == LS_OK) st = ls::pool_map(&P.pk_s, h, 0, 64, 2, false);
+  if (st == LS_OK) st = ls::pool_map(&P.pk_s_tail, h, 0, 64, 2, true);
+  if (st == LS_OK) st = ls::pool_map(&P.pv_s, h, 1, 64, 2, false);
+  if (st == LS_OK) st = ls::pool_map(&P.pv_s_tail, h, 1, 64, 2, true);
+  if (st == LS_OK) st = ls::pool_map(&P.pk_m, h, 0, mbox, 1, false);
+  if (st == LS_OK) st = ls::pool_map(&P.pk_m_tail, h, 0, mbox, 1, true);
+  if (st == LS_OK) st = ls::pool_map(&P.pv_m, h, 1, mbox, 1, false);
+  if (st == LS_OK) st = ls::pool_map(&P.pv_m_tail, h, 1, mbox, 1, true);
   if (st != LS_OK) return st;
-  const int64_t n4 = rows * D / 4;
-  ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 16), 256, 0, cs>>>(
-      dq_part, parts + 1, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
+  if (cudaMemsetAsync(ctl, 0, ctl_bytes, cs) != cudaSuccess) return LS_ERR_CUDA;
+  const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
+  st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq3(P, grid2, cs);
+  if (st != LS_OK) return st;
 
-  // ---- dK and dV of the response keys: rows = keys, columns = queries of the KV group
-  const int grid_kv = Hkv * P.tiles_per_head;
+  // ---- dK and dV: rows = keys, columns = queries of the KV group
+  st = dense_map(&P.b1r_map, q, Hq, 128, 2);
+  if (st == LS_OK) st = dense_map(&P.b2r_map, d_o, Hq, 128, 2);
+  if (st != LS_OK) return st;
+  const int pg = d.page_size;
+  // keys of every suffix block, read through their pages: the sums go into the block's fp32 gradient pages
+  for (size_t b = 0; b < h->suffix_blocks.size(); ++b) {
+    const ls::SuffixBlock& blk = h->suffix_blocks[b];
+    P.keys_paged = 1;
+    P.key_page_off = (int)(h->num_logical_pages + blk.first_slot);
+    P.key_tokens = blk.tokens;
+    P.grad_slot0 = blk.first_slot;
+    const int grid_b = Hkv * ((blk.tokens + 127) / 128);
+    st = ls::pool_map(&P.a1_map, h, 0, mbox, 1, false);
+    if (st == LS_OK) st = ls::pool_map(&P.a2_map, h, 1, mbox, 1, false);
+    if (st != LS_OK) return st;
+    P.b3r_map = P.b1r_map;
+    P.grad = h->dk_grad;
+    st = (D == 128) ? ls::launch_kv<128, ls::MODE_DK>(P, grid_b, cs, false)
+                    : ls::launch_kv<256, ls::MODE_DK>(P, grid_b, cs, false);
+    if (st != LS_OK) return st;
+    P.b3r_map = P.b2r_map;
+    P.grad = h->dv_grad;
+    st = (D == 128) ? ls::launch_kv<128, ls::MODE_DV>(P, grid_b, cs, false)
+                    : ls::launch_kv<256, ls::MODE_DV>(P, grid_b, cs, false);
+    if (st != LS_OK) return st;
+  }
+  // keys of the response block itself (causal); with LS_FLAG_ADD_SUFFIX_GRAD the gradient pages that later
+  // blocks left for this block (its slots start where the suffix now ends) are added
+  P.keys_paged = 0;
+  P.key_tokens = R;
+  P.grad_slot0 = (int)h->suffix_phys.size();
+  if (add_grad && P.grad_slot0 + (R + pg - 1) / pg > h->suffix_cap_pages) return LS_ERR_INVALID_ARG;
+  const int grid_kv = Hkv * tiles_per_head;
   st = dense_map(&P.a1_map, k_resp, Hkv, 128, 1);
   if (st == LS_OK) st = dense_map(&P.a2_map, v_resp, Hkv, 128, 1);
-  if (st == LS_OK) st = dense_map(&P.b1r_map, q, Hq, 128, 2);
-  if (st == LS_OK) st = dense_map(&P.b2r_map, d_o, Hq, 128, 2);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
   P.out = static_cast<__nv_bfloat16*>(dk_resp);
-  st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DK>(P, grid_kv, cs) : ls::launch_bwd<256, ls::MODE_DK>(P, grid_kv, cs);
+  P.grad = add_grad ? h->dk_grad : nullptr;
+  st = (D == 128) ? ls::launch_kv<128, ls::MODE_DK>(P, grid_kv, cs, true) : ls::launch_kv<256, ls::MODE_DK>(P, grid_kv, cs, true);
   if (st != LS_OK) return st;
   P.b3r_map = P.b2r_map;
   P.out = static_cast<__nv_bfloat16*>(dv_resp);
-  st = (D == 128) ? ls::launch_bwd<128, ls::MODE_DV>(P, grid_kv, cs) : ls::launch_bwd<256, ls::MODE_DV>(P, grid_kv, cs);
+  P.grad = add_grad ? h->dv_grad : nullptr;
+  st = (D == 128) ? ls::launch_kv<128, ls::MODE_DV>(P, grid_kv, cs, true) : ls::launch_kv<256, ls::MODE_DV>(P, grid_kv, cs, true);
   if (st != LS_OK) return st;
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------------
-// Backward without caller scratch: the per-partial dQ sums and Delta live in a fixed
-// array inside the library's device image instead of a caller-provided workspace.
+// Backward without caller scratch: Delta, the hand-over counters and the running dQ live in a
+// fixed array inside the library's device image instead of a caller-provided workspace.
 // ---------------------------------------------------------------------------------
 namespace ls {
 
@@ -1494,16 +1499,18 @@ extern "C" ls_status_t ls_replay_attn_bwd_static(const ls_pages_t* h, const ls_a
                                                  const void* k_resp, const void* v_resp, const float* o_f32,
                                                  const float* lse, const void* d_o, void* dq, void* dk_resp,
                                                  void* dv_resp, int32_t* status_dev, void* stream) {
-  if (!h || !prm) return LS_ERR_INVALID_ARG;
+  // the handle must belong to the current device: the scratch address is looked up per device
+  ls_status_t st = ls::check_handle(h, prm);
+  if (st != LS_OK) return st;
   const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_BWD);
   if (need == 0) return LS_ERR_INVALID_ARG;
   if (need > ls::kStaticScratchBytes) return LS_ERR_WORKSPACE;   // shape too large for the built-in scratch
   void* scratch = nullptr;
-  ls_status_t st = ls::static_scratch(&scratch);
+  st = ls::static_scratch(&scratch);
   if (st != LS_OK) return st;
-  // Nothing in the scratch has to start at zero: the dQ pass writes every partial of every
-  // row (zeros for an empty partial) and the Delta kernel writes every row before either
-  // is read, so the previous call's leftovers are never observed.
+  // The array keeps the previous call's contents.  The only words that must start at zero are
+  // the hand-over counters, which the backward clears itself (a memset node on `stream`, no
+  // allocation); Delta and the running dQ are written before they are read.
   return ls_replay_attn_bwd(h, prm, q, k_resp, v_resp, o_f32, lse, d_o, dq, dk_resp, dv_resp, scratch,
                             ls::kStaticScratchBytes, status_dev, stream);
 }

@@ -19,6 +19,8 @@
 // TMEM columns: ACC [0, 64 NACC), then two buffers of (S 64 | T 64) from column 256.
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "ls_internal.h"
 #include "ls_sm100.cuh"
 
@@ -40,7 +42,7 @@ struct MlaBwdParams {
   float* dq_part;          // [(S+1), R, Hq, 576] fp32, unscaled
   __nv_bfloat16* out;      // dk_resp [R, Hkv, 576] or dv_resp [R, Hkv, 512]
   int32_t* status;
-  int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles;   // tiles of 64 rows
+  int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;   // tiles of 64 rows
   int part_first, part_count;   // mode DQ: partials [part_first, part_first + part_count) are computed
   float scale, scale_log2;
 };
@@ -148,7 +150,8 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
       const bool dense = (MODE != MLA_DQ) || is_resp;
       auto fetch = [&](int tile) -> int {
         const int ps = (tile * 64) >> p.pg_shift;
-        return (!dense && tile < n_tiles && ps < n_pages) ? __ldg(pages + ps) : 0;
+        if (dense) return 0;
+        return (tile < n_tiles && ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
       };
       uint32_t slot = 0, phase = 0, issued = 0;
       bool ok = true;
@@ -406,14 +409,10 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
 
 template <int MODE>
 static ls_status_t launch_mla(const MlaBwdParams& prm, int64_t grid, cudaStream_t st, bool timed = true) {
-  static bool configured = false;
+  static bool configured[64] = {};
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  if (!configured) {
-    if (cudaFuncSetAttribute(bwd_mla_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMlaSmem) !=
-        cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
+  const ls_status_t cfg = configure_smem(bwd_mla_kernel<MODE>, kMlaSmem, configured);
+  if (cfg != LS_OK) return cfg;
   constexpr int which = MODE == MLA_DQ ? LS_KERNEL_BWD_DQ : MODE == MLA_DK ? LS_KERNEL_BWD_DK : LS_KERNEL_BWD_DV;
   if (timed) profile_begin(which, st);
   bwd_mla_kernel<MODE><<<(int)grid, kMlaThreads, kMlaSmem, st>>>(prm);
@@ -432,10 +431,10 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
     return encode_map5(m, base, dim, R, heads, 1, (int64_t)heads * dim, dim, (int64_t)R * heads * dim, 64, 1);
   };
   MlaBwdParams P;
-  P.shard_phys_pages = h->d_shard_phys_pages;
-  P.shard_page_offset = h->d_shard_page_offset;
-  P.shard_tail_slot = h->d_shard_tail_slot;
-  P.shard_tokens = h->d_shard_tokens;
+  P.shard_phys_pages = h->d_part_pages;
+  P.shard_page_offset = h->d_part_page_offset;
+  P.shard_tail_slot = h->d_part_tail_slot;
+  P.shard_tokens = h->d_part_tokens;
   P.lse = lse;
   P.delta = delta;
   P.dq_part = dq_part;
@@ -445,10 +444,11 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   P.Hq = Hq;
   P.Hkv = Hkv;
   P.g = Hq / Hkv;
-  P.S = d.num_shards * h->fine;
-  P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
+  P.S = h->num_parts();
+  P.pg_shift = pg_shift_of(d.page_size);
   P.tiles_per_head = (R + 63) / 64;
   P.nq_tiles = P.g * P.tiles_per_head;
+  P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.part_first = dq_resp_only ? P.S : 0;
   P.part_count = dq_resp_only ? 1 : P.S + 1;
   P.scale = prm->scale;
@@ -458,10 +458,10 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, kD2);
   if (st == LS_OK) st = dense_map(&P.b1r_map, k_resp, Hkv, kD1);
   if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, kD2);
-  if (st == LS_OK) st = encode_pool_map5(&P.bk_map, h, 0, 64, 1, false);
-  if (st == LS_OK) st = encode_pool_map5(&P.bk_tail, h, 0, 64, 1, true);
-  if (st == LS_OK) st = encode_pool_map5(&P.bv_map, h, 1, 64, 1, false);
-  if (st == LS_OK) st = encode_pool_map5(&P.bv_tail, h, 1, 64, 1, true);
+  if (st == LS_OK) st = pool_map(&P.bk_map, h, 0, 64, 1, false);
+  if (st == LS_OK) st = pool_map(&P.bk_tail, h, 0, 64, 1, true);
+  if (st == LS_OK) st = pool_map(&P.bv_map, h, 1, 64, 1, false);
+  if (st == LS_OK) st = pool_map(&P.bv_tail, h, 1, 64, 1, true);
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
   st = launch_mla<MLA_DQ>(P, (int64_t)Hkv * P.part_count * P.nq_tiles * 3, cs, !dq_resp_only);

@@ -23,7 +23,7 @@
 // [S^T | T^T] of tile i + 2 while the key threads work on tile i + 1.
 #include <cuda_bf16.h>
 
-#include <cstdlib>
+#include <algorithm>
 
 #include "ls_internal.h"
 #include "ls_sm100.cuh"
@@ -43,16 +43,17 @@ struct MlaDqParams {
   const float* dq_resp;              // [R, Hq, 576] fp32, unscaled: the response block's part
   __nv_bfloat16* dq;                 // [R, Hq, 576]
   int32_t* status;
-  int R, Hq, g, nparts, pg_shift, tiles_per_head;
+  long long* timing;   // diagnostic builds only
+  int R, Hq, g, nparts, pg_shift, tiles_per_head, num_phys_pages;
   int ablate;   // diagnostic builds only: 1 = no key loads, 2 = no tensor-core instructions
   float scale, scale_log2;
 };
 
 // Build with -DLS_TIMING to make CTA 0 write per-role cycle counts (time spent in each kind
-// of wait, and in total) as int64 words starting 64 bytes past `status`; a profiling aid.
+// of wait, and in total) into the buffer given to ls_debug_timing_buffer; a profiling aid.
 #ifdef LS_TIMING
 #define LS_TQWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
-#define LS_TQDUMP(slot, val) do { if (blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
+#define LS_TQDUMP(slot, val) do { if (blockIdx.x == 0 && p.timing) p.timing[(slot)] = (val); } while (0)
 #define LS_TQABLATE(bit) (p.ablate & (bit))
 #else
 #define LS_TQWAIT(acc, expr) (expr)
@@ -168,7 +169,9 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
         for (int half = 0; half < 2; ++half) {
           const int tok = w.tile * 128 + half * 64;
           const int ps = tok >> p.pg_shift;
-          w.page[half] = ps < w.c_pages ? __ldg(p.shard_phys_pages + w.c_off + ps) : 0;
+          // past the part's last page: a coordinate beyond the pool, where TMA fills zeros (the bytes of
+          // an arbitrary page could be NaN patterns, and 0 * NaN would poison dQ^T)
+          w.page[half] = ps < w.c_pages ? __ldg(p.shard_phys_pages + w.c_off + ps) : p.num_phys_pages;
           w.tok[half] = tok & pg_mask;
           w.tail[half] = ps == w.c_tail;
         }
@@ -420,9 +423,7 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
 
 bool mla_dq_fast(const ls_pages* h) {
   const ls_pages_desc_t& d = h->desc;
-  if (!(d.dim_k == 576 && d.dim_v == 512 && d.v_aliases_k && d.prefix_len > 0)) return false;
-  const char* e = getenv("LS_MLA_DQ");
-  return !(e && e[0] == '0');
+  return d.dim_k == 576 && d.dim_v == 512 && d.v_aliases_k && d.prefix_len > 0;
 }
 
 // dQ (bf16, final) of the 576/512 shape with V aliasing K: prefix part in this kernel, plus
@@ -433,10 +434,10 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   const ls_pages_desc_t& d = h->desc;
   const int R = prm->R, Hq = prm->num_q_heads;
   MlaDqParams P;
-  P.shard_phys_pages = h->d_shard_phys_pages;
-  P.shard_page_offset = h->d_shard_page_offset;
-  P.shard_tail_slot = h->d_shard_tail_slot;
-  P.shard_tokens = h->d_shard_tokens;
+  P.shard_phys_pages = h->d_part_pages;
+  P.shard_page_offset = h->d_part_page_offset;
+  P.shard_tail_slot = h->d_part_tail_slot;
+  P.shard_tokens = h->d_part_tokens;
   P.lse = lse;
   P.delta = delta;
   P.dq_resp = dq_resp;
@@ -445,28 +446,24 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   P.R = R;
   P.Hq = Hq;
   P.g = Hq / d.num_kv_heads;
-  P.nparts = d.num_shards * h->fine;
-  P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
+  P.nparts = h->prefix_parts();
+  P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
+  P.pg_shift = pg_shift_of(d.page_size);
   P.tiles_per_head = (R + kTqRows - 1) / kTqRows;
-  P.ablate = 0;
-#ifdef LS_TIMING
-  if (const char* e = getenv("LS_TQ_ABLATE")) P.ablate = atoi(e);
-#endif
+  P.ablate = (prm->flags & LS_DBG_ABLATE_LOADS ? 1 : 0) | (prm->flags & LS_DBG_ABLATE_MMA ? 2 : 0);
+  P.timing = g_timing_buffer;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * kLog2eTq;
   ls_status_t st = encode_map5(&P.q_map, q, 576, R, Hq, 1, (int64_t)Hq * 576, 576, (int64_t)R * Hq * 576, 64, 1);
   if (st == LS_OK) st = encode_map5(&P.do_map, d_o, 512, R, Hq, 1, (int64_t)Hq * 512, 512, (int64_t)R * Hq * 512, 64, 1);
-  if (st == LS_OK) st = encode_pool_map5(&P.k_map, h, 0, 64, 1, false);
-  if (st == LS_OK) st = encode_pool_map5(&P.k_tail, h, 0, 64, 1, true);
-  if (st == LS_OK) st = encode_pool_map5(&P.k2_map, h, 0, 64, 2, false);
-  if (st == LS_OK) st = encode_pool_map5(&P.k2_tail, h, 0, 64, 2, true);
+  if (st == LS_OK) st = pool_map(&P.k_map, h, 0, 64, 1, false);
+  if (st == LS_OK) st = pool_map(&P.k_tail, h, 0, 64, 1, true);
+  if (st == LS_OK) st = pool_map(&P.k2_map, h, 0, 64, 2, false);
+  if (st == LS_OK) st = pool_map(&P.k2_tail, h, 0, 64, 2, true);
   if (st != LS_OK) return st;
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(bwd_mla_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTqSmem) != cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
+  static bool configured[64] = {};
+  const ls_status_t cfg = configure_smem(bwd_mla_dq_kernel, kTqSmem, configured);
+  if (cfg != LS_OK) return cfg;
   const int64_t grid = (int64_t)Hq * P.tiles_per_head;
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   profile_begin(LS_KERNEL_BWD_DQ, cs);

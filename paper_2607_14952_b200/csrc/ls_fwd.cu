@@ -20,48 +20,158 @@
 // TMEM columns: O [0, DVT), S/P buffer 0 [DVT, DVT+128), S/P buffer 1 [DVT+128, DVT+256).
 // K chunk  = 128 keys x 64*KSLABS channels (K-major, 128-byte swizzle): k-slices of S.
 // V chunk  = VKEYS keys x DVT channels as DVT/64 sub-slabs (MN-major): VKEYS/16 k-steps of PV.
-#include <cstdlib>
-
 #include "ls_internal.h"
 #include "ls_sm100.cuh"
 
 namespace ls {
 
+// How the CTAs of one launch hand their results over (FwdParams::chain_mode):
+//   0  every work item writes its own partial (o_r, l_r);
+//   1  the `fine` consecutive sub-shards of a shard fold into that shard's partial, in order;
+//   2  every part -- the response block first, then the prefix sub-shards, then the suffix
+//      blocks -- folds into one composed output (Eq. qwen-global-attn), in that order.
+// Folding is the pairwise form of Eq. qwen-lse-parts on normalised values:
+//   m = max(l, l_r); a = e^{l-m} + e^{l_r-m}; o = (e^{l-m} o + e^{l_r-m} o_r) / a; l = m + log a.
 struct FwdParams {
   CUtensorMap q_map;               // box 64 x 128 tokens x KSLABS channel groups
   CUtensorMap k_map, k_tail_map;   // pool K: box 64 x 128 x KSLABS (pages >= 128 tokens) or 64 x 64 x 1
-  CUtensorMap v_map, v_tail_map;   // pool V: box 64 x 64 tokens x DV/64 groups
-  CUtensorMap kr_map, vr_map;      // response K (64 x 128 x KSLABS) and V (64 x 64 x DV/64)
+  CUtensorMap v_map, v_tail_map;   // pool V: box 64 x VKEYS tokens x DVT/64 groups
+  CUtensorMap kr_map, vr_map;      // response K (64 x 128 x KSLABS) and V (64 x VKEYS x DVT/64)
   // CTA-pair variant (D = 256): every box is 64 channels x 64 tokens x 2 groups (16 KB)
   CUtensorMap pk2, pk2_tail, pv2, pv2_tail, rk2, rv2;
-  const int32_t* shard_phys_pages;
-  const int32_t* shard_page_offset;
-  const int32_t* shard_tail_slot;
-  const int64_t* shard_tokens;
-  float* o_part;       // prefix partials [S, R, Hq, dv] (S = sub-shards seen by the kernel)
-  float* lse_part;
-  float* o_resp;       // the response block's partial [R, Hq, dv]
+  const int32_t* part_pages;
+  const int32_t* part_page_offset;
+  const int32_t* part_tail_slot;
+  const int64_t* part_tokens;
+  float* o_out;        // modes 0, 1: prefix partials [S_out, R, Hq, dv]; mode 2: the running output [R, Hq, dv]
+  float* lse_out;
+  float* o_resp;       // modes 0, 1: the response block's partial [R, Hq, dv]
   float* lse_resp;
+  __nv_bfloat16* o_bf16;   // mode 2: composed output in bf16, written by the last link (nullable)
+  float* lse_aux;      // two O tiles per Q tile: running l of the second tile's chain
+  int* ctl;            // hand-over control words (ticket, abort, counters) or NULL
   int32_t* status;
-  int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  long long* timing;   // diagnostic builds only
+  int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  int chain_mode, fine;
   int dv_total;   // channels of one output row (DVT times the number of O tiles)
-  int prefetch;   // L2 prefetch distance in 128-key tiles (0 = off)
   int packed;     // 1: one Q tile holds every (head, token) row of a KV group (g * R <= 128 rows);
                   //    row r is head r / R, token r % R.  Lets a short response stream K/V once.
   int q_bytes;    // bytes the Q loads deliver
-  int ablate;   // diagnostic: LS_FLAG_ABLATE_* bits (results are then meaningless)
+  int ablate;     // diagnostic builds only (LS_DBG_ABLATE_*)
   float scale, scale_log2;
 };
 
 // Build with -DLS_TIMING to make CTA 0 write per-role cycle counts (time spent in each kind
-// of wait, and in total) as int64 words starting 64 bytes past `status`; a profiling aid.
+// of wait, and in total) into the buffer given to ls_debug_timing_buffer; a profiling aid.
 #ifdef LS_TIMING
 #define LS_TWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
-#define LS_TDUMP(slot, val) do { if (blockIdx.x == 0 && p.status) reinterpret_cast<long long*>(p.status)[8 + (slot)] = (val); } while (0)
+#define LS_TDUMP(slot, val) do { if (blockIdx.x == 0 && p.timing) p.timing[(slot)] = (val); } while (0)
+#define LS_ABLATE(bit) ((p.ablate & (bit)) != 0)
 #else
 #define LS_TWAIT(acc, expr) (expr)
 #define LS_TDUMP(slot, val) do { } while (0)
+#define LS_ABLATE(bit) false
 #endif
+
+// One work item: which keys (part), which Q rows, and where the result goes.
+struct FwdItem {
+  int kvh, part, qunit, link;
+  bool is_resp, chained, first, last;
+};
+__device__ __forceinline__ FwdItem fwd_item(const FwdParams& p, int idx, int n_qunits) {
+  FwdItem it;
+  it.qunit = idx % n_qunits;
+  idx /= n_qunits;
+  const int slots = p.parts + 1;
+  const int slot = idx % slots;
+  it.kvh = idx / slots;
+  if (p.chain_mode == 2) {
+    it.link = slot;
+    it.is_resp = slot == 0;
+    it.part = it.is_resp ? p.parts : slot - 1;
+    it.chained = true;
+    it.first = slot == 0;
+    it.last = slot == p.parts;
+  } else {
+    it.is_resp = slot == p.parts;
+    it.part = slot;
+    it.chained = p.chain_mode == 1 && !it.is_resp;
+    it.link = it.chained ? slot % p.fine : 0;
+    it.first = it.link == 0;
+    it.last = false;
+  }
+  return it;
+}
+// index of the partial that receives the item's rows, and of its hand-over counter
+__device__ __forceinline__ int fwd_out_part(const FwdParams& p, const FwdItem& it) {
+  return (p.chain_mode == 2 || it.is_resp) ? 0 : (p.chain_mode == 1 ? it.part / p.fine : it.part);
+}
+__device__ __forceinline__ int fwd_chain_index(const FwdParams& p, const FwdItem& it, int qtile) {
+  const int group = p.chain_mode == 2 ? it.kvh : it.kvh * (p.parts / p.fine) + it.part / p.fine;
+  return group * p.nq_tiles + qtile;
+}
+
+// One row thread's share of the epilogue: its (unnormalised) accumulator row in TMEM, the
+// row's running sum l and scaled reference maximum, normalised and either stored (fold =
+// false) or folded into the value already there.  Rows whose own partial weighs nothing
+// leave the running value untouched.
+template <int DV>
+__device__ __forceinline__ void fwd_store_row(uint32_t tmem_row, bool have_acc, float l, float m_scaled, bool fold,
+                                              float* o_dst, float* lse_dst, bool write_lse, __nv_bfloat16* bf_dst,
+                                              bool row_ok) {
+  const bool own = have_acc && l > 0.f;
+  const float lse_own = own ? m_scaled + logf(l) : -INFINITY;
+  float c_own = own ? 1.0f / l : 0.f, c_run = 0.f, lse_new = lse_own;
+  if (fold) {
+    const float lse_run = row_ok ? __ldcg(lse_dst) : -INFINITY;
+    const float m = fmaxf(lse_run, lse_own);
+    if (m == -INFINITY) {
+      c_own = 0.f;
+    } else {
+      const float w_run = expf(lse_run - m), w_own = expf(lse_own - m);
+      const float inv_a = 1.0f / (w_run + w_own);
+      c_run = w_run * inv_a;
+      c_own *= w_own * inv_a;
+      lse_new = m + logf(w_run + w_own);
+    }
+  }
+  const bool store = row_ok && (!fold || c_own != 0.f || bf_dst != nullptr);
+  const bool load_run = fold && c_run != 0.f;
+#pragma unroll 1
+  for (int c = 0; c < DV; c += 32) {
+    uint32_t o[32];
+    if (have_acc) {
+      tmem_ld32(tmem_row + c, o);
+      tc_wait_ld32(o);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[j] = 0u;
+    }
+    if (store) {
+      float4 run[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        run[j] = load_run ? __ldcg(reinterpret_cast<const float4*>(o_dst + c) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float4 v;
+        v.x = fmaf(c_run, run[j].x, c_own * __uint_as_float(o[4 * j]));
+        v.y = fmaf(c_run, run[j].y, c_own * __uint_as_float(o[4 * j + 1]));
+        v.z = fmaf(c_run, run[j].z, c_own * __uint_as_float(o[4 * j + 2]));
+        v.w = fmaf(c_run, run[j].w, c_own * __uint_as_float(o[4 * j + 3]));
+        *(reinterpret_cast<float4*>(o_dst + c) + j) = v;
+        if (bf_dst) {
+          uint2 pk;
+          pk.x = pack_bf16(v.x, v.y);
+          pk.y = pack_bf16(v.z, v.w);
+          *(reinterpret_cast<uint2*>(bf_dst + c) + j) = pk;
+        }
+      }
+    }
+  }
+  if (store && write_lse) *lse_dst = lse_new;
+}
 
 constexpr int kFwdThreads = 192;
 constexpr float kRescaleLog2 = 8.0f;   // the reference max lags the true max by at most 2^8
@@ -79,6 +189,11 @@ struct FwdCfg {
   static constexpr int Q_BYTES = (DK / 64) * 16384;
   static constexpr int SMEM_BYTES = 1024 + Q_BYTES + RING * CHUNK + 512;
 };
+
+// Row-thread wait: the warp leaves together (the TMEM loads and votes that follow need every lane).
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+}
 
 template <int DK, int DVT, int NDV>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_constant__ FwdParams p) {
@@ -98,34 +213,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   uint64_t* o_final = pv_done + 1;      // the last tile's P V finished
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(o_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* work_idx = const_cast<int*>(abort_flag) + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
   (void)tw0; (void)tw1; (void)tw2;
-
-  // ---- work item
-  int idx = blockIdx.x;
-  const int dvh = idx % NDV;            // which DVT-wide slice of the value channels
-  idx /= NDV;
-  const int qtile = idx % p.nq_tiles;
-  idx /= p.nq_tiles;
-  const int part = idx % (p.S + 1);
-  const int kvh = idx / (p.S + 1);
-  const int h = kvh * p.g + qtile / p.tiles_per_head;
-  const int ttile = qtile % p.tiles_per_head;
-  const int t0 = ttile * 128;
-  const bool is_resp = (part == p.S);
-  int64_t tokens;
-  int page_off = 0, n_pages = 0, tail_slot = -1;
-  if (is_resp) {
-    tokens = min(p.R, t0 + 128);                       // keys 0 .. last row of this tile
-  } else {
-    tokens = p.shard_tokens[part];
-    page_off = p.shard_page_offset[part];
-    n_pages = p.shard_page_offset[part + 1] - page_off;
-    tail_slot = p.shard_tail_slot[part];
-  }
-  const int n_tiles = (int)((tokens + 127) / 128);
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -140,6 +232,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     mbar_init(pv_done, 1);
     mbar_init(o_final, 1);
     *abort_flag = 0;
+    // work items are handed out in launch order of the CTAs that ask, so an item never waits
+    // for one that no CTA has started
+    *work_idx = p.ctl ? atomicAdd(p.ctl, 1) : (int)blockIdx.x;
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -153,17 +248,39 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   const uint32_t tmem_o = tmem_base;
   const uint32_t tmem_s0 = tmem_base + DV;
 
+  // ---- work item
+  int idx = *work_idx;
+  const int dvh = idx % NDV;            // which DVT-wide slice of the value channels
+  idx /= NDV;
+  const FwdItem it = fwd_item(p, idx, p.nq_tiles);
+  const int qtile = it.qunit, part = it.part, kvh = it.kvh;
+  const int h = kvh * p.g + qtile / p.tiles_per_head;
+  const int ttile = qtile % p.tiles_per_head;
+  const int t0 = ttile * 128;
+  const bool is_resp = it.is_resp;
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, t0 + 128);                       // keys 0 .. last row of this tile
+  } else {
+    tokens = p.part_tokens[part];
+    page_off = p.part_page_offset[part];
+    n_pages = p.part_page_offset[part + 1] - page_off;
+    tail_slot = p.part_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 127) / 128);
+
   if (warp == 0) {
     // =========================================================== producer (one thread)
     if (lane == 0 && n_tiles > 0) {
-      const bool no_loads = (p.ablate & LS_FLAG_ABLATE_LOADS) != 0;
+      const bool no_loads = LS_ABLATE(LS_DBG_ABLATE_LOADS);
       mbar_arrive_expect_tx(q_full, p.q_bytes);
       for (int c = 0; c < DK / 64; ++c) tma_load_5d(q_smem + c * 16384, &p.q_map, q_full, 0, t0, c, h, 0);
 
-      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
       const bool small_pages = p.pg_shift == 6;          // 64-token pages: a tile spans two pages
-      // physical page of the shard's page slot; past the shard's last page the coordinate points
+      // physical page of the part's page slot; past the part's last page the coordinate points
       // beyond the pool and TMA fills zeros
       auto fetch = [&](int slot_idx) -> int {
         return (slot_idx < n_pages) ? __ldg(pages + slot_idx) : p.num_phys_pages;
@@ -224,29 +341,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           advance();
         }
       };
-      // L2 prefetch of the K and V boxes of a tile that will be loaded `prefetch` tiles later
-      auto prefetch_tile = [&](int tile, int pa, int pb) {
-        if (is_resp || tile >= n_tiles) return;
-        const int tok = tile * 128;
-        if (!small_pages) {
-          const bool tail = (tok >> p.pg_shift) == tail_slot;
-          for (int c = 0; c < C::KCH; ++c)
-            tma_prefetch_5d(tail ? &p.k_tail_map : &p.k_map, 0, tok & pg_mask, c * C::KSLABS, kvh, pa);
-          for (int r = 0; r < C::NVCH; ++r)
-            tma_prefetch_5d(tail ? &p.v_tail_map : &p.v_map, 0, (tok + r * C::VKEYS) & pg_mask, dvh * C::VSUB, kvh, pa);
-        } else {
-          for (int c = 0; c < C::KCH * C::KSLABS; ++c) {
-            tma_prefetch_5d((tok >> 6) == tail_slot ? &p.k_tail_map : &p.k_map, 0, 0, c, kvh, pa);
-            tma_prefetch_5d((tok >> 6) + 1 == tail_slot ? &p.k_tail_map : &p.k_map, 0, 0, c, kvh, pb);
-          }
-          for (int r = 0; r < C::NVCH; ++r) {
-            const int tk = tok + r * C::VKEYS;
-            tma_prefetch_5d((tk >> 6) == tail_slot ? &p.v_tail_map : &p.v_map, 0, tk & 63, dvh * C::VSUB, kvh,
-                            (r * C::VKEYS >= 64) ? pb : pa);
-          }
-        }
-      };
       const long long t_begin_p = clock64();
+      (void)t_begin_p;
       // page ids of tile i: slots (128 i) >> pg_shift and, for 64-token pages, the next one
       int pa0 = 0, pb0 = 0, pa1 = 0, pb1 = 0;
       if (!is_resp) {
@@ -258,29 +354,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         }
       }
       load_k(0, pa0, pb0);
-      const int pf = p.prefetch;
-      int pfa = 0, pfb = 0;                          // pages of tile i + pf (fetched one round early)
-      if (pf > 0 && !is_resp && pf < n_tiles) {
-        const int sp = (pf * 128) >> p.pg_shift;
-        pfa = fetch(sp);
-        pfb = small_pages ? fetch(sp + 1) : pfa;
-      }
       for (int i = 0; i < n_tiles; ++i) {
         int pa2 = 0, pb2 = 0;                       // prefetched two tiles ahead, used next iteration
         if (!is_resp && i + 2 < n_tiles) {
           const int s2 = ((i + 2) * 128) >> p.pg_shift;
           pa2 = fetch(s2);
           pb2 = small_pages ? fetch(s2 + 1) : pa2;
-        }
-        if (pf > 0) {
-          int na = 0, nb = 0;
-          if (!is_resp && i + 1 + pf < n_tiles) {
-            const int sp = ((i + 1 + pf) * 128) >> p.pg_shift;
-            na = fetch(sp);
-            nb = small_pages ? fetch(sp + 1) : na;
-          }
-          prefetch_tile(i + pf, pfa, pfb);
-          pfa = na; pfb = nb;
         }
         if (i + 1 < n_tiles) load_k(i + 1, pa1, pb1);
         load_v(i, pa0, pb0);
@@ -308,9 +387,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
       const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major chunk
       const uint32_t ring_v_lo = sdesc_lo(smem_u32(ring), C::VKEYS * 128);   // MN-major chunk: sub-slab pitch
       uint32_t slot = 0, phase = 0;
-      const bool no_mma = (p.ablate & LS_FLAG_ABLATE_MMA) != 0;
+      const bool no_mma = LS_ABLATE(LS_DBG_ABLATE_MMA);
       bool ok = mbar_wait(q_full, 0, abort_flag);
       const long long t_begin = clock64();
+      (void)t_begin;
       auto advance = [&]() {
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
@@ -377,27 +457,25 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
     const bool row_ok = p.packed ? row < p.g * p.R : t < p.R;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const size_t out_row = ((size_t)(is_resp ? 0 : part) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
-    float* o_dst = (is_resp ? p.o_resp : p.o_part) + out_row * p.dv_total + dvh * DVT;
-    float* lse_dst = (is_resp ? p.lse_resp : p.lse_part) + out_row;
-    if (n_tiles == 0) {
-      if (row_ok) {
-        for (int c = 0; c < DV; c += 4) *reinterpret_cast<float4*>(o_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (dvh == 0) *lse_dst = -INFINITY;
-      }
-    } else {
+    const size_t out_row = ((size_t)fwd_out_part(p, it) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
+    const bool to_resp = is_resp && p.chain_mode != 2;
+    float* o_dst = (to_resp ? p.o_resp : p.o_out) + out_row * p.dv_total + dvh * DVT;
+    float* lse_dst = (to_resp ? p.lse_resp : p.lse_out) + out_row;
+    if (dvh != 0 && it.chained) lse_dst = p.lse_aux + out_row;     // the second O tile's chain keeps its own copy of l
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    if (n_tiles > 0) {
       // last visible key index of this row inside this partial
       const int64_t lim = is_resp ? (int64_t)min(t, p.R - 1) : tokens - 1;
-      float m_ref = -INFINITY, l = 0.f;
       const long long t_begin_sm = clock64();
+      (void)t_begin_sm;
       const float thresh = kRescaleLog2 / p.scale_log2;
-      bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
         const uint32_t ts = tmem_s0 + (i & 1) * 128 + lane_sel;
-        ok = LS_TWAIT(tw0, mbar_wait(&s_full[i & 1], (i >> 1) & 1, abort_flag));
+        ok = LS_TWAIT(tw0, mbar_wait_warp(&s_full[i & 1], (i >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        if (p.ablate & LS_FLAG_ABLATE_SOFTMAX) {
+        if (LS_ABLATE(LS_DBG_ABLATE_SOFTMAX)) {
           tc_fence_before();
           mbar_arrive(&p_full[i & 1]);
           continue;
@@ -427,7 +505,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
           m_ref = (mx == -INFINITY) ? 0.f : mx;
         } else if (__any_sync(0xffffffffu, mx > m_ref + thresh)) {
           // rare: raise the reference maximum and rescale the running sum and O
-          ok = LS_TWAIT(tw1, mbar_wait(pv_done, (i - 1) & 1, abort_flag));
+          ok = LS_TWAIT(tw1, mbar_wait_warp(pv_done, (i - 1) & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
           const float m_new = fmaxf(m_ref, mx);
@@ -469,25 +547,20 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         LS_TDUMP(17, tw1);
         LS_TDUMP(18, clock64() - t_begin_sm);
       }
-      if (ok) ok = mbar_wait(o_final, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
-#pragma unroll 1
-        for (int c = 0; c < DV; c += 32) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_sel + c, o);
-          tc_wait_ld32(o);
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(o_dst + c + j) =
-                  make_float4(__uint_as_float(o[j]) * inv_l, __uint_as_float(o[j + 1]) * inv_l,
-                              __uint_as_float(o[j + 2]) * inv_l, __uint_as_float(o[j + 3]) * inv_l);
-          }
-        }
-        if (row_ok && dvh == 0) *lse_dst = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
-      }
+      if (ok) ok = mbar_wait_warp(o_final, 0, abort_flag);
+      if (ok) tc_fence_after();
+    }
+    // ---- epilogue: store this partial, or fold it into the running value of its chain
+    int* counter = it.chained ? p.ctl + kChainHeaderInts + fwd_chain_index(p, it, qtile) * NDV + dvh : nullptr;
+    const bool fold = it.chained && !it.first;
+    if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
+    if (ok)
+      fwd_store_row<DV>(tmem_o + lane_sel, n_tiles > 0, l, m_ref * p.scale, fold, o_dst, lse_dst,
+                        dvh == 0 || it.chained, (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total + dvh * DVT : nullptr,
+                        row_ok);
+    if (it.chained) {
+      const bool all_ok = bar_and(2, 128, ok);     // every row of the tile is written
+      if (row == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
 
@@ -497,7 +570,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
-  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+    if (p.ctl) st_relaxed_gpu(p.ctl + 1, 1);    // ends every other chain wait of this launch
+  }
 }
 
 // ---------------------------------------------------------------------------------
@@ -534,42 +610,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   uint64_t* o_final = pv_done + 1;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(o_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* work_idx = const_cast<int*>(abort_flag) + 1;   // (even CTA) the pair's work item
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
-
-  // ---- work item of the pair, and this CTA's Q tile
-  const int npairs = (p.nq_tiles + 1) / 2;
-  int idx = blockIdx.x >> 1;
-  const int pairi = idx % npairs;
-  idx /= npairs;
-  const int part = idx % (p.S + 1);
-  const int kvh = idx / (p.S + 1);
-  const bool is_resp = (part == p.S);
-  auto tile_of = [&](int qt, int& hh, int& r0) {
-    if (qt < p.nq_tiles) {
-      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
-      r0 = (qt % p.tiles_per_head) * 128;
-    } else {                                 // odd tile count: the pair's second CTA works on zero rows
-      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
-      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
-    }
-  };
-  int h, t0, h_o, t0_o;
-  tile_of(2 * pairi + (int)rank, h, t0);
-  tile_of(2 * pairi + 1 - (int)rank, h_o, t0_o);
-  int64_t tokens;
-  int page_off = 0, n_pages = 0, tail_slot = -1;
-  if (is_resp) {
-    tokens = min(p.R, max(t0, t0_o) + 128);          // both CTAs walk the longer causal range
-  } else {
-    tokens = p.shard_tokens[part];
-    page_off = p.shard_page_offset[part];
-    n_pages = p.shard_page_offset[part + 1] - page_off;
-    tail_slot = p.shard_tail_slot[part];
-  }
-  const int n_tiles = (int)((tokens + 127) / 128);
 
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
@@ -584,6 +629,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     mbar_init(pv_done, 1);
     mbar_init(o_final, 1);
     *abort_flag = 0;
+    // work items are handed out in launch order of the pairs that ask (see chain_wait)
+    if (leader) *work_idx = p.ctl ? atomicAdd(p.ctl, 1) : (int)(blockIdx.x >> 1);
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -598,12 +645,42 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   const uint32_t tmem_o = tmem_base;
   const uint32_t tmem_s0 = tmem_base + DV;
 
+  // ---- work item of the pair, and this CTA's Q tile
+  const int npairs = (p.nq_tiles + 1) / 2;
+  const FwdItem it = fwd_item(p, (int)ld_shared_cluster_u32(mapa_u32(smem_u32(work_idx), 0)), npairs);
+  const int pairi = it.qunit, part = it.part, kvh = it.kvh;
+  const bool is_resp = it.is_resp;
+  auto tile_of = [&](int qt, int& hh, int& r0) {
+    if (qt < p.nq_tiles) {
+      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      r0 = (qt % p.tiles_per_head) * 128;
+    } else {                                 // odd tile count: the pair's second CTA works on zero rows
+      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
+    }
+  };
+  const int qtile = 2 * pairi + (int)rank;
+  int h, t0, h_o, t0_o;
+  tile_of(qtile, h, t0);
+  tile_of(2 * pairi + 1 - (int)rank, h_o, t0_o);
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = min(p.R, max(t0, t0_o) + 128);          // both CTAs walk the longer causal range
+  } else {
+    tokens = p.part_tokens[part];
+    page_off = p.part_page_offset[part];
+    n_pages = p.part_page_offset[part + 1] - page_off;
+    tail_slot = p.part_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 127) / 128);
+
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
       if (leader) mbar_arrive_expect_tx(q_full, 2 * p.q_bytes);
       for (int c = 0; c < 4; ++c) tma_load_5d_pair(q_smem + c * 16384, &p.q_map, q_full, 0, t0, c, h, 0);
-      const int32_t* pages = p.shard_phys_pages + page_off;
+      const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
       auto page_at = [&](int tok) -> int {
         if (is_resp) return 0;
@@ -726,25 +803,22 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     const int row = quad * 32 + lane;
     const int t = p.packed ? t0 + row % p.R : t0 + row;
     const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
-    const bool row_ok = t < p.R && (!p.packed || row < p.g * p.R);
+    const bool tile_ok = qtile < p.nq_tiles;
+    const bool row_ok = tile_ok && t < p.R && (!p.packed || row < p.g * p.R);
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const size_t out_row = ((size_t)(is_resp ? 0 : part) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
-    float* o_dst = (is_resp ? p.o_resp : p.o_part) + out_row * p.dv_total;
-    float* lse_dst = (is_resp ? p.lse_resp : p.lse_part) + out_row;
-    if (n_tiles == 0) {
-      if (row_ok) {
-        for (int c = 0; c < DV; c += 4) *reinterpret_cast<float4*>(o_dst + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-        *lse_dst = -INFINITY;
-      }
-    } else {
+    const size_t out_row = ((size_t)fwd_out_part(p, it) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
+    const bool to_resp = is_resp && p.chain_mode != 2;
+    float* o_dst = (to_resp ? p.o_resp : p.o_out) + out_row * p.dv_total;
+    float* lse_dst = (to_resp ? p.lse_resp : p.lse_out) + out_row;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    if (n_tiles > 0) {
       const int64_t lim = is_resp ? (int64_t)min(t, p.R - 1) : tokens - 1;
-      float m_ref = -INFINITY, l = 0.f;
       const float thresh = kRescaleLog2 / p.scale_log2;
       const uint32_t p_remote[2] = {mapa_u32(smem_u32(&p_full[0]), 0), mapa_u32(smem_u32(&p_full[1]), 0)};
-      bool ok = true;
       for (int i = 0; i < n_tiles && ok; ++i) {
         const uint32_t ts = tmem_s0 + (i & 1) * 128 + lane_sel;
-        ok = mbar_wait(&s_full[i & 1], (i >> 1) & 1, abort_flag);
+        ok = mbar_wait_warp(&s_full[i & 1], (i >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
         uint32_t sr[128];
@@ -772,7 +846,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
           m_ref = (mx == -INFINITY) ? 0.f : mx;
         } else if (__any_sync(0xffffffffu, mx > m_ref + thresh)) {
           // rare: raise the reference maximum and rescale the running sum and O (this CTA's rows)
-          ok = mbar_wait(pv_done, (i - 1) & 1, abort_flag);
+          ok = mbar_wait_warp(pv_done, (i - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const float m_new = fmaxf(m_ref, mx);
@@ -809,25 +883,20 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(p_remote[i & 1]);   // one arrival per warp, at the even CTA
       }
-      if (ok) ok = mbar_wait(o_final, 0, abort_flag);
-      if (ok) {
-        tc_fence_after();
-        const float inv_l = (l > 0.f) ? 1.0f / l : 0.f;
-#pragma unroll 1
-        for (int c = 0; c < DV; c += 32) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_sel + c, o);
-          tc_wait_ld32(o);
-          if (row_ok) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(o_dst + c + j) =
-                  make_float4(__uint_as_float(o[j]) * inv_l, __uint_as_float(o[j + 1]) * inv_l,
-                              __uint_as_float(o[j + 2]) * inv_l, __uint_as_float(o[j + 3]) * inv_l);
-          }
-        }
-        if (row_ok) *lse_dst = (l > 0.f) ? m_ref * p.scale + logf(l) : -INFINITY;
-      }
+      if (ok) ok = mbar_wait_warp(o_final, 0, abort_flag);
+      if (ok) tc_fence_after();
+    }
+    // ---- epilogue: store this partial, or fold it into the running value of its chain
+    const bool chained = it.chained && tile_ok;
+    int* counter = chained ? p.ctl + kChainHeaderInts + fwd_chain_index(p, it, qtile) : nullptr;
+    const bool fold = chained && !it.first;
+    if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
+    if (ok)
+      fwd_store_row<DV>(tmem_o + lane_sel, n_tiles > 0, l, m_ref * p.scale, fold, o_dst, lse_dst, true,
+                        (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total : nullptr, row_ok);
+    if (chained) {
+      const bool all_ok = bar_and(2, 128, ok);     // every row of the tile is written
+      if (row == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
 
@@ -838,18 +907,17 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
   }
-  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+    if (p.ctl) st_relaxed_gpu(p.ctl + 1, 1);    // ends every other chain wait of this launch
+  }
 }
 
 static ls_status_t launch_fwd2(const FwdParams& prm, int64_t grid, cudaStream_t st) {
-  static bool configured = false;
+  static bool configured[64] = {};
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  if (!configured) {
-    if (cudaFuncSetAttribute(fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Fwd2Cfg::SMEM_BYTES) !=
-        cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
+  const ls_status_t cs = configure_smem(fwd2_kernel, Fwd2Cfg::SMEM_BYTES, configured);
+  if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_FWD, st);
   fwd2_kernel<<<(int)grid, kFwdThreads, Fwd2Cfg::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_FWD, st);
@@ -859,127 +927,185 @@ static ls_status_t launch_fwd2(const FwdParams& prm, int64_t grid, cudaStream_t 
 template <int DK, int DVT, int NDV>
 static ls_status_t launch_fwd(const FwdParams& prm, int64_t grid, cudaStream_t st) {
   using C = FwdCfg<DK, DVT>;
-  static bool configured = false;
+  static bool configured[64] = {};
   if (grid * NDV > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  if (!configured) {
-    if (cudaFuncSetAttribute(fwd_kernel<DK, DVT, NDV>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             C::SMEM_BYTES) != cudaSuccess)
-      return LS_ERR_CUDA;
-    configured = true;
-  }
+  const ls_status_t cs = configure_smem(fwd_kernel<DK, DVT, NDV>, C::SMEM_BYTES, configured);
+  if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_FWD, st);
   fwd_kernel<DK, DVT, NDV><<<(int)(grid * NDV), kFwdThreads, C::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_FWD, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
+// Shape facts shared by the entry points.
+struct FwdShape {
+  int R, Hq, Hkv, g, dk, dv, nq_tiles, tiles_per_head, ndv;
+  bool mla, packed;
+};
+static FwdShape fwd_shape(const ls_pages* h, const ls_attn_params_t* prm) {
+  FwdShape f;
+  const ls_pages_desc_t& d = h->desc;
+  f.R = prm->R;
+  f.Hq = prm->num_q_heads;
+  f.Hkv = d.num_kv_heads;
+  f.g = f.Hq / f.Hkv;
+  f.dk = d.dim_k;
+  f.dv = d.dim_v;
+  f.mla = d.dim_k == 576;
+  f.packed = f.g * f.R <= 128 && f.g > 1;      // short response: every row of a KV group in one Q tile
+  f.tiles_per_head = (f.R + 127) / 128;
+  f.nq_tiles = f.packed ? 1 : f.g * f.tiles_per_head;
+  f.ndv = f.mla ? 2 : 1;
+  return f;
+}
+// bytes of hand-over control words for `chains` chains, rounded to 16
+static size_t ctl_bytes(int64_t chains) { return (size_t)((kChainHeaderInts + chains) * sizeof(int) + 15) & ~(size_t)15; }
+
+// mode: 0 / 1 = (S+1) partials (1 when shards are walked as sub-shards), 2 = composed output.
+static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, int mode, const void* q,
+                               const void* k_resp, const void* v_resp, float* o_out, float* lse_out, float* o_resp,
+                               float* lse_resp, void* o_bf16, void* workspace, int32_t* status_dev,
+                               cudaStream_t cs) {
+  const ls_pages_desc_t& d = h->desc;
+  const FwdShape f = fwd_shape(h, prm);
+  FwdParams P;
+  const int R = f.R, Hq = f.Hq, Hkv = f.Hkv;
+  const int kslabs = d.dim_k == 256 ? 2 : 1;
+  const int dvt = f.mla ? 256 : d.dim_v;                    // O channels per CTA
+  const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
+  const bool small_pages = d.page_size == 64;
+  const bool pair = d.dim_k == 256 && !f.packed;            // CTA pairs share every key tile between two Q tiles
+  ls_status_t st = f.packed ? encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, R, f.g)
+                            : encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, 128, 1);
+  if (pair) {
+    if (st == LS_OK) st = encode_map5(&P.rk2, k_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
+    if (st == LS_OK) st = encode_map5(&P.rv2, v_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
+    if (st == LS_OK) st = pool_map(&P.pk2, h, 0, 64, 2, false);
+    if (st == LS_OK) st = pool_map(&P.pk2_tail, h, 0, 64, 2, true);
+    if (st == LS_OK) st = pool_map(&P.pv2, h, 1, 64, 2, false);
+    if (st == LS_OK) st = pool_map(&P.pv2_tail, h, 1, 64, 2, true);
+  } else {
+    if (st == LS_OK)
+      st = encode_map5(&P.kr_map, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k,
+                       (int64_t)R * Hkv * d.dim_k, 128, kslabs);
+    if (st == LS_OK)
+      st = encode_map5(&P.vr_map, v_resp, d.dim_v, R, Hkv, 1, (int64_t)Hkv * d.dim_v, d.dim_v,
+                       (int64_t)R * Hkv * d.dim_v, vkeys, dvt / 64);
+    const int kbox = small_pages ? 64 : 128, kgroups = small_pages ? 1 : kslabs;
+    if (st == LS_OK) st = pool_map(&P.k_map, h, 0, kbox, kgroups, false);
+    if (st == LS_OK) st = pool_map(&P.k_tail_map, h, 0, kbox, kgroups, true);
+    if (st == LS_OK) st = pool_map(&P.v_map, h, 1, vkeys, dvt / 64, false);
+    if (st == LS_OK) st = pool_map(&P.v_tail_map, h, 1, vkeys, dvt / 64, true);
+  }
+  if (st != LS_OK) return st;
+  P.part_pages = h->d_part_pages;
+  P.part_page_offset = h->d_part_page_offset;
+  P.part_tail_slot = h->d_part_tail_slot;
+  P.part_tokens = h->d_part_tokens;
+  const int parts = h->num_parts();
+  P.o_out = o_out;
+  P.lse_out = lse_out;
+  P.o_resp = o_resp;
+  P.lse_resp = lse_resp;
+  P.o_bf16 = static_cast<__nv_bfloat16*>(o_bf16);
+  P.status = status_dev;
+  P.timing = g_timing_buffer;
+  P.R = R;
+  P.Hq = Hq;
+  P.Hkv = Hkv;
+  P.g = f.g;
+  P.parts = parts;
+  P.pg_shift = pg_shift_of(d.page_size);
+  P.tiles_per_head = f.tiles_per_head;
+  P.nq_tiles = f.nq_tiles;
+  P.packed = f.packed ? 1 : 0;
+  P.q_bytes = (d.dim_k / 64) * (f.packed ? f.g * R : 128) * 128;
+  P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
+  P.dv_total = d.dim_v;
+  P.chain_mode = mode;
+  P.fine = h->fine;
+  P.ablate = prm->flags & LS_DBG_ABLATE_MASK;
+  P.scale = prm->scale;
+  P.scale_log2 = prm->scale * 1.4426950408889634f;
+  // hand-over control words (and the second running l of the two-tile shape) at the workspace's start
+  P.ctl = nullptr;
+  P.lse_aux = nullptr;
+  if (mode != 0) {
+    const int64_t groups = mode == 2 ? Hkv : (int64_t)Hkv * d.num_shards;
+    const size_t cb = ctl_bytes(groups * f.nq_tiles * f.ndv);
+    P.ctl = static_cast<int*>(workspace);
+    P.lse_aux = reinterpret_cast<float*>(static_cast<char*>(workspace) + cb);
+    if (cudaMemsetAsync(workspace, 0, cb, cs) != cudaSuccess) return LS_ERR_CUDA;
+  }
+  if (pair) return launch_fwd2(P, (int64_t)Hkv * (parts + 1) * ((f.nq_tiles + 1) / 2) * 2, cs);
+  const int64_t grid = (int64_t)Hkv * (parts + 1) * f.nq_tiles;
+  return f.mla ? launch_fwd<576, 256, 2>(P, grid, cs)
+               : d.dim_k == 128 ? launch_fwd<128, 128, 1>(P, grid, cs) : launch_fwd<256, 256, 1>(P, grid, cs);
+}
+
+static ls_status_t check_forward_args(const ls_pages* h, const ls_attn_params_t* prm, const void* q,
+                                      const void* k_resp, const void* v_resp) {
+  ls_status_t st = check_handle(h, prm);
+  if (st != LS_OK) return st;
+  if (!q || !k_resp || !v_resp) return LS_ERR_INVALID_ARG;
+  const ls_pages_desc_t& d = h->desc;
+  if (prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % d.num_kv_heads != 0) return LS_ERR_INVALID_ARG;
+  if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_resp) || !aligned16(v_resp)) return LS_ERR_ALIGNMENT;
+  return LS_OK;
+}
+
 }  // namespace ls
 
 extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_attn_params_t* prm, int which) {
-  if (!h || !prm || prm->R < 1 || prm->num_q_heads < 1) return 0;
-  const size_t rows = (size_t)prm->R * prm->num_q_heads;
-  const size_t parts = (size_t)h->desc.num_shards * h->fine;      // sub-shard partials
-  // forward: sub-shard partials (O and LSE) when shards are sub-split, else nothing
-  if (which == LS_WORKSPACE_FWD) return h->fine > 1 ? parts * rows * (h->desc.dim_v + 1) * sizeof(float) : 0;
-  // backward: per-partial dQ (fp32) + Delta (fp32); the aliased 576/512 path sums the prefix
-  // partials in its accumulator and keeps only the response block's partial
-  if (ls::mla_dq_fast(h)) return rows * h->desc.dim_k * sizeof(float) + rows * sizeof(float);
-  return (parts + 1) * rows * h->desc.dim_k * sizeof(float) + rows * sizeof(float);
+  if (!h || !prm || prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % h->desc.num_kv_heads != 0) return 0;
+  const ls::FwdShape f = ls::fwd_shape(h, prm);
+  const size_t rows = (size_t)f.R * f.Hq;
+  const ls_pages_desc_t& d = h->desc;
+  if (which == LS_WORKSPACE_FWD) {
+    // nothing unless shards are walked as sub-shards: then one hand-over counter per (KV head, shard, Q tile)
+    if (h->fine == 1) return 0;
+    return ls::ctl_bytes((int64_t)f.Hkv * d.num_shards * f.nq_tiles * f.ndv) +
+           (f.mla ? (size_t)d.num_shards * rows * sizeof(float) : 0);
+  }
+  if (which == LS_WORKSPACE_FWD_MERGED)
+    return ls::ctl_bytes((int64_t)f.Hkv * f.nq_tiles * f.ndv) + (f.mla ? rows * sizeof(float) : 0);
+  if (which != LS_WORKSPACE_BWD) return 0;
+  // backward: Delta (fp32) + hand-over counters + the fp32 dQ that the partials are summed into
+  const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes((int64_t)f.Hkv * f.g * f.tiles_per_head);
+  if (f.mla && !ls::mla_dq_fast(h))     // 576/512 with a separate V pool: one fp32 dQ per partial
+    return head + (size_t)(h->num_parts() + 1) * rows * d.dim_k * sizeof(float);
+  return head + rows * d.dim_k * sizeof(float);
 }
 
 extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_params_t* prm, const void* q,
                                           const void* k_resp, const void* v_resp, float* o_part, float* lse_part,
                                           void* workspace, size_t workspace_bytes, int32_t* status_dev,
                                           void* stream) {
-  if (!h || !prm || !q || !k_resp || !v_resp || !o_part || !lse_part) return LS_ERR_INVALID_ARG;
-  if (!h->on_device) return LS_ERR_INVALID_ARG;
-  const ls_pages_desc_t& d = h->desc;
-  if (prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % d.num_kv_heads != 0) return LS_ERR_INVALID_ARG;
-  if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;
-  if (!ls::aligned16(q) || !ls::aligned16(k_resp) || !ls::aligned16(v_resp) || !ls::aligned16(o_part))
-    return LS_ERR_ALIGNMENT;
-  const bool mla = d.dim_k == 576 && d.dim_v == 512;
-  if (!((d.dim_k == 128 && d.dim_v == 128) || (d.dim_k == 256 && d.dim_v == 256) || mla))
-    return LS_ERR_UNSUPPORTED_SHAPE;
-
-  ls::FwdParams P;
-  const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads;
-  const int kslabs = d.dim_k == 256 ? 2 : 1;
-  const int dvt = mla ? 256 : d.dim_v;                    // O channels per CTA
-  const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
-  const bool small_pages = d.page_size == 64;
-  const int g = Hq / Hkv;
-  const bool packed = g * R <= 128 && g > 1;
-  ls_status_t st = packed ? ls::encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, R, g)
-                          : ls::encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, 128, 1);
-  if (st == LS_OK)
-    st = ls::encode_map5(&P.kr_map, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k,
-                         (int64_t)R * Hkv * d.dim_k, 128, kslabs);
-  if (st == LS_OK)
-    st = ls::encode_map5(&P.vr_map, v_resp, d.dim_v, R, Hkv, 1, (int64_t)Hkv * d.dim_v, d.dim_v,
-                         (int64_t)R * Hkv * d.dim_v, vkeys, dvt / 64);
-  const int kbox = small_pages ? 64 : 128, kgroups = small_pages ? 1 : kslabs;
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.k_map, h, 0, kbox, kgroups, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.k_tail_map, h, 0, kbox, kgroups, true);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_map, h, 1, vkeys, dvt / 64, false);
-  if (st == LS_OK) st = ls::encode_pool_map5(&P.v_tail_map, h, 1, vkeys, dvt / 64, true);
+  ls_status_t st = ls::check_forward_args(h, prm, q, k_resp, v_resp);
   if (st != LS_OK) return st;
-  P.shard_phys_pages = h->d_shard_phys_pages;
-  P.shard_page_offset = h->d_shard_page_offset;
-  P.shard_tail_slot = h->d_shard_tail_slot;
-  P.shard_tokens = h->d_shard_tokens;
-  const int64_t rows_all = (int64_t)R * Hq;
-  const int fine = h->fine;
-  const int parts = d.num_shards * fine;
-  float* fine_o = nullptr;
-  float* fine_lse = nullptr;
-  if (fine > 1) {
-    const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_FWD);
-    if (!workspace || workspace_bytes < need || !ls::aligned16(workspace)) return LS_ERR_WORKSPACE;
-    fine_o = static_cast<float*>(workspace);
-    fine_lse = fine_o + (size_t)parts * rows_all * d.dim_v;
-  }
-  P.o_part = fine > 1 ? fine_o : o_part;
-  P.lse_part = fine > 1 ? fine_lse : lse_part;
-  P.o_resp = o_part + (size_t)d.num_shards * rows_all * d.dim_v;
-  P.lse_resp = lse_part + (size_t)d.num_shards * rows_all;
-  P.status = status_dev;
-  P.R = R;
-  P.Hq = Hq;
-  P.Hkv = Hkv;
-  P.g = Hq / Hkv;
-  P.S = parts;
-  P.pg_shift = d.page_size == 64 ? 6 : d.page_size == 128 ? 7 : d.page_size == 256 ? 8 : 9;
-  P.tiles_per_head = (R + 127) / 128;
-  P.nq_tiles = packed ? 1 : P.g * P.tiles_per_head;
-  P.packed = packed ? 1 : 0;
-  P.q_bytes = (d.dim_k / 64) * (packed ? g * R : 128) * 128;
-  P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
-  P.dv_total = d.dim_v;
-  {
-    const char* e = getenv("LS_FWD_PREFETCH");
-    P.prefetch = e ? atoi(e) : 0;
-  }
-  P.ablate = prm->flags & LS_FLAG_ABLATE_MASK;
-  P.scale = prm->scale;
-  P.scale_log2 = prm->scale * 1.4426950408889634f;
-  const int64_t grid = (int64_t)Hkv * (parts + 1) * P.nq_tiles;
-  cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  const char* pair_env = getenv("LS_FWD_PAIR");
-  if (d.dim_k == 256 && !(pair_env && pair_env[0] == '0')) {
-    st = ls::encode_map5(&P.rk2, k_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
-    if (st == LS_OK)
-      st = ls::encode_map5(&P.rv2, v_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk2, h, 0, 64, 2, false);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pk2_tail, h, 0, 64, 2, true);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv2, h, 1, 64, 2, false);
-    if (st == LS_OK) st = ls::encode_pool_map5(&P.pv2_tail, h, 1, 64, 2, true);
-    if (st != LS_OK) return st;
-    st = ls::launch_fwd2(P, (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2, cs);
-  } else {
-    st = mla ? ls::launch_fwd<576, 256, 2>(P, grid, cs)
-             : d.dim_k == 128 ? ls::launch_fwd<128, 128, 1>(P, grid, cs) : ls::launch_fwd<256, 256, 1>(P, grid, cs);
-  }
-  if (st != LS_OK || fine == 1) return st;
-  return ls::group_merge(d.num_shards, fine, rows_all, d.dim_v, fine_o, fine_lse, o_part, lse_part, cs);
+  if (!o_part || !lse_part) return LS_ERR_INVALID_ARG;
+  if (!ls::aligned16(o_part)) return LS_ERR_ALIGNMENT;
+  if (!h->suffix_blocks.empty()) return LS_ERR_INVALID_ARG;     // per-shard partials describe the prefix only
+  const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_FWD);
+  if (need && (!workspace || workspace_bytes < need || !ls::aligned16(workspace))) return LS_ERR_WORKSPACE;
+  const int64_t rows_all = (int64_t)prm->R * prm->num_q_heads;
+  const int S = h->desc.num_shards;
+  return ls::run_forward(h, prm, h->fine > 1 ? 1 : 0, q, k_resp, v_resp, o_part, lse_part,
+                         o_part + (size_t)S * rows_all * h->desc.dim_v, lse_part + (size_t)S * rows_all, nullptr,
+                         workspace, status_dev, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" ls_status_t ls_replay_attn_fwd_merged(const ls_pages_t* h, const ls_attn_params_t* prm, const void* q,
+                                                 const void* k_resp, const void* v_resp, void* o_bf16, float* o_f32,
+                                                 float* lse, void* workspace, size_t workspace_bytes,
+                                                 int32_t* status_dev, void* stream) {
+  ls_status_t st = ls::check_forward_args(h, prm, q, k_resp, v_resp);
+  if (st != LS_OK) return st;
+  if (!o_f32 || !lse) return LS_ERR_INVALID_ARG;
+  if (!ls::aligned16(o_f32) || !ls::aligned16(o_bf16)) return LS_ERR_ALIGNMENT;
+  const size_t need = ls_replay_attn_workspace_bytes(h, prm, LS_WORKSPACE_FWD_MERGED);
+  if (!workspace || workspace_bytes < need || !ls::aligned16(workspace)) return LS_ERR_WORKSPACE;
+  return ls::run_forward(h, prm, 2, q, k_resp, v_resp, o_f32, lse, nullptr, nullptr, o_bf16, workspace, status_dev,
+                         static_cast<cudaStream_t>(stream));
 }

@@ -3,24 +3,42 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include <mutex>
 #include <vector>
 
 #include "ls.h"
 
+// Diagnostic builds only (-DLS_TIMING): flag bits in ls_attn_params_t::flags that skip one
+// pipeline stage (operand loads, tensor-core instructions, per-row arithmetic) while keeping
+// every barrier hand-off, so the cost of the remaining stages can be timed.  Outputs are
+// meaningless when one is set.  A regular build ignores these bits.
+#define LS_DBG_ABLATE_LOADS   (1 << 16)
+#define LS_DBG_ABLATE_MMA     (1 << 17)
+#define LS_DBG_ABLATE_SOFTMAX (1 << 18)
+#define LS_DBG_ABLATE_MASK    (7 << 16)
+
 namespace ls {
 
-constexpr int kNumBoxSizes = 4;               // token extents of the TMA boxes we encode
-constexpr int kBoxTok[kNumBoxSizes] = {16, 32, 64, 128};
-
-inline int box_index(int tok) { return tok == 16 ? 0 : tok == 32 ? 1 : tok == 64 ? 2 : 3; }
-
-// TMA descriptors of one bf16 pool viewed as (d, token, head, page); [box][0] covers a
-// full page, [box][1] the partially filled last logical page (tokens past the valid
-// count read as zero).
-struct PoolMaps {
-  CUtensorMap full[kNumBoxSizes];
-  CUtensorMap tail[kNumBoxSizes];
+// One cached TMA descriptor of the page pool: K (which = 0) or V (1) viewed as
+// (64 channels, token, 64-channel group, head, page) with a box of 64 x box_tok x box_groups;
+// tail = token extent bounded to the valid tokens of the partially filled last logical page.
+struct PoolMapEntry {
+  int which, box_tok, box_groups, tail;
+  CUtensorMap map;
 };
+
+// One block of response tokens appended behind the prefix (Sec. "Four-Block Response
+// Replay"): its pages in the pool and its slot range in the gradient pages.
+struct SuffixBlock {
+  int32_t tokens;
+  int32_t first_slot;     // first suffix page slot of the block
+  int32_t num_pages;
+};
+
+// Control words of the ordered hand-over between CTAs of one launch (see ls_sm100.cuh):
+// [0] ticket counter, [1] abort word, [2..3] unused, [4..] one completed-link counter per chain.
+constexpr int kChainHeaderInts = 4;
 
 }  // namespace ls
 
@@ -39,30 +57,39 @@ struct ls_pages {
 
   // Kernel-side plan: every shard is cut into `fine` contiguous sub-shards so that one
   // (KV head, sub-shard) stream of K and V fits comfortably in L2 while the CTAs that share it
-  // drift apart.  The device arrays below describe the S * fine sub-shards; the kernels treat
-  // them as S * fine partials and the host folds them back into the S the caller asked for.
+  // drift apart.  The kernels walk S * fine prefix parts (then one part per appended suffix
+  // block) and fold them back in a fixed order.
   int32_t fine;
   std::vector<int32_t> fine_page_offset;      // [S * fine + 1]
   std::vector<int64_t> fine_tokens;           // [S * fine]
   std::vector<int32_t> fine_tail_slot;        // [S * fine]
 
+  // Response suffix (blocks appended behind the prefix; they live in pool pages that the
+  // prefix does not map).  Device arrays are sized for the reserved capacity.
+  int32_t suffix_cap_pages, suffix_cap_blocks;
+  std::vector<ls::SuffixBlock> suffix_blocks;
+  std::vector<int32_t> suffix_phys;           // physical page of every suffix page slot in use
+  int64_t suffix_tokens;
+  float* dk_grad;                              // caller-owned fp32 gradient pages (may be NULL)
+  float* dv_grad;
+  uint64_t generation;                         // bumped by every append / pop
+
   bool on_device;
   int device;
-  int32_t* d_shard_phys_pages;   // [Np]
-  int32_t* d_shard_page_offset;  // [S * fine + 1]  (sub-shards)
-  int32_t* d_shard_tail_slot;    // [S * fine]
-  int64_t* d_shard_tokens;       // [S * fine]
+  int32_t* d_part_pages;         // [Np + suffix_cap_pages] physical ids: prefix (shard-local order), then suffix slots
+  int32_t* d_part_page_offset;   // [S * fine + suffix_cap_blocks + 1]
+  int32_t* d_part_tail_slot;     // [S * fine + suffix_cap_blocks]
+  int64_t* d_part_tokens;        // [S * fine + suffix_cap_blocks]
   int32_t* d_page_table;         // [Np]
-  ls::PoolMaps k_maps, v_maps;
+
+  mutable std::mutex map_mutex;
+  mutable std::vector<ls::PoolMapEntry> map_cache;
+
+  int prefix_parts() const { return desc.num_shards * fine; }
+  int num_parts() const { return prefix_parts() + (int)suffix_blocks.size(); }   // parts the kernels walk before the response block
 };
 
 namespace ls {
-
-// Encodes a rank-4 bf16 tensor map (d, token, head, page) with a 128-byte swizzle and a
-// box of 64 channels x box_tok tokens.  Strides in elements.  Returns LS_OK or an error.
-ls_status_t encode_map(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok,
-                       int64_t dim_head, int64_t dim_page, int64_t stride_tok, int64_t stride_head,
-                       int64_t stride_page, int box_tok);
 
 // One-shot event pairs armed by ls_profile_arm_events.
 struct ProfileSlot {
@@ -77,6 +104,10 @@ inline void profile_end(int k, cudaStream_t st) {
   g_profile[k].start = g_profile[k].stop = nullptr;
 }
 
+// Diagnostic builds: device buffer of int64 words that CTA 0 of the big kernels fills with
+// per-role cycle counts (NULL = off).  Set through ls_debug_timing_buffer (LS_TIMING builds only).
+extern long long* g_timing_buffer;
+
 // Rank-5 view (64 channels, token, channel group, head, page) with a box of
 // 64 x box_tok x box_groups: one TMA instruction fills box_groups swizzled slabs.
 ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok, int64_t dim_head,
@@ -88,13 +119,30 @@ ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64
 ls_status_t encode_map_rows(CUtensorMap* out, const void* base, int64_t dim_d, int64_t R, int64_t heads,
                             int box_tok, int box_heads);
 
-// The pool's K (which = 0) or V (which = 1) map for the given box; tail = bounded to the valid
-// tokens of the partially filled last logical page.
-ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
-                             bool tail);
+// The pool's K (which = 0) or V (which = 1) map for the given box, from the handle's cache
+// (encoded on first use; the combinations the kernels of this shape use are encoded by
+// ls_prefix_pages_build).
+ls_status_t pool_map(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups, bool tail);
+
+// LS_OK when the handle is usable by a compute call on the current device with these
+// parameters: device-resident, built on the current device, generation as the caller expects.
+ls_status_t check_handle(const ls_pages* h, const ls_attn_params_t* prm);
+
+// Sets the dynamic shared-memory limit of a kernel once per device.
+template <typename K>
+inline ls_status_t configure_smem(K kernel, int bytes, bool (&done)[64]) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LS_ERR_CUDA;
+  if (!done[dev]) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+      return LS_ERR_CUDA;
+    done[dev] = true;
+  }
+  return LS_OK;
+}
 
 // Backward of the shared-latent 576/512 shape (ls_bwd_mla.cu): fills dq_part (fp32, unscaled,
-// [(S+1), R, Hq, 576]; with dq_resp_only just the response block's partial, [R, Hq, 576]) and
+// [(parts+1), R, Hq, 576]; with dq_resp_only just the response block's partial, [R, Hq, 576]) and
 // the bf16 dk_resp / dv_resp.
 ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
@@ -105,13 +153,11 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
 ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
                        const float* lse, const float* delta, const float* dq_resp, void* dq, int32_t* status_dev,
                        cudaStream_t cs);
-// True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix, LS_MLA_DQ != 0).
+// True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix).
 bool mla_dq_fast(const ls_pages* h);
 
-// Folds `fine` consecutive sub-shard partials into each of `groups` shard partials.
-ls_status_t group_merge(int groups, int fine, int64_t rows, int dv, const float* in_o, const float* in_lse,
-                        float* out_o, float* out_lse, cudaStream_t st);
-
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int pg_shift_of(int page_size) { return page_size == 64 ? 6 : page_size == 128 ? 7 : page_size == 256 ? 8 : 9; }
 
 }  // namespace ls

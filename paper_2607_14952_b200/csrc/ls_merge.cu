@@ -14,7 +14,8 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_kernel(int num_parts, 
                                                                  const float* __restrict__ lse_part,
                                                                  __nv_bfloat16* __restrict__ o_bf16,
                                                                  float* __restrict__ o_f32,
-                                                                 float* __restrict__ lse_out) {
+                                                                 float* __restrict__ lse_out,
+                                                                 int32_t* __restrict__ status) {
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -50,60 +51,19 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_kernel(int num_parts, 
       *reinterpret_cast<uint2*>(o_bf16 + row * dv + c) = pk;
     }
   }
-  if (lane == 0) lse_out[row] = a > 0.f ? m_safe + logf(a) : -INFINITY;
-}
-
-// Folds `fine` consecutive sub-shard partials into one shard partial (same identity; output
-// stays fp32 and normalised, an all-empty group gives l = -inf, o = 0).  grid = (rows/8, groups).
-__global__ void __launch_bounds__(kMergeWarps * 32) group_merge_kernel(int fine, int64_t rows, int dv,
-                                                                       const float* __restrict__ in_o,
-                                                                       const float* __restrict__ in_lse,
-                                                                       float* __restrict__ out_o,
-                                                                       float* __restrict__ out_lse) {
-  const int lane = threadIdx.x & 31;
-  const int64_t row = (int64_t)blockIdx.x * kMergeWarps + (threadIdx.x >> 5);
-  if (row >= rows) return;
-  const int64_t g0 = (int64_t)blockIdx.y * fine;
-  float m = -INFINITY;
-  for (int r = lane; r < fine; r += 32) m = fmaxf(m, in_lse[(g0 + r) * rows + row]);
-  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-  const float m_safe = (m == -INFINITY) ? 0.f : m;
-  float a = 0.f;
-  for (int r = lane; r < fine; r += 32) a += expf(in_lse[(g0 + r) * rows + row] - m_safe);
-  for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-  const float inv_a = a > 0.f ? 1.f / a : 0.f;
-  for (int c = lane * 4; c < dv; c += 128) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int r = 0; r < fine; ++r) {
-      const float w = expf(in_lse[(g0 + r) * rows + row] - m_safe);
-      if (w == 0.f) continue;
-      const float4 v = *reinterpret_cast<const float4*>(in_o + ((g0 + r) * rows + row) * dv + c);
-      acc.x = fmaf(w, v.x, acc.x);
-      acc.y = fmaf(w, v.y, acc.y);
-      acc.z = fmaf(w, v.z, acc.z);
-      acc.w = fmaf(w, v.w, acc.w);
-    }
-    acc.x *= inv_a;
-    acc.y *= inv_a;
-    acc.z *= inv_a;
-    acc.w *= inv_a;
-    *reinterpret_cast<float4*>(out_o + ((int64_t)blockIdx.y * rows + row) * dv + c) = acc;
+  if (lane == 0) {
+    // a = 0 with m = -inf is the all-empty row (l = -inf); NaN or +inf can only come from non-finite inputs
+    const float l = (a > 0.f || a != a) ? m_safe + logf(a) : -INFINITY;
+    lse_out[row] = l;
+    if (status && (l != l || l == INFINITY)) atomicExch(status, (int)LS_ERR_NONFINITE);
   }
-  if (lane == 0) out_lse[(int64_t)blockIdx.y * rows + row] = a > 0.f ? m_safe + logf(a) : -INFINITY;
-}
-
-ls_status_t group_merge(int groups, int fine, int64_t rows, int dv, const float* in_o, const float* in_lse,
-                        float* out_o, float* out_lse, cudaStream_t st) {
-  if (groups <= 0 || rows <= 0) return LS_OK;
-  dim3 grid((unsigned)((rows + kMergeWarps - 1) / kMergeWarps), (unsigned)groups);
-  group_merge_kernel<<<grid, kMergeWarps * 32, 0, st>>>(fine, rows, dv, in_o, in_lse, out_o, out_lse);
-  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
 }  // namespace ls
 
 extern "C" ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim_v, const float* o_part,
-                                    const float* lse_part, void* o_bf16, float* o_f32, float* lse, void* stream) {
+                                    const float* lse_part, void* o_bf16, float* o_f32, float* lse,
+                                    int32_t* status_dev, void* stream) {
   if (num_parts < 1 || rows < 0 || dim_v < 4 || dim_v % 4 != 0) return LS_ERR_INVALID_ARG;
   if (!o_part || !lse_part || !lse) return LS_ERR_INVALID_ARG;
   if (!ls::aligned16(o_part) || (o_f32 && !ls::aligned16(o_f32)) || (o_bf16 && !ls::aligned16(o_bf16)))
@@ -112,6 +72,6 @@ extern "C" ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim
   const int64_t blocks = (rows + ls::kMergeWarps - 1) / ls::kMergeWarps;
   if (blocks > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   ls::merge_kernel<<<(int)blocks, ls::kMergeWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(
-      num_parts, rows, dim_v, o_part, lse_part, static_cast<__nv_bfloat16*>(o_bf16), o_f32, lse);
+      num_parts, rows, dim_v, o_part, lse_part, static_cast<__nv_bfloat16*>(o_bf16), o_f32, lse, status_dev);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

@@ -3,7 +3,6 @@
 // Eq. glm-tr-zigzag-pages), upload of the plan, TMA descriptors of the page pool, and
 // the integrity checksum used between replays.
 #include <algorithm>
-#include <cstdlib>
 #include <mutex>
 #include <new>
 
@@ -28,23 +27,6 @@ static EncodeTiledFn encode_fn() {
       fn = reinterpret_cast<EncodeTiledFn>(p);
   });
   return fn;
-}
-
-ls_status_t encode_map(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok,
-                       int64_t dim_head, int64_t dim_page, int64_t stride_tok, int64_t stride_head,
-                       int64_t stride_page, int box_tok) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return LS_ERR_CUDA;
-  if (!aligned16(base)) return LS_ERR_ALIGNMENT;
-  if ((stride_tok * 2) % 16 || (stride_head * 2) % 16 || (stride_page * 2) % 16) return LS_ERR_ALIGNMENT;
-  cuuint64_t dims[4] = {(cuuint64_t)dim_d, (cuuint64_t)dim_tok, (cuuint64_t)dim_head, (cuuint64_t)dim_page};
-  cuuint64_t strides[3] = {(cuuint64_t)stride_tok * 2, (cuuint64_t)stride_head * 2, (cuuint64_t)stride_page * 2};
-  cuuint32_t box[4] = {64, (cuuint32_t)box_tok, 1, 1};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? LS_OK : LS_ERR_CUDA;
 }
 
 ls_status_t encode_map5(CUtensorMap* out, const void* base, int64_t dim_d, int64_t dim_tok, int64_t dim_head,
@@ -82,8 +64,8 @@ ls_status_t encode_map_rows(CUtensorMap* out, const void* base, int64_t dim_d, i
   return r == CUDA_SUCCESS ? LS_OK : LS_ERR_CUDA;
 }
 
-ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
-                             bool tail) {
+static ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups,
+                                    bool tail) {
   const ls_pages_desc_t& d = h->desc;
   const bool v = which == 1;
   const bool alias = v && d.v_aliases_k;
@@ -95,6 +77,35 @@ ls_status_t encode_pool_map5(CUtensorMap* out, const ls_pages* h, int which, int
   const int64_t tok = tail && h->last_valid > 0 ? h->last_valid : d.page_size;
   return encode_map5(out, base, dim, tok, d.num_kv_heads, std::max<int64_t>(d.num_phys_pages, 1), s_tok, s_head,
                      s_page, std::min<int>(box_tok, d.page_size), box_groups);
+}
+
+ls_status_t pool_map(CUtensorMap* out, const ls_pages* h, int which, int box_tok, int box_groups, bool tail) {
+  std::lock_guard<std::mutex> lock(h->map_mutex);
+  for (const PoolMapEntry& e : h->map_cache)
+    if (e.which == which && e.box_tok == box_tok && e.box_groups == box_groups && e.tail == (int)tail) {
+      *out = e.map;
+      return LS_OK;
+    }
+  PoolMapEntry e;
+  e.which = which;
+  e.box_tok = box_tok;
+  e.box_groups = box_groups;
+  e.tail = tail;
+  const ls_status_t st = encode_pool_map5(&e.map, h, which, box_tok, box_groups, tail);
+  if (st != LS_OK) return st;
+  h->map_cache.push_back(e);
+  *out = e.map;
+  return LS_OK;
+}
+
+ls_status_t check_handle(const ls_pages* h, const ls_attn_params_t* prm) {
+  if (!h || !prm) return LS_ERR_INVALID_ARG;
+  if (!h->on_device) return LS_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LS_ERR_CUDA;
+  if (dev != h->device) return LS_ERR_STALE;
+  if (prm->generation != 0 && prm->generation != h->generation) return LS_ERR_STALE;
+  return LS_OK;
 }
 
 static void even_chunks(int64_t n, int64_t parts, std::vector<int64_t>& bounds) {
@@ -116,14 +127,40 @@ static cudaError_t upload(T** dst, const std::vector<T>& src) {
   return e;
 }
 
+static void free_part_arrays(ls_pages* h) {
+  cudaFree(h->d_part_pages);
+  cudaFree(h->d_part_page_offset);
+  cudaFree(h->d_part_tail_slot);
+  cudaFree(h->d_part_tokens);
+  h->d_part_pages = h->d_part_page_offset = h->d_part_tail_slot = nullptr;
+  h->d_part_tokens = nullptr;
+}
+
 static void free_device(ls_pages* h) {
-  cudaFree(h->d_shard_phys_pages);
-  cudaFree(h->d_shard_page_offset);
-  cudaFree(h->d_shard_tail_slot);
-  cudaFree(h->d_shard_tokens);
+  free_part_arrays(h);
   cudaFree(h->d_page_table);
-  h->d_shard_phys_pages = h->d_shard_page_offset = h->d_shard_tail_slot = h->d_page_table = nullptr;
-  h->d_shard_tokens = nullptr;
+  h->d_page_table = nullptr;
+}
+
+// (Re)creates the device arrays that describe the parts the kernels walk -- prefix sub-shards,
+// then one part per suffix block -- with room for the reserved suffix capacity.
+static cudaError_t upload_part_arrays(ls_pages* h) {
+  const int64_t Np = h->num_logical_pages;
+  const int np = h->prefix_parts();
+  std::vector<int32_t> pages(h->shard_phys_pages);
+  pages.resize(Np + h->suffix_cap_pages, 0);
+  std::vector<int32_t> off(h->fine_page_offset);
+  off.resize(np + h->suffix_cap_blocks + 1, (int32_t)Np);
+  std::vector<int32_t> tail(h->fine_tail_slot);
+  tail.resize(np + h->suffix_cap_blocks, -1);
+  std::vector<int64_t> toks(h->fine_tokens);
+  toks.resize(np + h->suffix_cap_blocks, 0);
+  free_part_arrays(h);
+  cudaError_t e = upload(&h->d_part_pages, pages);
+  if (e == cudaSuccess) e = upload(&h->d_part_page_offset, off);
+  if (e == cudaSuccess) e = upload(&h->d_part_tail_slot, tail);
+  if (e == cudaSuccess) e = upload(&h->d_part_tokens, toks);
+  return e;
 }
 
 }  // namespace ls
@@ -151,8 +188,12 @@ extern "C" ls_status_t ls_prefix_pages_build(const ls_pages_desc_t* d, const int
   h->last_valid = d->prefix_len == 0 ? 0 : (int32_t)(d->prefix_len - (Np - 1) * pg);
   h->on_device = false;
   h->device = -1;
-  h->d_shard_phys_pages = h->d_shard_page_offset = h->d_shard_tail_slot = h->d_page_table = nullptr;
-  h->d_shard_tokens = nullptr;
+  h->d_part_pages = h->d_part_page_offset = h->d_part_tail_slot = h->d_page_table = nullptr;
+  h->d_part_tokens = nullptr;
+  h->suffix_cap_pages = h->suffix_cap_blocks = 0;
+  h->suffix_tokens = 0;
+  h->dk_grad = h->dv_grad = nullptr;
+  h->generation = 1;
 
   // page table: one-to-one into the pool
   h->page_table.resize(Np);
@@ -207,13 +248,14 @@ extern "C" ls_status_t ls_prefix_pages_build(const ls_pages_desc_t* d, const int
     h->shard_tokens[s] = tokens;
   }
 
-  // sub-shards for the kernels: aim at <= 32 MB of K+V per (KV head, sub-shard)
+  // sub-shards for the kernels: aim at <= stream_budget_kib (default 32 MB) of K+V per
+  // (KV head, sub-shard), at most 16 per shard
   {
     int64_t max_tokens = 0;
     for (int s = 0; s < S; ++s) max_tokens = std::max(max_tokens, h->shard_tokens[s]);
     const int64_t bytes_per_tok = (int64_t)(d->dim_k + (d->v_aliases_k ? 0 : d->dim_v)) * 2;
-    int64_t fine = (max_tokens * bytes_per_tok + (32ll << 20) - 1) / (32ll << 20);
-    if (const char* e = getenv("LS_SUBSPLIT")) fine = atoi(e);
+    const int64_t budget = (d->stream_budget_kib > 0 ? (int64_t)d->stream_budget_kib : 32768ll) << 10;
+    int64_t fine = (max_tokens * bytes_per_tok + budget - 1) / budget;
     fine = std::max<int64_t>(1, std::min<int64_t>(fine, 16));
     h->fine = (int32_t)fine;
     h->fine_page_offset.assign(S * fine + 1, 0);
@@ -244,9 +286,6 @@ extern "C" ls_status_t ls_prefix_pages_build(const ls_pages_desc_t* d, const int
   }
 
   const void* vbase = d->v_aliases_k ? d->k_pool : d->v_pool;
-  int64_t vs_page = d->v_aliases_k ? d->k_stride_page : d->v_stride_page;
-  int64_t vs_tok = d->v_aliases_k ? d->k_stride_tok : d->v_stride_tok;
-  int64_t vs_head = d->v_aliases_k ? d->k_stride_head : d->v_stride_head;
   if (!vbase) {
     delete h;
     return LS_ERR_INVALID_ARG;
@@ -255,33 +294,34 @@ extern "C" ls_status_t ls_prefix_pages_build(const ls_pages_desc_t* d, const int
     delete h;
     return LS_ERR_ALIGNMENT;
   }
-  const int64_t nphys = std::max<int64_t>(d->num_phys_pages, 1);
-  for (int bi = 0; bi < ls::kNumBoxSizes; ++bi) {
-    int bt = ls::kBoxTok[bi];
-    if (bt > pg) bt = (int)pg;
-    int64_t tail_tok = h->last_valid > 0 ? h->last_valid : pg;
-    ls_status_t st = ls::encode_map(&h->k_maps.full[bi], d->k_pool, d->dim_k, pg, d->num_kv_heads, nphys,
-                                    d->k_stride_tok, d->k_stride_head, d->k_stride_page, bt);
-    if (st == LS_OK)
-      st = ls::encode_map(&h->k_maps.tail[bi], d->k_pool, d->dim_k, tail_tok, d->num_kv_heads, nphys,
-                          d->k_stride_tok, d->k_stride_head, d->k_stride_page, bt);
-    if (st == LS_OK)
-      st = ls::encode_map(&h->v_maps.full[bi], vbase, d->dim_v, pg, d->num_kv_heads, nphys, vs_tok, vs_head,
-                          vs_page, bt);
-    if (st == LS_OK)
-      st = ls::encode_map(&h->v_maps.tail[bi], vbase, d->dim_v, tail_tok, d->num_kv_heads, nphys, vs_tok,
-                          vs_head, vs_page, bt);
-    if (st != LS_OK) {
-      delete h;
-      return st;
+  // the pool's TMA descriptors for every box the kernels of this shape use
+  {
+    const bool mla = d->dim_k == 576;
+    const bool small_pages = pg == 64;
+    struct Box { int which, tok, groups; };
+    std::vector<Box> boxes;
+    if (mla) {
+      boxes = {{0, small_pages ? 64 : 128, 1}, {1, 32, 4}, {0, 64, 1}, {0, 64, 2}, {1, 64, 1}};
+    } else if (d->dim_k == 256) {
+      boxes = {{0, 64, 2}, {1, 64, 2}, {0, small_pages ? 64 : 128, 1}, {1, small_pages ? 64 : 128, 1},
+               {0, small_pages ? 64 : 128, small_pages ? 1 : 2}, {1, 64, 4}, {1, small_pages ? 64 : 128, small_pages ? 1 : 2}};
+    } else {
+      boxes = {{0, small_pages ? 64 : 128, 1}, {1, 64, 2}, {0, 64, 2}, {1, small_pages ? 64 : 128, 1},
+               {0, small_pages ? 64 : 128, small_pages ? 1 : 2}, {1, small_pages ? 64 : 128, small_pages ? 1 : 2}};
     }
+    CUtensorMap tmp;
+    for (const Box& b : boxes)
+      for (int tail = 0; tail < 2; ++tail) {
+        const ls_status_t st = ls::pool_map(&tmp, h, b.which, b.tok, b.groups, tail != 0);
+        if (st != LS_OK) {
+          delete h;
+          return st;
+        }
+      }
   }
 
   cudaError_t e = cudaGetDevice(&h->device);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_phys_pages, h->shard_phys_pages);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_page_offset, h->fine_page_offset);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_tail_slot, h->fine_tail_slot);
-  if (e == cudaSuccess) e = ls::upload(&h->d_shard_tokens, h->fine_tokens);
+  if (e == cudaSuccess) e = ls::upload_part_arrays(h);
   if (e == cudaSuccess) e = ls::upload(&h->d_page_table, h->page_table);
   if (e != cudaSuccess) {
     ls::free_device(h);
@@ -351,6 +391,9 @@ extern "C" ls_status_t ls_prefix_pages_checksum(const ls_pages_t* h, uint64_t* s
                                                 void* stream) {
   if (!h || !scratch_dev || !out) return LS_ERR_INVALID_ARG;
   if (!h->on_device) return LS_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LS_ERR_CUDA;
+  if (dev != h->device) return LS_ERR_STALE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ls_pages_desc_t& d = h->desc;
   if (cudaMemsetAsync(scratch_dev, 0, sizeof(uint64_t), st) != cudaSuccess) return LS_ERR_CUDA;
@@ -372,9 +415,145 @@ extern "C" ls_status_t ls_prefix_pages_checksum(const ls_pages_t* h, uint64_t* s
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------------------------
+// Response suffix as temporary pages (Sec. "Four-Block Response Replay"): append copies one
+// block of response K/V into pool pages the prefix does not map, pop unmaps the last block.
+// ---------------------------------------------------------------------------------
+namespace ls {
+
+// Copies a dense [n, heads, dim] bf16 block into pool pages (16 bytes per thread step) and
+// zero-fills the rest of the last page.  slot_pages: physical ids of the block's pages.
+__global__ void suffix_copy_kernel(const uint4* __restrict__ src, uint16_t* __restrict__ pool,
+                                   const int32_t* __restrict__ slot_pages, int n_tokens, int num_pages, int pg,
+                                   int heads, int dim, int64_t s_page, int64_t s_tok, int64_t s_head) {
+  const int vec_per_tok = heads * dim / 8;
+  const int64_t total = (int64_t)num_pages * pg * vec_per_tok;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t tok = i / vec_per_tok;
+    const int r = (int)(i % vec_per_tok);
+    const int hd = (r * 8) / dim, c = (r * 8) % dim;
+    const uint4 v = tok < n_tokens ? src[i] : make_uint4(0u, 0u, 0u, 0u);
+    uint16_t* dst = pool + (int64_t)slot_pages[tok / pg] * s_page + (tok % pg) * s_tok + (int64_t)hd * s_head + c;
+    *reinterpret_cast<uint4*>(dst) = v;
+  }
+}
+
+}  // namespace ls
+
+extern "C" ls_status_t ls_suffix_pages_reserve(ls_pages_t* h, int32_t max_blocks, int32_t max_pages, float* dk_grad,
+                                               float* dv_grad) {
+  if (!h || max_blocks < 0 || max_pages < 0 || max_blocks > 4096) return LS_ERR_INVALID_ARG;
+  if (!h->on_device || !h->suffix_blocks.empty()) return LS_ERR_INVALID_ARG;
+  if ((dk_grad == nullptr) != (dv_grad == nullptr)) return LS_ERR_INVALID_ARG;
+  if (h->desc.dim_k == 576) return LS_ERR_UNSUPPORTED_SHAPE;
+  if (!ls::aligned16(dk_grad) || !ls::aligned16(dv_grad)) return LS_ERR_ALIGNMENT;
+  if (h->num_logical_pages + max_pages > h->desc.num_phys_pages) return LS_ERR_INVALID_ARG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LS_ERR_CUDA;
+  if (dev != h->device) return LS_ERR_STALE;
+  h->suffix_cap_blocks = max_blocks;
+  h->suffix_cap_pages = max_pages;
+  h->dk_grad = dk_grad;
+  h->dv_grad = dv_grad;
+  if (cudaDeviceSynchronize() != cudaSuccess) return LS_ERR_CUDA;   // no kernel may still read the old arrays
+  if (ls::upload_part_arrays(h) != cudaSuccess) return LS_ERR_CUDA;
+  ++h->generation;
+  return LS_OK;
+}
+
+extern "C" ls_status_t ls_suffix_pages_append(ls_pages_t* h, int32_t n_tokens, const int32_t* phys_pages,
+                                              const void* k_block, const void* v_block, void* stream) {
+  if (!h || n_tokens < 1 || !phys_pages || !k_block) return LS_ERR_INVALID_ARG;
+  if (!h->on_device) return LS_ERR_INVALID_ARG;
+  const ls_pages_desc_t& d = h->desc;
+  if (!d.v_aliases_k && !v_block) return LS_ERR_INVALID_ARG;
+  if (!ls::aligned16(k_block) || !ls::aligned16(v_block)) return LS_ERR_ALIGNMENT;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LS_ERR_CUDA;
+  if (dev != h->device) return LS_ERR_STALE;
+  const int pg = d.page_size;
+  const int n_pages = (n_tokens + pg - 1) / pg;
+  const int first_slot = (int)h->suffix_phys.size();
+  if ((int)h->suffix_blocks.size() + 1 > h->suffix_cap_blocks || first_slot + n_pages > h->suffix_cap_pages)
+    return LS_ERR_INVALID_ARG;
+  // the new pages must be free: in range, distinct, mapped neither by the prefix nor by the suffix
+  {
+    std::vector<uint8_t> used(d.num_phys_pages, 0);
+    for (int32_t p : h->page_table) used[p] = 1;
+    for (int32_t p : h->suffix_phys) used[p] = 1;
+    for (int i = 0; i < n_pages; ++i) {
+      const int64_t p = phys_pages[i];
+      if (p < 0 || p >= d.num_phys_pages || used[p]) return LS_ERR_BAD_PAGE_TABLE;
+      used[p] = 1;
+    }
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t Np = h->num_logical_pages;
+  const int part = h->prefix_parts() + (int)h->suffix_blocks.size();
+  for (int i = 0; i < n_pages; ++i) h->suffix_phys.push_back(phys_pages[i]);
+  ls::SuffixBlock blk;
+  blk.tokens = n_tokens;
+  blk.first_slot = first_slot;
+  blk.num_pages = n_pages;
+  h->suffix_blocks.push_back(blk);
+  h->suffix_tokens += n_tokens;
+  ++h->generation;
+  // device plan: the block is one more part behind the prefix parts (pageable host sources: the
+  // runtime stages them before returning, so the vectors may change afterwards)
+  const int32_t off_end = (int32_t)(Np + first_slot + n_pages);
+  const int64_t tokens64 = n_tokens;
+  cudaError_t e = cudaMemcpyAsync(h->d_part_pages + Np + first_slot, h->suffix_phys.data() + first_slot,
+                                  n_pages * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(h->d_part_page_offset + part + 1, &off_end, sizeof(int32_t), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(h->d_part_tokens + part, &tokens64, sizeof(int64_t), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return LS_ERR_CUDA;
+  const int32_t* slot_pages = h->d_part_pages + Np + first_slot;
+  const int blocks = (int)std::min<int64_t>(((int64_t)n_pages * pg * d.num_kv_heads * d.dim_k / 8 + 255) / 256, 148 * 8);
+  ls::suffix_copy_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(k_block),
+                                                const_cast<uint16_t*>(static_cast<const uint16_t*>(d.k_pool)),
+                                                slot_pages, n_tokens, n_pages, pg, d.num_kv_heads, d.dim_k,
+                                                d.k_stride_page, d.k_stride_tok, d.k_stride_head);
+  if (!d.v_aliases_k)
+    ls::suffix_copy_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(v_block),
+                                                  const_cast<uint16_t*>(static_cast<const uint16_t*>(d.v_pool)),
+                                                  slot_pages, n_tokens, n_pages, pg, d.num_kv_heads, d.dim_v,
+                                                  d.v_stride_page, d.v_stride_tok, d.v_stride_head);
+  if (h->dk_grad) {
+    const size_t per_page_k = (size_t)pg * d.num_kv_heads * d.dim_k * sizeof(float);
+    const size_t per_page_v = (size_t)pg * d.num_kv_heads * d.dim_v * sizeof(float);
+    e = cudaMemsetAsync(reinterpret_cast<char*>(h->dk_grad) + first_slot * per_page_k, 0, n_pages * per_page_k, st);
+    if (e == cudaSuccess)
+      e = cudaMemsetAsync(reinterpret_cast<char*>(h->dv_grad) + first_slot * per_page_v, 0, n_pages * per_page_v, st);
+    if (e != cudaSuccess) return LS_ERR_CUDA;
+  }
+  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
+extern "C" ls_status_t ls_suffix_pages_pop(ls_pages_t* h) {
+  if (!h || h->suffix_blocks.empty()) return LS_ERR_INVALID_ARG;
+  const ls::SuffixBlock blk = h->suffix_blocks.back();
+  h->suffix_blocks.pop_back();
+  h->suffix_phys.resize(blk.first_slot);
+  h->suffix_tokens -= blk.tokens;
+  ++h->generation;
+  return LS_OK;
+}
+
+extern "C" uint64_t ls_pages_generation(const ls_pages_t* h) { return h ? h->generation : 0; }
+
+extern "C" int64_t ls_suffix_pages_tokens(const ls_pages_t* h) { return h ? h->suffix_tokens : 0; }
+
 namespace ls {
 ProfileSlot g_profile[LS_KERNEL_COUNT] = {};
+long long* g_timing_buffer = nullptr;
 }
+
+#ifdef LS_TIMING
+// Diagnostic builds only: device buffer (>= 64 int64 words) for the kernels' cycle counters.
+extern "C" void ls_debug_timing_buffer(void* dev_buffer) { ls::g_timing_buffer = static_cast<long long*>(dev_buffer); }
+#endif
 
 extern "C" ls_status_t ls_profile_arm_events(int kernel, void* start_event, void* stop_event) {
   if (kernel < 0 || kernel >= LS_KERNEL_COUNT) return LS_ERR_INVALID_ARG;

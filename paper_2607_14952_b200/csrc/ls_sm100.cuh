@@ -86,18 +86,74 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   return mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetNs, kWaitHintNs);
 }
 
-// ------------------------------------------------------------------ TMA
-// Loads one box of a rank-4 tensor map (d, token, head, page) into shared memory and
-// signals `bar` with the byte count.  c0 * 2 bytes must be a multiple of 16.
-__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0,
-                                            int c1, int c2, int c3) {
+// ------------------------------------------------------------------ named barriers
+// Barrier `id` over `nthreads` threads (whole warps) that also ANDs a predicate over them, so
+// a group of threads can agree on "everyone is still fine" at a point all of them reach.
+// A thread must never leave a loop that contains a named barrier on its own flag: it votes
+// here and all leave together.
+__device__ __forceinline__ bool bar_and(int id, int nthreads, bool pred) {
+  uint32_t r;
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(smem_u32(smem_dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %3, 0;\n\t"
+      "barrier.red.and.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(nthreads), "r"((uint32_t)pred)
       : "memory");
+  return r != 0;
 }
-// Rank-5 variant: (64 channels, token, 64-channel group, head, page).  One instruction
+__device__ __forceinline__ void bar_sync(int id, int nthreads) {
+  asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// ------------------------------------------------------------------ ordered hand-over between CTAs
+// Work items of one launch that fold their result into a shared running value (the partials
+// of one output row tile) do so in a fixed order, so the sum order -- and with it every bit of
+// the result -- does not depend on scheduling.  Link k of a chain waits until the chain's
+// counter reads k, updates the running value, and publishes k + 1.  Work items are handed out
+// by a ticket counter, so every item a CTA may wait for has already been started by some CTA
+// and no wait depends on an item that is not running.  The wait is bounded like every other
+// device-side wait; a CTA that gives up raises the launch-wide abort word, which ends every
+// other chain wait at once.
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ int ld_relaxed_gpu(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_gpu(int* p, int v) {
+  asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// ctl[0] ticket, ctl[1] launch-wide abort word
+__device__ __forceinline__ bool chain_wait(const int* counter, int want, const int* ctl,
+                                           volatile int* abort_flag) {
+  if (ld_acquire_gpu(counter) >= want) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+    if (ld_acquire_gpu(counter) >= want) return true;
+    if (*abort_flag || ld_relaxed_gpu(ctl + 1) != 0) return false;
+    if (globaltimer_ns() - t0 > kWaitBudgetNs) {
+      *abort_flag = 1;
+      return false;
+    }
+    __nanosleep(256);
+  }
+}
+// Called by ONE thread after a CTA-level barrier that all writers of the running value passed.
+__device__ __forceinline__ void chain_publish(int* counter, int value) {
+  __threadfence();
+  st_release_gpu(counter, value);
+}
+
+// ------------------------------------------------------------------ TMA
+// Rank-5 tile load: (64 channels, token, 64-channel group, head, page).  One instruction
 // fills several 128-byte-swizzled slabs (one per channel group) back to back.
 __device__ __forceinline__ void tma_load_5d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0,
                                             int c1, int c2, int c3, int c4) {
@@ -181,6 +237,11 @@ __device__ __forceinline__ uint32_t mapa_u32(uint32_t smem_addr, uint32_t rank) 
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
+}
+__device__ __forceinline__ uint32_t ld_shared_cluster_u32(uint32_t cluster_addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+  return v;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");

@@ -26,7 +26,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layout_matches_header():
     assert C.sizeof(B.ls_pages_desc_t) == 8 + 8 * 4 + 8 + 8 * 2 + 8 * 6
-    assert C.sizeof(B.ls_attn_params_t) == 16
+    assert C.sizeof(B.ls_attn_params_t) == 24
 
 
 POLICIES = [(B.LS_SHARD_CONTIGUOUS, op.CONTIGUOUS), (B.LS_SHARD_CYCLIC, op.CYCLIC), (B.LS_SHARD_ZIGZAG, op.ZIGZAG)]
@@ -105,19 +105,38 @@ def test_error_paths_before_any_launch():
     assert B.lib().ls_status_string(B.LS_ERR_TIMEOUT) != b"unknown status"
 
 
-def test_backward_workspace_sizes(monkeypatch):
-    # per-partial fp32 dQ sums + Delta in general; the aliased 576/512 shape sums the prefix
-    # partials in its accumulator and keeps only the response block's partial
+def _ctl(chains):
+    return ((4 + chains) * 4 + 15) // 16 * 16
+
+
+def test_workspace_sizes():
+    # backward: Delta, the hand-over counters (one per Q tile) and ONE fp32 running dQ, whatever
+    # the number of shards; the 576/512 shape with a V pool of its own keeps one dQ per partial
     R, Hq = 96, 8
     rows = R * Hq
+    head = rows * 4 + _ctl(Hq * 1)
     plain = B.ls_prefix_pages_build(256 * 12, 256, 3, 2, 256, 256, 12)
-    assert B.ls_replay_attn_workspace_bytes(plain, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == (3 + 1) * rows * 256 * 4 + rows * 4
+    assert B.ls_replay_attn_workspace_bytes(plain, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == head + rows * 256 * 4
     assert B.ls_replay_attn_workspace_bytes(plain, R, Hq, 0.0625, B.LS_WORKSPACE_FWD) == 0
+    assert B.ls_replay_attn_workspace_bytes(plain, R, Hq, 0.0625, B.LS_WORKSPACE_FWD_MERGED) == _ctl(2 * 4)
+    many = B.ls_prefix_pages_build(256 * 12, 256, 12, 2, 256, 256, 12)
+    assert B.ls_replay_attn_workspace_bytes(many, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == head + rows * 256 * 4
+    # a tiny stream budget walks every shard as sub-ranges: the forward then needs its counters, nothing more
+    cut = B.ls_prefix_pages_build(256 * 12, 256, 3, 2, 256, 256, 12, stream_budget_kib=512)
+    assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_FWD) == _ctl(2 * 3 * 4)
+    assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == head + rows * 256 * 4
     mla = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=True)
-    monkeypatch.delenv("LS_MLA_DQ", raising=False)
-    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == rows * 576 * 4 + rows * 4
-    monkeypatch.setenv("LS_MLA_DQ", "0")
-    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == (4 + 1) * rows * 576 * 4 + rows * 4
-    monkeypatch.delenv("LS_MLA_DQ")
+    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + rows * 576 * 4
+    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_FWD_MERGED) == _ctl(Hq * 2) + rows * 4
+    sep = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=False)
+    assert B.ls_replay_attn_workspace_bytes(sep, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + (4 + 1) * rows * 576 * 4
     empty = B.ls_prefix_pages_build(0, 64, 1, 1, 576, 512, 1, v_aliases_k=True)
-    assert B.ls_replay_attn_workspace_bytes(empty, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == (1 + 1) * rows * 576 * 4 + rows * 4
+    assert B.ls_replay_attn_workspace_bytes(empty, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + (1 + 1) * rows * 576 * 4
+
+
+def test_suffix_bookkeeping_needs_a_device_handle():
+    # a host-only plan has no pool to append pages to
+    plan = B.ls_prefix_pages_build(256, 64, 2, 1, 128, 128, 8)
+    assert B.ls_pages_generation(plan) == 1 and B.ls_suffix_pages_tokens(plan) == 0
+    assert status_of(lambda: B.ls_suffix_pages_reserve(plan, 2, 4)) == B.LS_ERR_INVALID_ARG
+    assert status_of(lambda: B.ls_suffix_pages_pop(plan)) == B.LS_ERR_INVALID_ARG

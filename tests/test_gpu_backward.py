@@ -98,45 +98,60 @@ def test_backward_split_count_does_not_change_dq():
         assert (o[0].float() - outs[0][0].float()).abs().max() < 2e-3
 
 
-@pytest.mark.parametrize("fine", [2, 3, 5])
-def test_sub_split_shards_forward_and_backward(fine, monkeypatch):
-    # shards are cut into sub-shards for the kernels (a locality measure for long prefixes) and folded
-    # back into the S partials of the ABI; force it on small cases, including sub-shards left empty
-    monkeypatch.setenv("LS_SUBSPLIT", str(fine))
+@pytest.mark.parametrize("budget_kib", [96, 256, 1024])
+def test_sub_split_shards_forward_and_backward(budget_kib):
+    # long shards are walked as consecutive sub-ranges (a locality measure for long prefixes) whose
+    # results fold back, in order, into the S partials of the ABI; a tiny stream budget forces that
+    # on small cases, including sub-ranges left empty
     for cfg in (small("sub_pg64", P=64 * 13 + 7, page_size=64, num_shards=4, R=130),
                 small("sub_pg256", P=256 * 9 + 100, page_size=256, num_shards=2, R=200, Hq=6, Hkv=2),
                 small("sub_d128", Dk=128, Dv=128, P=128 * 11, page_size=128, num_shards=3, R=96, Hq=8, Hkv=2),
                 small("sub_mla", Dk=576, Dv=512, v_aliases_k=True, Hq=4, Hkv=1, P=64 * 9 + 3, page_size=64,
                       num_shards=2, R=70)):
-        case = parity.Case(cfg)
+        case = parity.Case(cfg, stream_budget_kib=budget_kib)
         fw = parity.check_forward(case, per_shard=True)
         parity.check_backward(case, fw)
 
 
-@pytest.mark.parametrize("fwd_pair,bwd_pair", [("0", "0"), ("0", "2"), ("1", "2")])
-def test_alternative_kernels_stay_correct(fwd_pair, bwd_pair, monkeypatch):
-    # head dim 256 defaults to the CTA-pair forward and the 256-key-tile pair dQ kernel; the
-    # single-CTA forward / dQ kernels and the 128-key-tile pair kernel remain selectable
-    monkeypatch.setenv("LS_FWD_PAIR", fwd_pair)
-    monkeypatch.setenv("LS_BWD_PAIR", bwd_pair)
-    for cfg in (small("alt_basic", P=2048 + 300, page_size=256, num_shards=3, R=200, Hq=6, Hkv=2),
-                small("alt_pg64", P=64 * 13 + 7, page_size=64, num_shards=4, R=130),
-                small("alt_short", P=3000, page_size=128, num_shards=5, R=5, Hq=6, Hkv=2)):
-        case = parity.Case(cfg)
-        fw = parity.check_forward(case, per_shard=True)
-        parity.check_backward(case, fw)
-
-
-@pytest.mark.parametrize("mla_dq", ["0", "1"])
-def test_shared_latent_dq_paths(mla_dq, monkeypatch):
+@pytest.mark.parametrize("aliased", [True, False])
+def test_shared_latent_dq_paths(aliased):
     # 576/512 pools whose V aliases K take the transposed dQ kernel that walks every partial in
-    # one accumulator (LS_MLA_DQ=1, the default); the per-partial kernel stays selectable.  Cases: ragged tail page, several heads per
-    # latent, more than one row tile per head, a response longer than one key tile.
-    monkeypatch.setenv("LS_MLA_DQ", mla_dq)
-    for cfg in (small("mla_t_pg64", Dk=576, Dv=512, v_aliases_k=True, Hq=8, Hkv=1, P=64 * 37 + 21, page_size=64,
+    # one accumulator; a 576/512 pool with a V tensor of its own takes the per-partial kernel.
+    # Cases: ragged tail page, several heads per latent, more than one row tile per head, a
+    # response longer than one key tile.
+    for cfg in (small("mla_t_pg64", Dk=576, Dv=512, v_aliases_k=aliased, Hq=8, Hkv=1, P=64 * 37 + 21, page_size=64,
                       num_shards=5, R=150),
-                small("mla_t_pg512", Dk=576, Dv=512, v_aliases_k=True, Hq=2, Hkv=1, P=512 * 5 + 300, page_size=512,
+                small("mla_t_pg512", Dk=576, Dv=512, v_aliases_k=aliased, Hq=2, Hkv=1, P=512 * 5 + 300, page_size=512,
                       num_shards=3, R=64)):
         case = parity.Case(cfg)
         fw = parity.check_forward(case, per_shard=True)
         parity.check_backward(case, fw)
+
+
+def test_shared_latent_dq_ignores_unmapped_pages():
+    # 64-token pages, an odd page count per shard (the last 128-key tile of a shard is half
+    # empty), a pool larger than the prefix whose unmapped pages -- physical page 0 among them --
+    # hold NaN patterns: nothing of them may reach dQ
+    cfg = small("mla_nan", Dk=576, Dv=512, v_aliases_k=True, Hq=4, Hkv=1, P=64 * 9, page_size=64, num_shards=3, R=96)
+    case = parity.Case(cfg, extra_phys_pages=3)
+    mapped = set(int(x) for x in case.table)
+    moved = None
+    if 0 in mapped:                                   # free physical page 0: move its logical page elsewhere
+        free = [p for p in range(case.k_pool.shape[0]) if p not in mapped]
+        lp = list(case.table).index(0)
+        case.k_pool[free[0]] = case.k_pool[0]
+        case.table[lp] = free[0]
+        moved = free[0]
+        case.pages.close()
+        case.pages = B.ls_prefix_pages_build(cfg.P, cfg.page_size, cfg.num_shards, cfg.Hkv, cfg.Dk, cfg.Dv,
+                                             case.k_pool.shape[0], page_table=case.table, k_pool=case.k_pool,
+                                             v_aliases_k=True)
+        case._host = {}
+    mapped = set(int(x) for x in case.table)
+    for p in range(case.k_pool.shape[0]):
+        if p not in mapped:
+            case.k_pool[p] = float("nan")
+    assert torch.isnan(case.k_pool[0]).all()
+    fw = parity.check_forward(case, per_shard=False)
+    bw = parity.check_backward(case, fw)
+    assert torch.isfinite(bw["dq"].float()).all()
