@@ -85,12 +85,69 @@ class Case:
         return oa.backward_rows(*args, W.bf16_bits(d_o[t_rows, heads]))
 
 
-def rel_gate(gpu, ref, d):
+    def oracle_forward_slabs(self, kv, t_rows, heads, q, k_resp, v_resp, slab=4096):
+        outs = [self.oracle_rows(kv, t_rows[lo:lo + slab], heads[lo:lo + slab], q, k_resp, v_resp)
+                for lo in range(0, len(t_rows), slab)]
+        return np.concatenate([x[0] for x in outs]), np.concatenate([x[1] for x in outs])
+
+    def oracle_backward_slabs(self, kv, t_rows, heads, q, k_resp, v_resp, d_o, slab=2048):
+        """backward_rows over many rows in slabs (bounds the host memory of the score matrices):
+        O, LSE, dQ per row concatenated, the dK / dV contributions summed."""
+        outs, dk, dv = [], 0.0, 0.0
+        for lo in range(0, len(t_rows), slab):
+            o, lse, dq, dk_p, dv_p = self.oracle_rows(kv, t_rows[lo:lo + slab], heads[lo:lo + slab], q, k_resp, v_resp, d_o)
+            outs.append((o, lse, dq))
+            dk, dv = dk + dk_p, dv + dv_p
+        return (np.concatenate([x[0] for x in outs]), np.concatenate([x[1] for x in outs]),
+                np.concatenate([x[2] for x in outs]), dk, dv)
+
+
+def dq_rounding_model(case, kv, t_rows, heads, q, k_resp, v_resp, d_o):
+    """Per-row size of the dQ error that the kernel's arithmetic cannot avoid, from oracle-side
+    quantities.  The kernel rounds ds_j = p_j (dp_j - Delta) to bf16 before the dQ product
+    (relative 2^-9 per element) and forms dp_j - Delta from two fp32 dot products of Dv terms,
+    one of them accumulated by the tensor core in Dv/16 steps that each truncate to fp32
+    (absolute ~ (Dv/16) 2^-23 (|dp_j| + |Delta|)); each key's error enters dQ times
+    scale * |k_j|.  Independent errors add in quadrature; the factor 4 covers the tail of that
+    sum.  This is what can exceed the plain relative gate when dQ is a near-cancelling sum over
+    keys of very unequal norm (needle keys, or a handful of visible keys)."""
+    cfg = case.cfg
+    kp, vp = case.host_pool(kv)
+    kr = W.bf16_bits(k_resp[:, kv:kv + 1])
+    vr = W.bf16_bits(v_resp[:, kv:kv + 1])
+    scale = float(np.float32(cfg.scale))
+    qr = W.bf16_bits(q[t_rows, heads])
+    o, lse, p = oa.forward_rows(qr, np.asarray(t_rows), 0, kp, vp, case.table, cfg.P, cfg.page_size, kr, vr, scale)
+    do = oa.widen(W.bf16_bits(d_o[t_rows, heads]))
+    pos = np.arange(cfg.P)
+    k_all = np.concatenate([oa.widen(kp[case.table[pos // cfg.page_size], pos % cfg.page_size, 0, :]),
+                            oa.widen(kr[:, 0, :])])
+    v_all = np.concatenate([oa.widen(vp[case.table[pos // cfg.page_size], pos % cfg.page_size, 0, :cfg.Dv]),
+                            oa.widen(vr[:, 0, :])])
+    dp = do @ v_all.T
+    delta = (do * o).sum(axis=1)
+    ds = p * (dp - delta[:, None])
+    knorm = np.linalg.norm(k_all, axis=1)
+    per_key = 2.0 ** -9 * np.abs(ds) + p * (cfg.Dv / 16) * 2.0 ** -23 * (np.abs(dp) + np.abs(delta)[:, None])
+    return 4.0 * scale * np.sqrt(((per_key * knorm[None, :]) ** 2).sum(axis=1))
+
+
+def needle_row_model(scale, k_needle, v_needle, do_row):
+    """dq_rounding_model for a row whose probability sits on one key (p = 1 there, ds = 0 by
+    cancellation): what is left of dp - Delta is the accumulation rounding of two dot products."""
+    dv = len(v_needle)
+    dp = abs(float(np.dot(do_row, v_needle)))
+    return 4.0 * scale * float(np.linalg.norm(k_needle)) * (dv / 16) * 2.0 ** -23 * 2.0 * dp
+
+
+def rel_gate(gpu, ref, d, extra=None):
     """Row-wise relative L2 gate; returns the worst ratio err / allowed (<= 1 passes)."""
     gpu = np.asarray(gpu, np.float64).reshape(-1, d)
     ref = np.asarray(ref, np.float64).reshape(-1, d)
     err = np.linalg.norm(gpu - ref, axis=1)
     allowed = REL * np.linalg.norm(ref, axis=1) + FLOOR * np.sqrt(d)
+    if extra is not None:
+        allowed = allowed + extra
     return float((err / allowed).max())
 
 
@@ -144,7 +201,7 @@ def check_forward(case, member=0, kv_groups=None, full=True, per_shard=True, ext
     report = {}
     for kv in (range(cfg.Hkv) if kv_groups is None else kv_groups):
         t_rows, heads = all_rows_of_group(cfg, kv) if full else sampled_rows(cfg, kv, extra=extra_rows)
-        o_ref, lse_ref = case.oracle_rows(kv, t_rows, heads, q, k_resp, v_resp)
+        o_ref, lse_ref = case.oracle_forward_slabs(kv, t_rows, heads, q, k_resp, v_resp)
         g_lse = f64(lse[t_rows, heads])
         g_o32 = f64(o_f32[t_rows, heads])
         g_o16 = f64(o_bf16[t_rows, heads])
@@ -190,9 +247,10 @@ def check_forward(case, member=0, kv_groups=None, full=True, per_shard=True, ext
                 lse_part=lse_part, o_bf16=o_bf16, report=report)
 
 
-def check_backward(case, fw, kv_groups=None, full=True, tail=16, extra_rows=(), strict_abs=False, rel_slack=1.0):
+def check_backward(case, fw, kv_groups=None, full=True, tail=16, extra_rows=(), strict_abs=False, dq_model=False):
     """Backward parity for dQ on the row set and for dK/dV on the response keys whose
-    contributing rows are all inside the set (all keys when full, the last `tail` otherwise)."""
+    contributing rows are all inside the set (all keys when full, the last `tail` otherwise).
+    dq_model adds dq_rounding_model's per-row term to the relative gate of dQ."""
     cfg = case.cfg
     q, k_resp, v_resp, d_o = fw["q"], fw["k_resp"], fw["v_resp"], fw["d_o"]
     dq, dk, dv = case.backward(q, k_resp, v_resp, fw["o_f32"], fw["lse"], d_o)
@@ -200,12 +258,12 @@ def check_backward(case, fw, kv_groups=None, full=True, tail=16, extra_rows=(), 
     report = {}
     for kv in (range(cfg.Hkv) if kv_groups is None else kv_groups):
         t_rows, heads = all_rows_of_group(cfg, kv) if full else sampled_rows(cfg, kv, tail=tail, extra=extra_rows)
-        _, _, dq_ref, dk_ref, dv_ref = case.oracle_rows(kv, t_rows, heads, q, k_resp, v_resp, d_o)
+        _, _, dq_ref, dk_ref, dv_ref = case.oracle_backward_slabs(kv, t_rows, heads, q, k_resp, v_resp, d_o)
         g_dq = f64(dq[t_rows, heads])
         assert np.isfinite(g_dq).all()
         e_dq = np.abs(g_dq - dq_ref).max()
-        # bf16 output rounding adds up to 2^-9 relative per element on top of REL
-        r_dq = rel_gate(g_dq, dq_ref, cfg.Dk)
+        extra = dq_rounding_model(case, kv, t_rows, heads, q, k_resp, v_resp, d_o) if dq_model else None
+        r_dq = rel_gate(g_dq, dq_ref, cfg.Dk, extra)
         j0 = 0 if full else max(0, cfg.R - tail)
         g_dk, g_dv = f64(dk[j0:, kv]), f64(dv[j0:, kv])
         e_dk = np.abs(g_dk - dk_ref[j0:]).max()
@@ -216,5 +274,5 @@ def check_backward(case, fw, kv_groups=None, full=True, tail=16, extra_rows=(), 
         assert abs_excess(g_dq, dq_ref, strict_abs) <= 1.0, ("dQ abs", report[kv])
         assert abs_excess(g_dk, dk_ref[j0:], strict_abs) <= 1.0, ("dK abs", report[kv])
         assert abs_excess(g_dv, dv_ref[j0:], strict_abs) <= 1.0, ("dV abs", report[kv])
-        assert r_dq <= rel_slack and r_dk <= rel_slack and r_dv <= rel_slack, report[kv]
+        assert r_dq <= 1.0 and r_dk <= 1.0 and r_dv <= 1.0, report[kv]
     return dict(dq=dq, dk=dk, dv=dv, report=report)

@@ -283,3 +283,30 @@ def test_mla_alias_value_is_prefix_of_key_page():
     c2 = dict(c, v_pool=np.ascontiguousarray(c["k_pool"][..., :8]))
     o2, lse2 = oa.replay_forward(**c2)
     assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
+
+
+def test_local_attention_value_slice_of_the_key_page():
+    # shared-latent pages: V is the first dv channels of the K page.  Brute force with scalar loops.
+    rng = np.random.default_rng(5)
+    pg, n_pages, dk, dv = 4, 3, 8, 5
+    pool = rng.standard_normal((n_pages, pg, 1, dk))
+    table = np.array([2, 0, 1])
+    q = rng.standard_normal((3, dk))
+    positions = np.array([1, 4, 5, 9, 10])
+    scale = 0.37
+    o, l = oa.local_attention(q, 0, pool, pool, table, pg, positions, scale, dv=dv)
+    assert o.shape == (3, dv)
+    for i in range(3):
+        s = []
+        for pos in positions:
+            key = pool[table[pos // pg], pos % pg, 0]
+            s.append(scale * sum(q[i, c] * key[c] for c in range(dk)))
+        m = max(s)
+        z = sum(np.exp(x - m) for x in s)
+        assert abs(l[i] - (m + np.log(z))) < 1e-12
+        for c in range(dv):
+            want = sum(np.exp(x - m) / z * pool[table[pos // pg], pos % pg, 0, c] for x, pos in zip(s, positions))
+            assert abs(o[i, c] - want) < 1e-12
+    # without dv the whole page would be the value: the slice is what makes the shapes differ
+    o_full, _ = oa.local_attention(q, 0, pool, pool, table, pg, positions, scale)
+    assert o_full.shape == (3, dk) and np.allclose(o_full[:, :dv], o)
