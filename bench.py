@@ -5,9 +5,16 @@ against a resident paged prefix) on B200.
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload p2m] [--impl reference]
 
 One "step" = one group member replayed against the resident prefix: ls_replay_attn_fwd,
-ls_lse_merge, ls_replay_attn_bwd.  Prints ONE JSON line (rank 0).  With N > 1 (torchrun)
-every rank holds its own replica of the prefix and replays different members: no
-collective on the data path, weak scaling.
+ls_lse_merge, ls_replay_attn_bwd.  Prints ONE JSON line (rank 0).  With N > 1 every rank
+holds its own replica of the prefix and replays different members: no collective on the
+data path, weak scaling.  `--gpus N` without a torchrun environment starts the N ranks itself.
+
+  --mode replay   forward (per-shard partials) + merge + backward              (default)
+  --mode fused    forward with the merge folded in + backward
+  --mode score    forward with the merge folded in only (a score-only pass)
+  --blocks B      blockwise replay of the response in B blocks with a paged suffix: a no-grad
+                  suffix pass (score + append per block), then the blocks in reverse (pop,
+                  forward, backward with gradient pages)
 """
 import argparse
 import json
@@ -29,12 +36,21 @@ from paper_2607_14952_b200 import workloads as W  # noqa: E402
 METRIC = "replay_attn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of the dQ kernel, from the one-pass ncu
-# capture summarised in profiles/dram_traffic_p2m.md (full-size workload, no scaling needed).
-DQ_KERNEL_NAME = {(256, 256): "bwd_dq3_kernel (query-gradient pass, CTA pairs)",
-                  (128, 128): "bwd_dq2_kernel<128> (query-gradient pass, CTA pairs)",
-                  (576, 512): "bwd_mla_dq_kernel (query-gradient pass, 576/512 shape)"}
-DQ_KERNEL_DRAM_BYTES = {"p2m": 16650.2e6 + 6615.7e6}
+DQ_KERNEL_NAME = {(256, 256): "bwd_dq3_kernel", (128, 128): "bwd_dq2_kernel", (576, 512): "bwd_mla_dq_kernel"}
+
+
+def measured_traffic(kernel, workload):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel` at `workload`, from the
+    committed ncu capture records (a JSON list of {kernel, workload, dram_bytes_per_launch, ...});
+    None when no capture of that kernel at that workload is on record."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        for rec in json.load(open(path)):
+            if rec.get("kernel") == kernel and rec.get("workload") == workload:
+                return rec.get("dram_bytes_per_launch")
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def algorithmic_flops(cfg):
@@ -103,6 +119,17 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def launch_ranks(args):
+    """`--gpus N` outside torchrun: start the N ranks (one per GPU) and pass their exit code on."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def run_cuda(args):
     from paper_2607_14952_b200 import binding as B
     rank = int(os.environ.get("RANK", "0"))
@@ -114,6 +141,8 @@ def run_cuda(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     cfg = W.CONFIGS[args.workload]
+    if args.prefix:
+        cfg = W.scaled(cfg, name="%s-P%d" % (cfg.name, args.prefix), P=args.prefix, needles=0)
     if args.small_r:
         # short-response regime: same resident prefix, R rows per head, finer key split so that
         # every SM streams its own slice of K/V -> bound by HBM, not by the tensor pipe
@@ -121,36 +150,83 @@ def run_cuda(args):
                        num_shards=args.shards or 64, needles=0)
     elif args.shards:
         cfg = W.scaled(cfg, name="%s-S%d" % (cfg.name, args.shards), num_shards=args.shards)
+    mode = "blocks" if args.blocks else args.mode
     fwd_f, dq_f, kv_f = algorithmic_flops(cfg)
-    step_flops = fwd_f + dq_f + kv_f
+    # algorithmic flops of one step: what the mode has to compute (the blockwise policy pass recomputes
+    # the forward that the suffix pass scored, as the method prescribes)
+    step_flops = {"replay": fwd_f + dq_f + kv_f, "fused": fwd_f + dq_f + kv_f, "score": fwd_f,
+                  "blocks": 2 * fwd_f + dq_f + kv_f}[mode]
 
-    k_pool, v_pool, table = W.make_prefix(cfg, dev)
+    torch.cuda.reset_peak_memory_stats(dev)
+    nblocks = args.blocks
+    rb = cfg.R // nblocks if nblocks else 0
+    if nblocks and (cfg.R % nblocks or rb % cfg.page_size):
+        raise SystemExit("--blocks must cut the response into whole pages")
+    extra_pages = nblocks * (rb // cfg.page_size) if nblocks else 0
+    k_pool, v_pool, table = W.make_prefix(cfg, dev, extra_phys_pages=extra_pages)
     pages = B.ls_prefix_pages_build(cfg.P, cfg.page_size, cfg.num_shards, cfg.Hkv, cfg.Dk, cfg.Dv, k_pool.shape[0],
                                     page_table=table, k_pool=k_pool, v_pool=None if cfg.v_aliases_k else v_pool,
                                     v_aliases_k=cfg.v_aliases_k)
+    pool_bytes = (k_pool.numel() + (0 if cfg.v_aliases_k else v_pool.numel())) * 2
     S = cfg.num_shards
     n_members = max(1, min(cfg.G, 4))
     members = [W.make_member(cfg, m, dev) for m in replicas.member_ids(rank, n_members)]
-    o_part = torch.empty((S + 1, cfg.R, cfg.Hq, cfg.Dv), dtype=torch.float32, device=dev)
-    lse_part = torch.empty((S + 1, cfg.R, cfg.Hq), dtype=torch.float32, device=dev)
-    o_bf16 = torch.empty((cfg.R, cfg.Hq, cfg.Dv), dtype=torch.bfloat16, device=dev)
-    o_f32 = torch.empty((cfg.R, cfg.Hq, cfg.Dv), dtype=torch.float32, device=dev)
-    lse = torch.empty((cfg.R, cfg.Hq), dtype=torch.float32, device=dev)
-    ws = torch.empty(B.ls_replay_attn_workspace_bytes(pages, cfg.R, cfg.Hq, cfg.scale, B.LS_WORKSPACE_BWD),
-                     dtype=torch.uint8, device=dev)
-    fwd_ws_bytes = B.ls_replay_attn_workspace_bytes(pages, cfg.R, cfg.Hq, cfg.scale, B.LS_WORKSPACE_FWD)
-    fwd_ws = torch.empty(fwd_ws_bytes, dtype=torch.uint8, device=dev) if fwd_ws_bytes else None
-    dq = torch.empty((cfg.R, cfg.Hq, cfg.Dk), dtype=torch.bfloat16, device=dev)
-    dk = torch.empty((cfg.R, cfg.Hkv, cfg.Dk), dtype=torch.bfloat16, device=dev)
-    dv = torch.empty((cfg.R, cfg.Hkv, cfg.Dv), dtype=torch.bfloat16, device=dev)
+    R_call = rb if nblocks else cfg.R
+    buf = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+    o_bf16 = buf((cfg.R, cfg.Hq, cfg.Dv), torch.bfloat16)
+    o_f32 = buf((cfg.R, cfg.Hq, cfg.Dv), torch.float32)
+    lse = buf((cfg.R, cfg.Hq), torch.float32)
+    dq = buf((cfg.R, cfg.Hq, cfg.Dk), torch.bfloat16)
+    dk = buf((cfg.R, cfg.Hkv, cfg.Dk), torch.bfloat16)
+    dv = buf((cfg.R, cfg.Hkv, cfg.Dv), torch.bfloat16)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws_bytes = {k: B.ls_replay_attn_workspace_bytes(pages, R_call, cfg.Hq, cfg.scale, k)
+                for k in (B.LS_WORKSPACE_FWD, B.LS_WORKSPACE_BWD, B.LS_WORKSPACE_FWD_MERGED)}
+    ws = buf(ws_bytes[B.LS_WORKSPACE_BWD], torch.uint8)
+    fwd_ws = buf(max(16, ws_bytes[B.LS_WORKSPACE_FWD], ws_bytes[B.LS_WORKSPACE_FWD_MERGED]), torch.uint8)
+    o_part = lse_part = None
+    if mode == "replay":
+        o_part = buf((S + 1, cfg.R, cfg.Hq, cfg.Dv), torch.float32)
+        lse_part = buf((S + 1, cfg.R, cfg.Hq), torch.float32)
+    free_ids = None
+    if nblocks:
+        mapped = set(int(x) for x in table)
+        free_ids = [p for p in range(k_pool.shape[0]) if p not in mapped][:extra_pages]
+        dk_grad = buf((extra_pages, cfg.page_size, cfg.Hkv, cfg.Dk), torch.float32)
+        dv_grad = buf((extra_pages, cfg.page_size, cfg.Hkv, cfg.Dv), torch.float32)
+        B.ls_suffix_pages_reserve(pages, nblocks, extra_pages, dk_grad, dv_grad)
+    mla = cfg.Dk == 576
 
     def step(q, kr, vr, d_o):
-        B.ls_replay_attn_fwd(pages, q, kr, vr, cfg.scale, o_part=o_part, lse_part=lse_part, status=status,
-                             workspace=fwd_ws)
-        B.ls_lse_merge(o_part, lse_part, o_bf16=o_bf16, o_f32=o_f32, lse=lse)
-        B.ls_replay_attn_bwd(pages, q, kr, vr, o_f32, lse, d_o, cfg.scale, workspace=ws, dq=dq, dk_resp=dk,
-                             dv_resp=dv, status=status)
+        if mode == "replay":
+            B.ls_replay_attn_fwd(pages, q, kr, vr, cfg.scale, o_part=o_part, lse_part=lse_part, status=status,
+                                 workspace=fwd_ws)
+            B.ls_lse_merge(o_part, lse_part, o_bf16=o_bf16, o_f32=o_f32, lse=lse, status=status)
+        elif mode in ("fused", "score"):
+            B.ls_replay_attn_fwd_merged(pages, q, kr, vr, cfg.scale, o_bf16=o_bf16, o_f32=o_f32, lse=lse,
+                                        status=status, workspace=fwd_ws)
+        if mode in ("replay", "fused"):
+            B.ls_replay_attn_bwd(pages, q, kr, vr, o_f32, lse, d_o, cfg.scale, workspace=ws, dq=dq, dk_resp=dk,
+                                 dv_resp=dv, status=status)
+        if mode == "blocks":
+            ppb = rb // cfg.page_size
+            sl = lambda x, b: x[b * rb:(b + 1) * rb]
+            for b in range(nblocks):            # no-grad suffix pass: score the block, append its pages
+                B.ls_replay_attn_fwd_merged(pages, sl(q, b), sl(kr, b), sl(vr, b), cfg.scale, o_bf16=sl(o_bf16, b),
+                                            o_f32=sl(o_f32, b), lse=sl(lse, b), status=status, workspace=fwd_ws)
+                B.ls_suffix_pages_append(pages, free_ids[b * ppb:(b + 1) * ppb], sl(kr, b), sl(vr, b))
+            for b in reversed(range(nblocks)):  # policy pass in reverse: pop, replay, backward
+                B.ls_suffix_pages_pop(pages)
+                B.ls_replay_attn_fwd_merged(pages, sl(q, b), sl(kr, b), sl(vr, b), cfg.scale, o_bf16=sl(o_bf16, b),
+                                            o_f32=sl(o_f32, b), lse=sl(lse, b), status=status, workspace=fwd_ws)
+                B.ls_replay_attn_bwd(pages, sl(q, b), sl(kr, b), sl(vr, b), sl(o_f32, b), sl(lse, b), sl(d_o, b),
+                                     cfg.scale, workspace=ws, dq=sl(dq, b), dk_resp=sl(dk, b), dv_resp=sl(dv, b),
+                                     status=status, flags=B.LS_FLAG_ADD_SUFFIX_GRAD)
+
+    # kernels of this library launched per step (memsets and copies are not kernels)
+    bwd_launches = 5 if mla else 4                       # Delta, dQ (+ the response block's dQ for 576/512), dK, dV
+    launches = {"replay": 2 + bwd_launches, "fused": 1 + bwd_launches, "score": 1,
+                "blocks": 0 if not nblocks else sum(1 + 2 + 1 + bwd_launches + 2 * b for b in range(nblocks))}[mode]
 
     def barrier():
         torch.cuda.synchronize()
@@ -164,29 +240,33 @@ def run_cuda(args):
 
     # ---- device-resident timing; the dominant kernels are timed alone through armed events
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
+    timed_kernels = (B.LS_KERNEL_FWD,) if mode == "score" else (B.LS_KERNEL_FWD, B.LS_KERNEL_BWD_DQ)
     kev = {k: [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
-           for k in (B.LS_KERNEL_FWD, B.LS_KERNEL_BWD_DQ)}
+           for k in timed_kernels}
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     barrier()
     for i in range(args.steps):
-        for k in kev:
-            B.ls_profile_arm_events(k, kev[k][i][0], kev[k][i][1])
+        if mode != "blocks":
+            for k in kev:
+                B.ls_profile_arm_events(k, kev[k][i][0], kev[k][i][1])
         ev[i][0].record()
         step(*members[i % n_members])
         ev[i][1].record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    ms = sum(a.elapsed_time(b) for a, b in ev)
-    k_ms = {k: sum(a.elapsed_time(b) for a, b in kev[k]) / args.steps for k in kev}
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    ms = sum(step_ms)
+    k_ms = {k: (sum(a.elapsed_time(b) for a, b in kev[k]) / args.steps if mode != "blocks" else float("nan")) for k in kev}
     ms_total = replicas.max_over_ranks(ms, dev, world)
     if int(status.item()) != 0:
         raise RuntimeError("device status %d" % int(status.item()))
 
     # ---- end to end: host buffers in, host results out, copies inside the timed region
+    outs = (o_bf16,) if mode == "score" else (o_bf16, dq, dk, dv)
     host_in = [[x.cpu().pin_memory() for x in m] for m in members]
-    host_out = [torch.empty_like(x, device="cpu").pin_memory() for x in (o_bf16, dq, dk, dv)]
+    host_out = [torch.empty_like(x, device="cpu").pin_memory() for x in outs]
     dev_in = [torch.empty_like(x) for x in members[0]]
     h2d = sum(x.numel() * x.element_size() for x in host_in[0])
     d2h = sum(x.numel() * x.element_size() for x in host_out)
@@ -195,7 +275,7 @@ def run_cuda(args):
         for d, hsrc in zip(dev_in, host_in[i % n_members]):
             d.copy_(hsrc, non_blocking=True)
         step(*dev_in)
-        for hdst, d in zip(host_out, (o_bf16, dq, dk, dv)):
+        for hdst, d in zip(host_out, outs):
             hdst.copy_(d, non_blocking=True)
 
     e2e_step(0)
@@ -209,6 +289,7 @@ def run_cuda(args):
     barrier()
     e2e_wall = time.perf_counter() - t0
     e2e_ms = replicas.max_over_ranks(max(e0.elapsed_time(e1), e2e_wall * 1e3), dev, world)
+    peak_bytes = torch.cuda.max_memory_allocated(dev)
 
     if rank != 0:
         if world > 1:
@@ -217,46 +298,66 @@ def run_cuda(args):
     peaks = measured_peaks()
     ms_per_step = ms_total / args.steps
     value = replicas.aggregate_throughput(step_flops, args.steps, world, ms_total) / 1e12
-    dq_tflops = dq_f / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e12
-    fwd_tflops = fwd_f / (k_ms[B.LS_KERNEL_FWD] * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
+    fwd_tflops = fwd_f / (k_ms[B.LS_KERNEL_FWD] * 1e-3) / 1e12
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_best": min(step_ms),
+        "ms_per_step_median": float(np.median(step_ms)), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "%s: P=%d R=%d Hq=%d Hkv=%d Dk=%d Dv=%d page=%d shards=%d, one member per step" % (
             cfg.name, cfg.P, cfg.R, cfg.Hq, cfg.Hkv, cfg.Dk, cfg.Dv, cfg.page_size, cfg.num_shards),
-            "l2": "inputs larger than L2 (%.2f GiB of K/V streamed per pass)" % (
-                (k_pool.numel() + (0 if cfg.v_aliases_k else v_pool.numel())) * 2 / 2**30),
+            "mode": mode if not nblocks else "blocks x%d of %d tokens (suffix pass + reverse policy pass)" % (nblocks, rb),
+            "l2": "inputs larger than L2 (%.2f GiB of K/V streamed per pass)" % (pool_bytes / 2**30),
             "parallelism": "replicas x%d" % world, "flops_per_step": step_flops,
             "prefix_positions_per_s": world * cfg.P / (ms_per_step * 1e-3)},
         "clocks": clocks,
         "e2e": {"value": world * step_flops / (e2e_ms / args.steps * 1e-3) / 1e12, "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": (7 + (1 if fwd_ws is not None else 0)) * args.steps,
-        "roofline": {"bound": "tensor", "kernel": DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv), "query-gradient pass"),
-                     "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
-                     "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
-                     "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
-                     "traffic": DQ_KERNEL_DRAM_BYTES.get(cfg.name),
-                     "algorithmic_flops_per_launch": dq_f,
-                     "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peak,
-                                    "ms_per_launch": k_ms[B.LS_KERNEL_FWD]},
-                     "whole_step_frac": value / world / peak,
-                     "frac_of_nominal_2250": value / world / 2250.0},
+        "gpu_launches": launches * args.steps,
+        "peak_device_bytes": peak_bytes,
+        "device_bytes": {"page_pool": pool_bytes, "workspace_fwd": ws_bytes[B.LS_WORKSPACE_FWD],
+                         "workspace_fwd_merged": ws_bytes[B.LS_WORKSPACE_FWD_MERGED],
+                         "workspace_bwd": ws_bytes[B.LS_WORKSPACE_BWD],
+                         "partials": 0 if o_part is None else (o_part.numel() + lse_part.numel()) * 4},
     }
-    if args.small_r:
-        kv_bytes = (k_pool.numel() + (0 if cfg.v_aliases_k else v_pool.numel())) * 2
+    if mode in ("replay", "fused"):
+        dq_tflops = dq_f / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e12
+        kname = DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv))
+        out["roofline"] = {"bound": "tensor", "kernel": "%s (query-gradient pass over all parts)" % kname,
+                           "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
+                           "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
+                           "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
+                           "traffic": measured_traffic(kname, cfg.name),
+                           "algorithmic_flops_per_launch": dq_f,
+                           "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peak,
+                                          "ms_per_launch": k_ms[B.LS_KERNEL_FWD]},
+                           "whole_step_frac": value / world / peak,
+                           "frac_of_nominal_2250": value / world / 2250.0}
+    elif mode == "score":
+        kname = "fwd2_kernel" if cfg.Dk == 256 else "fwd_kernel"
+        out["roofline"] = {"bound": "tensor", "kernel": "%s (forward with the merge folded in)" % kname,
+                           "achieved": fwd_tflops, "peak": peak, "unit": UNIT, "frac": fwd_tflops / peak,
+                           "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
+                           "ms_per_launch": k_ms[B.LS_KERNEL_FWD], "traffic": measured_traffic(kname + ":merged", cfg.name),
+                           "algorithmic_flops_per_launch": fwd_f, "frac_of_nominal_2250": value / world / 2250.0}
+    else:
+        out["roofline"] = {"bound": "tensor", "kernel": "whole blockwise step (no single dominant launch)",
+                           "achieved": value / world, "peak": peak, "unit": UNIT, "frac": value / world / peak,
+                           "peak_source": "%s sustained bf16 cuBLAS" % peaks["source"], "traffic": None}
+    if args.small_r and mode != "blocks":
+        kv_bytes = pool_bytes
         fwd_gbs = kv_bytes / (k_ms[B.LS_KERNEL_FWD] * 1e-3) / 1e9
-        dq_gbs = kv_bytes / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e9
-        out["roofline"] = {"bound": "hbm", "kernel": "fwd_kernel (K and V pages streamed once per launch)",
+        fname = "fwd_kernel" if cfg.Hq // cfg.Hkv * cfg.R <= 128 or cfg.Dk != 256 else "fwd2_kernel"
+        out["roofline"] = {"bound": "hbm", "kernel": "%s (K and V pages streamed once per launch)" % fname,
                            "achieved": fwd_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": fwd_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
-                           "ms_per_launch": k_ms[B.LS_KERNEL_FWD], "traffic": None,
-                           "algorithmic_bytes_per_launch": kv_bytes,
-                           "dq_kernel": {"achieved": dq_gbs, "frac": dq_gbs / peaks["hbm_gbs"],
-                                         "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ]},
-                           "frac_of_nominal_8000": fwd_gbs / 8000.0}
+                           "ms_per_launch": k_ms[B.LS_KERNEL_FWD], "traffic": measured_traffic(fname, cfg.name),
+                           "algorithmic_bytes_per_launch": kv_bytes, "frac_of_nominal_8000": fwd_gbs / 8000.0}
+        if B.LS_KERNEL_BWD_DQ in k_ms:
+            dq_gbs = kv_bytes / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e9
+            out["roofline"]["dq_kernel"] = {"achieved": dq_gbs, "frac": dq_gbs / peaks["hbm_gbs"],
+                                            "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ]}
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, seconds_target=15.0)
     print(json.dumps(out))
@@ -341,11 +442,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--small-r", type=int, default=0, help="short-response regime: R rows per head")
     ap.add_argument("--shards", type=int, default=0, help="key shards for --small-r (default 64)")
+    ap.add_argument("--prefix", type=int, default=0, help="override the workload's prefix length (profiling on a small case)")
+    ap.add_argument("--mode", default="replay", choices=["replay", "fused", "score"])
+    ap.add_argument("--blocks", type=int, default=0, help="blockwise replay with a paged suffix in this many blocks")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args))
     else:
         run_cuda(args)
 
