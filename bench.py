@@ -166,7 +166,7 @@ def run_cuda(args):
     k_pool, v_pool, table = W.make_prefix(cfg, dev, extra_phys_pages=extra_pages)
     pages = B.ls_prefix_pages_build(cfg.P, cfg.page_size, cfg.num_shards, cfg.Hkv, cfg.Dk, cfg.Dv, k_pool.shape[0],
                                     page_table=table, k_pool=k_pool, v_pool=None if cfg.v_aliases_k else v_pool,
-                                    v_aliases_k=cfg.v_aliases_k)
+                                    v_aliases_k=cfg.v_aliases_k, stream_budget_kib=args.stream_budget_kib)
     pool_bytes = (k_pool.numel() + (0 if cfg.v_aliases_k else v_pool.numel())) * 2
     S = cfg.num_shards
     n_members = max(1, min(cfg.G, 4))
@@ -443,6 +443,8 @@ def main():
     ap.add_argument("--small-r", type=int, default=0, help="short-response regime: R rows per head")
     ap.add_argument("--shards", type=int, default=0, help="key shards for --small-r (default 64)")
     ap.add_argument("--prefix", type=int, default=0, help="override the workload's prefix length (profiling on a small case)")
+    ap.add_argument("--stream-budget-kib", type=int, default=0,
+                    help="K+V bytes of one (KV head, key range) stream, in KiB (0 = the library's default)")
     ap.add_argument("--mode", default="replay", choices=["replay", "fused", "score"])
     ap.add_argument("--blocks", type=int, default=0, help="blockwise replay with a paged suffix in this many blocks")
     args = ap.parse_args()

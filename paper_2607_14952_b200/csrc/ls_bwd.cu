@@ -65,7 +65,7 @@ struct BwdParams {
 
 #ifdef LS_TIMING
 #define LS_BTWAIT(acc, expr) ([&] { const long long t0_ = clock64(); const bool r_ = (expr); (acc) += clock64() - t0_; return r_; }())
-#define LS_BTDUMP(slot, val) do { if (blockIdx.x == 0 && p.timing) p.timing[(slot)] = (val); } while (0)
+#define LS_BTDUMP(slot, val) do { if (p.timing && it.link == 1 && it.kvh == 0 && it.pairi == 0 && rank == 0) p.timing[(slot)] = (val); } while (0)
 #else
 #define LS_BTWAIT(acc, expr) (expr)
 #define LS_BTDUMP(slot, val) do { } while (0)
@@ -447,6 +447,7 @@ template <int NCOL>
 __device__ __forceinline__ void dq_store_row(uint32_t tmem_row, bool have_acc, bool fold, bool last, float scale,
                                              float* acc_dst, __nv_bfloat16* dq_dst, bool row_ok) {
   if (!have_acc && fold && !last) return;
+  const uint64_t pol = last ? l2_policy_evict_first() : l2_policy_evict_last();
 #pragma unroll 1
   for (int c = 0; c < NCOL; c += 32) {
     uint32_t o[32];
@@ -461,7 +462,7 @@ __device__ __forceinline__ void dq_store_row(uint32_t tmem_row, bool have_acc, b
       float4 run[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        run[j] = fold ? __ldcg(reinterpret_cast<const float4*>(acc_dst + c) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        run[j] = fold ? ld_cg_hint(reinterpret_cast<const float4*>(acc_dst + c) + j, pol) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         float4 v;
@@ -475,7 +476,7 @@ __device__ __forceinline__ void dq_store_row(uint32_t tmem_row, bool have_acc, b
           pk.y = pack_bf16(v.z * scale, v.w * scale);
           *(reinterpret_cast<uint2*>(dq_dst + c) + j) = pk;
         } else {
-          *(reinterpret_cast<float4*>(acc_dst + c) + j) = v;
+          st_hint(reinterpret_cast<float4*>(acc_dst + c) + j, v, pol);
         }
       }
     }
@@ -483,12 +484,15 @@ __device__ __forceinline__ void dq_store_row(uint32_t tmem_row, bool have_acc, b
 }
 
 // ---------------------------------------------------------------------------------
-// dQ pass on CTA pairs (cta_group::2).  Two neighbouring SMs take two Q tiles of the same
-// (KV head, partial) and stream the keys once between them: each CTA loads only half of
-// every K/V chunk (64 of the 128 keys for S and T, 64 of the 128 channels for ACC), so the
-// ring covers twice as many keys and the shared-memory write traffic halves.  One thread of
+// dQ pass on CTA pairs (cta_group::2), 128-key tiles.  Two neighbouring SMs take two Q tiles of
+// the same (KV head, part) and stream the keys once between them: each CTA loads only half of
+// every K/V chunk (64 of the 128 keys for S and T, half of the channels for ACC).  One thread of
 // the even CTA issues all MMAs (256 rows); completions are multicast to both CTAs' barriers;
-// the odd CTA's row threads report their E quarters to the even CTA's barrier.
+// the odd CTA's row threads report to the even CTA's barriers.
+// TMEM: ACC [0, D), S [D, D+128), T [D+128, D+256).  E (bf16) is written over T, not over S, so
+// the S buffer is free as soon as the row threads have pulled it and the tensor pipe runs
+//     S(0) T(0) | S(i+1)  ACC(i)  T(i+1) | ...
+// with S(i+1) overlapping the row threads' E(i) and ACC(i) / T(i+1) overlapping their p(i+1).
 // ---------------------------------------------------------------------------------
 constexpr int kDq2Chunk = 16384;
 
@@ -515,7 +519,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   uint64_t* full = bars + 1;             // (even CTA) both halves of a chunk landed
   uint64_t* empty = full + C::RING;      // (each CTA) chunk consumed
   uint64_t* s_full = empty + C::RING;    // (each CTA) S in TMEM
-  uint64_t* t_full = s_full + 1;         // (each CTA) T in TMEM
+  uint64_t* s_read = s_full + 1;         // (even CTA) every row thread of both CTAs has pulled S: 16 warp arrivals
+  uint64_t* t_full = s_read + 1;         // (each CTA) T in TMEM
   uint64_t* e_full = t_full + 1;         // [4] (even CTA) quarter of E in both CTAs' TMEM: 16 warp arrivals
   uint64_t* acc_final = e_full + 4;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
@@ -537,6 +542,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
       mbar_init(&empty[i], 1);
     }
     mbar_init(s_full, 1);
+    mbar_init(s_read, 16);
     mbar_init(t_full, 1);
     for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 16);
     mbar_init(acc_final, 1);
@@ -641,19 +647,21 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
         ++issued;
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
-      auto load_st = [&](int i, int pa, int pb) {
-        for (int c = 0; c < C::NC; ++c) load(0, i, c, pa, pb);
-        for (int c = 0; c < C::NC; ++c) load(1, i, c, pa, pb);
+      // chunk order = consumption order: S(0) T(0) [S(i+1) ACC(i) T(i+1)] ...
+      auto load_op = [&](int which, int i, int pa, int pb) {
+        for (int c = 0; c < C::NC; ++c) load(which, i, c, pa, pb);
       };
       const int sh = p.pg_shift - 7;
       auto slot_of = [&](int i) { return small_pages ? 2 * i : (i >> sh); };
       int pa0 = fetch(slot_of(0)), pb0 = small_pages ? fetch(1) : pa0;
       int pa1 = fetch(slot_of(1)), pb1 = small_pages ? fetch(3) : pa1;
-      load_st(0, pa0, pb0);
+      load_op(0, 0, pa0, pb0);
+      load_op(1, 0, pa0, pb0);
       for (int i = 0; i < n_tiles; ++i) {
         const int pa2 = fetch(slot_of(i + 2)), pb2 = small_pages ? fetch(2 * i + 5) : pa2;
-        for (int c = 0; c < C::NC; ++c) load(2, i, c, pa0, pb0);
-        if (i + 1 < n_tiles) load_st(i + 1, pa1, pb1);
+        if (i + 1 < n_tiles) load_op(0, i + 1, pa1, pb1);
+        load_op(2, i, pa0, pb0);
+        if (i + 1 < n_tiles) load_op(1, i + 1, pa1, pb1);
         pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
       }
       LS_BTDUMP(0, tw0);
@@ -682,9 +690,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
       auto advance = [&]() {
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
-      auto issue_st = [&](int i) {
-#pragma unroll
-        for (int op = 0; op < 2; ++op) {
+      // S = Q K^T (op 0) or T = dO V^T (op 1) of tile i
+      auto issue_op = [&](int op) {
+        {
           const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
           const uint32_t d = op == 0 ? tmem_s : tmem_t;
 #pragma unroll
@@ -727,12 +735,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
             tc_fence_after();
           }
           if (C::NC == 2) {
-            // D = 256: the two 64-channel groups sit in adjacent slots (6 chunks per tile in a ring
-            // of 6 keeps them at slots 4 and 5): one 256-wide MMA per 16 keys
+            // D = 256: the two 64-channel groups sit in adjacent slots (every operand takes two slots
+            // of a ring of six, so a pair never wraps): one 256-wide MMA per 16 keys
             const uint32_t b_lo = ring2_lo + cs[0] * (kDq2Chunk >> 4);
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk)
-              mma_ts_pair(tmem_acc, tmem_s + (2 * qd + kk) * 8, sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi),
+              mma_ts_pair(tmem_acc, tmem_t + (2 * qd + kk) * 8, sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi),
                           idesc_acc2, (i | qd | kk) != 0);
           } else {
 #pragma unroll
@@ -740,7 +748,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
               const uint32_t b_lo = ring_lo + cs[c] * (kDq2Chunk >> 4);
 #pragma unroll
               for (int kk = 0; kk < 2; ++kk)
-                mma_ts_pair(tmem_acc + c * 128, tmem_s + (2 * qd + kk) * 8,
+                mma_ts_pair(tmem_acc + c * 128, tmem_t + (2 * qd + kk) * 8,
                             sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi), idesc_acc, (i | qd | kk) != 0);
             }
           }
@@ -751,10 +759,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
         }
         if (i == n_tiles - 1) mma_commit_pair(acc_final);
       };
-      if (ok) issue_st(0);
+      // E overwrites T (not S), so S of the next tile only waits for the row threads to have pulled S:
+      // the tensor pipe runs S(i+1) while the row threads form E(i), then ACC(i), then T(i+1).
+      if (ok) issue_op(0);
+      if (ok) issue_op(1);
       for (int i = 0; i < n_tiles && ok; ++i) {
-        issue_acc(i);
-        if (ok && i + 1 < n_tiles) issue_st(i + 1);
+        if (i + 1 < n_tiles) {
+          ok = ok && LS_BTWAIT(tw0, mbar_wait(s_read, i & 1, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          issue_op(0);
+        }
+        if (ok) issue_acc(i);
+        if (ok && i + 1 < n_tiles) issue_op(1);
       }
       LS_BTDUMP(8, tw0);
       LS_BTDUMP(9, tw1);
@@ -778,43 +795,54 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
       const float lse2_row = p.lse[ri] * kLog2e;
       const float delta_row = p.delta[ri];
       const int64_t lim = is_resp ? (int64_t)min(r_idx, p.R - 1) : tokens - 1;
+      const uint32_t s_read_remote = mapa_u32(smem_u32(s_read), 0);
       uint32_t e_remote[4];
 #pragma unroll
       for (int qd = 0; qd < 4; ++qd) e_remote[qd] = mapa_u32(smem_u32(&e_full[qd]), 0);
       for (int i = 0; i < n_tiles; ++i) {
         const int key0 = i * 128;
         const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim);
+        // No thread leaves this loop on its own: a wait that gave up is remembered in `ok` and put
+        // to the vote at the tile's named barrier, where all 256 leave together.
         ok = ok && LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
         tc_fence_after();
+        // p = exp(s - LSE) for this thread's 4 x 16 columns; once S is in registers the next tile's
+        // S may overwrite the buffer
+        uint32_t sr[64];
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr + 16 * qd);
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(sr + 16 * qd);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(s_read_remote);
         float pr[64];
 #pragma unroll
-        for (int qd = 0; qd < 4; ++qd) {
-          uint32_t sr[16];
-          tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr);
-          tc_wait_ld16(sr);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
-            if (edge && (int64_t)key0 + 32 * qd + 16 * half + j > lim) e = 0.f;
-            pr[16 * qd + j] = e;
-          }
+        for (int j = 0; j < 64; ++j) {
+          float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
+          if (edge && (int64_t)key0 + 32 * (j >> 4) + 16 * half + (j & 15) > lim) e = 0.f;
+          pr[j] = e;
         }
-        // all S reads of this CTA done before any E write; the barrier also carries the vote on
-        // whether any wait gave up, so the row threads leave the loop together or not at all
+        // T of the tile, all of it into registers: E (bf16) goes over T's columns, which the row's
+        // other thread reads too, so every T read of the CTA comes before any E write (named barrier 1)
+        ok = ok && LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
+        tc_fence_after();
+        uint32_t tr[64];
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr + 16 * qd);
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(tr + 16 * qd);
         ok = bar_and(1, 256, ok);
         if (!ok) break;
-        ok = LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));   // a failure here is voted on in the next round
-        tc_fence_after();
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-          uint32_t tr[16], pk[8];
-          tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr);
-          tc_wait_ld16(tr);
+          uint32_t pk[8];
 #pragma unroll
           for (int j = 0; j < 16; j += 2)
-            pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[j]) - delta_row),
-                                   pr[16 * qd + j + 1] * (__uint_as_float(tr[j + 1]) - delta_row));
-          tmem_st8(tmem_s + lane_sel + 16 * qd + 8 * half, pk);
+            pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[16 * qd + j]) - delta_row),
+                                   pr[16 * qd + j + 1] * (__uint_as_float(tr[16 * qd + j + 1]) - delta_row));
+          // quarter q of E (bf16 pairs) lands in columns [16 q, 16 q + 16) of the T region
+          tmem_st8(tmem_t + lane_sel + 16 * qd + 8 * half, pk);
           tc_wait_st();
           tc_fence_before();
           __syncwarp();

@@ -119,7 +119,7 @@ __device__ __forceinline__ int fwd_chain_index(const FwdParams& p, const FwdItem
 template <int DV>
 __device__ __forceinline__ void fwd_store_row(uint32_t tmem_row, bool have_acc, float l, float m_scaled, bool fold,
                                               float* o_dst, float* lse_dst, bool write_lse, __nv_bfloat16* bf_dst,
-                                              bool row_ok) {
+                                              bool row_ok, bool chained, bool chain_last) {
   const bool own = have_acc && l > 0.f;
   const float lse_own = own ? m_scaled + logf(l) : -INFINITY;
   float c_own = own ? 1.0f / l : 0.f, c_run = 0.f, lse_new = lse_own;
@@ -138,6 +138,8 @@ __device__ __forceinline__ void fwd_store_row(uint32_t tmem_row, bool have_acc, 
   }
   const bool store = row_ok && (!fold || c_own != 0.f || bf_dst != nullptr);
   const bool load_run = fold && c_run != 0.f;
+  // the running value of a chain is kept in L2 past the K/V stream; the last link hands it back
+  const uint64_t pol = (chain_last || !chained) ? l2_policy_evict_first() : l2_policy_evict_last();
 #pragma unroll 1
   for (int c = 0; c < DV; c += 32) {
     uint32_t o[32];
@@ -152,7 +154,7 @@ __device__ __forceinline__ void fwd_store_row(uint32_t tmem_row, bool have_acc, 
       float4 run[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        run[j] = load_run ? __ldcg(reinterpret_cast<const float4*>(o_dst + c) + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        run[j] = load_run ? ld_cg_hint(reinterpret_cast<const float4*>(o_dst + c) + j, pol) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         float4 v;
@@ -160,7 +162,8 @@ __device__ __forceinline__ void fwd_store_row(uint32_t tmem_row, bool have_acc, 
         v.y = fmaf(c_run, run[j].y, c_own * __uint_as_float(o[4 * j + 1]));
         v.z = fmaf(c_run, run[j].z, c_own * __uint_as_float(o[4 * j + 2]));
         v.w = fmaf(c_run, run[j].w, c_own * __uint_as_float(o[4 * j + 3]));
-        *(reinterpret_cast<float4*>(o_dst + c) + j) = v;
+        if (chained) st_hint(reinterpret_cast<float4*>(o_dst + c) + j, v, pol);
+        else *(reinterpret_cast<float4*>(o_dst + c) + j) = v;
         if (bf_dst) {
           uint2 pk;
           pk.x = pack_bf16(v.x, v.y);
@@ -557,7 +560,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     if (ok)
       fwd_store_row<DV>(tmem_o + lane_sel, n_tiles > 0, l, m_ref * p.scale, fold, o_dst, lse_dst,
                         dvh == 0 || it.chained, (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total + dvh * DVT : nullptr,
-                        row_ok);
+                        row_ok, it.chained, it.chained && (p.chain_mode == 2 ? it.last : it.link == p.fine - 1));
     if (it.chained) {
       const bool all_ok = bar_and(2, 128, ok);     // every row of the tile is written
       if (row == 0 && all_ok) chain_publish(counter, it.link + 1);
@@ -893,7 +896,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
     if (ok)
       fwd_store_row<DV>(tmem_o + lane_sel, n_tiles > 0, l, m_ref * p.scale, fold, o_dst, lse_dst, true,
-                        (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total : nullptr, row_ok);
+                        (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total : nullptr, row_ok, chained,
+                        chained && (p.chain_mode == 2 ? it.last : it.link == p.fine - 1));
     if (chained) {
       const bool all_ok = bar_and(2, 128, ok);     // every row of the tile is written
       if (row == 0 && all_ok) chain_publish(counter, it.link + 1);

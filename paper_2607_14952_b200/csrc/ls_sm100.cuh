@@ -146,6 +146,32 @@ __device__ __forceinline__ bool chain_wait(const int* counter, int want, const i
     __nanosleep(256);
   }
 }
+// Accesses to a chain's running value carry an L2 eviction hint: the value is re-read one part
+// later by another CTA and should outlive the K/V stream that passes through L2 in between
+// (evict_last); the chain's last link reads it with evict_first, which hands the lines back.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ float4 ld_cg_hint(const float4* ptr, uint64_t pol) {
+  float4 v;
+  asm volatile("ld.global.cg.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(ptr), "l"(pol)
+               : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_hint(float4* ptr, float4 v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(ptr), "f"(v.x), "f"(v.y), "f"(v.z),
+               "f"(v.w), "l"(pol)
+               : "memory");
+}
 // Called by ONE thread after a CTA-level barrier that all writers of the running value passed.
 __device__ __forceinline__ void chain_publish(int* counter, int value) {
   __threadfence();
