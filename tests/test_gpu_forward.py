@@ -75,6 +75,24 @@ def test_forward_is_deterministic_and_page_permutation_invariant():
     assert torch.equal(o_part, a[0]) and torch.equal(lse_part, a[1])
 
 
+def test_merged_forward_is_bit_reproducible_and_close_to_the_two_step_path():
+    # the forward with the merge folded in hands its partial results over between CTAs in a fixed
+    # order: two runs agree bit for bit (also with sub-ranges forced by a small stream budget), and the
+    # result agrees with forward + ls_lse_merge up to fp32 rounding of a different summation order
+    for budget in (0, 256):
+        cfg = small("merged_det", P=256 * 19 + 77, page_size=256, num_shards=3, R=300, Hq=6, Hkv=2)
+        case = parity.Case(cfg, stream_budget_kib=budget)
+        q, k, v, _ = case.member(0)
+        a = case.forward_merged(q, k, v)
+        b = case.forward_merged(q, k, v)
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+        _, _, o_bf16, o_f32, lse = case.forward(q, k, v)
+        assert (a[2] - lse).abs().max() < 1e-5
+        assert (a[1] - o_f32).abs().max() < 1e-5
+        assert (a[0].float() - o_bf16.float()).abs().max() <= 2.0 ** -8 * o_bf16.float().abs().max()
+
+
 def test_forward_split_count_does_not_change_the_merge():
     outs = []
     for S in (1, 2, 4, 8, 32):
