@@ -143,6 +143,11 @@ typedef struct {
 /* Backward only: add the retained suffix gradient pages of the block that was popped last
  * (the one being replayed) to dk_resp / dv_resp.  See ls_suffix_pages_append. */
 #define LS_FLAG_ADD_SUFFIX_GRAD (1 << 0)
+/* Forward and backward: leave the causal response block out.  The call then covers the prefix
+ * (and suffix) parts only: k_resp / v_resp / dk_resp / dv_resp are not used (may be NULL), the
+ * forward writes the response block's partial as empty, dQ sums the remaining parts.  Used to
+ * compose attention over several key sets that share one response (sparse replay). */
+#define LS_FLAG_NO_RESPONSE_BLOCK (1 << 1)
 
 enum { LS_WORKSPACE_FWD = 0, LS_WORKSPACE_BWD = 1, LS_WORKSPACE_FWD_MERGED = 2 };
 
@@ -268,6 +273,62 @@ ls_status_t ls_suffix_pages_append(ls_pages_t* pages, int32_t n_tokens, const in
 ls_status_t ls_suffix_pages_pop(ls_pages_t* pages);
 uint64_t ls_pages_generation(const ls_pages_t* pages);
 int64_t ls_suffix_pages_tokens(const ls_pages_t* pages);
+
+/*
+ * Sparse (DSA) replay over the shared latent (Sec. "GLM Attention: MLA, DSA, and IndexShare",
+ * Eq. dsa-index, Eq. dsa-attention; the selection is global over the logical context as
+ * Eq. glm-global-dsa requires, not per shard).  For response query t:
+ *   I[t,s] = sum_j w[t,j] ReLU(<q_index[t,j], k_index[s]>)          s = 0 .. P-1
+ *   S_t    = the top_k prefix positions by I[t,:]; ties go to the lower position; all P when P <= top_k
+ *   u_t    = softmax attention of q[t,h] over the latent rows {c_s : s in S_t} and the causal response
+ *            block (j <= t, always attended: the response is short and dense), value = first dim_v
+ *            channels of the latent row
+ * The backward holds S_t fixed (TopK is piecewise constant): dQ over the selected rows and the
+ * response block, dK / dV of the response tokens; the prefix gets no gradient.
+ * Requires the 576/512 shape with v_aliases_k, one KV head, 64-channel-aligned strides, no suffix
+ * blocks; num_q_heads <= 128; num_index_heads in {8,16,32,64}; index_dim 128.
+ *  ki_pool  [num_phys_pages, page_size, index_dim] bf16: indexer-key pages under the SAME page table
+ *           as the latent pool (strides in elements)
+ *  gathered caller-owned device buffer of ls_dsa_gathered_bytes() bytes that receives the selected
+ *           latent rows of every query token ([pages of 64, 64, R, dim_k]); ls_dsa_attn_bwd reads
+ *           what the last ls_dsa_attn_fwd of the plan left there
+ * ls_dsa_plan_create builds two small internal page plans (allocates a few KB of device metadata).
+ *  ls_dsa_index_scores: q_index [R, H_I, index_dim] bf16, w_index [R, H_I] fp32 -> scores [R, P] fp32
+ *  ls_dsa_topk: scores -> sel [R, ls_dsa_selected_count()] int32, ascending positions per row
+ *  ls_dsa_attn_fwd: q [R,Hq,dim_k], k_resp [R,1,dim_k], v_resp [R,1,dim_v] bf16 -> o_bf16 (nullable),
+ *           o_f32 [R,Hq,dim_v], lse [R,Hq]; workspace ls_dsa_workspace_bytes(plan, LS_WORKSPACE_FWD)
+ *  ls_dsa_attn_bwd: + d_o -> dq [R,Hq,dim_k], dk_resp [R,1,dim_k], dv_resp [R,1,dim_v] bf16;
+ *           workspace ls_dsa_workspace_bytes(plan, LS_WORKSPACE_BWD)
+ */
+typedef struct ls_dsa_plan ls_dsa_plan_t;
+typedef struct {
+  int32_t R;                 /* response tokens */
+  int32_t num_q_heads;       /* attention heads that share the latent */
+  int32_t num_index_heads;   /* H_I (32 in the paper's configuration) */
+  int32_t index_dim;         /* 128 */
+  int32_t top_k;             /* positions kept per query (2,048 in the paper) */
+  int32_t reserved;
+  const void* ki_pool;
+  int64_t ki_stride_page, ki_stride_tok;
+  void* gathered;
+} ls_dsa_desc_t;
+size_t ls_dsa_gathered_bytes(const ls_pages_t* latent, const ls_dsa_desc_t* desc);
+ls_status_t ls_dsa_plan_create(const ls_pages_t* latent, const ls_dsa_desc_t* desc, ls_dsa_plan_t** out);
+ls_status_t ls_dsa_plan_destroy(ls_dsa_plan_t* plan);
+int32_t ls_dsa_selected_count(const ls_dsa_plan_t* plan);
+size_t ls_dsa_workspace_bytes(const ls_dsa_plan_t* plan, int which);
+ls_status_t ls_dsa_index_scores(const ls_dsa_plan_t* plan, const void* q_index, const float* w_index,
+                                float* scores, int32_t* status_dev, void* stream);
+ls_status_t ls_dsa_topk(const ls_dsa_plan_t* plan, const float* scores, int32_t* sel, void* stream);
+ls_status_t ls_dsa_attn_fwd(const ls_dsa_plan_t* plan, const int32_t* sel, float scale,
+                            const void* q, const void* k_resp, const void* v_resp,
+                            void* o_bf16, float* o_f32, float* lse,
+                            void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+ls_status_t ls_dsa_attn_bwd(const ls_dsa_plan_t* plan, float scale,
+                            const void* q, const void* k_resp, const void* v_resp,
+                            const float* o_f32, const float* lse, const void* d_o,
+                            void* dq, void* dk_resp, void* dv_resp,
+                            void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
 
 /*
  * ls_replay_attn_bwd for callers that cannot hand over scratch memory (the paper has no

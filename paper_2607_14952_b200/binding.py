@@ -37,6 +37,12 @@ class ls_attn_params_t(C.Structure):
                 ("generation", C.c_uint64)]
 
 
+class ls_dsa_desc_t(C.Structure):
+    _fields_ = [("R", C.c_int32), ("num_q_heads", C.c_int32), ("num_index_heads", C.c_int32),
+                ("index_dim", C.c_int32), ("top_k", C.c_int32), ("reserved", C.c_int32), ("ki_pool", C.c_void_p),
+                ("ki_stride_page", C.c_int64), ("ki_stride_tok", C.c_int64), ("gathered", C.c_void_p)]
+
+
 class LsError(RuntimeError):
     def __init__(self, status, where):
         self.status = status
@@ -68,6 +74,21 @@ def lib():
         L.ls_suffix_pages_reserve.argtypes = [vp, i32, i32, vp, vp]
         L.ls_suffix_pages_append.argtypes = [vp, i32, vp, vp, vp, vp]
         L.ls_suffix_pages_pop.argtypes = [vp]
+        L.ls_dsa_gathered_bytes.argtypes = [vp, C.POINTER(ls_dsa_desc_t)]
+        L.ls_dsa_gathered_bytes.restype = C.c_size_t
+        L.ls_dsa_plan_create.argtypes = [vp, C.POINTER(ls_dsa_desc_t), C.POINTER(vp)]
+        L.ls_dsa_plan_destroy.argtypes = [vp]
+        L.ls_dsa_selected_count.argtypes = [vp]
+        L.ls_dsa_selected_count.restype = C.c_int32
+        L.ls_dsa_workspace_bytes.argtypes = [vp, C.c_int]
+        L.ls_dsa_workspace_bytes.restype = C.c_size_t
+        L.ls_dsa_index_scores.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.ls_dsa_topk.argtypes = [vp, vp, vp, vp]
+        L.ls_dsa_attn_fwd.argtypes = [vp, vp, C.c_float, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+        L.ls_dsa_attn_bwd.argtypes = [vp, C.c_float, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+        for f in ("ls_dsa_plan_create", "ls_dsa_plan_destroy", "ls_dsa_index_scores", "ls_dsa_topk", "ls_dsa_attn_fwd",
+                  "ls_dsa_attn_bwd"):
+            getattr(L, f).restype = C.c_int
         L.ls_pages_generation.argtypes = [vp]
         L.ls_pages_generation.restype = C.c_uint64
         L.ls_suffix_pages_tokens.argtypes = [vp]
@@ -321,3 +342,84 @@ def ls_profile_arm_events(kernel, start_event, stop_event):
 def ls_selftest_bounded_wait(status, budget_ns):
     """Runs the bounded-wait self test; `status` is a zeroed int32 CUDA tensor."""
     _check(lib().ls_selftest_bounded_wait(_ptr(status), int(budget_ns), _stream()), "ls_selftest_bounded_wait")
+
+
+class DsaPlan:
+    """Owner of an ls_dsa_plan_t handle, of its gathered buffer and of references to the pools."""
+
+    def __init__(self, handle, pages, ki_pool, gathered, desc):
+        self.handle, self.pages, self.ki_pool, self.gathered, self.desc = handle, pages, ki_pool, gathered, desc
+        self.count = int(lib().ls_dsa_selected_count(handle))
+
+    def close(self):
+        if self.handle:
+            lib().ls_dsa_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def ls_dsa_plan_create(pages, ki_pool, R, num_q_heads, num_index_heads, top_k):
+    """ki_pool: bf16 CUDA tensor [num_phys_pages, page_size, index_dim] (indexer-key pages, same page
+    ids as the latent pool).  Allocates the gathered buffer with torch (device memory only)."""
+    d = ls_dsa_desc_t()
+    d.R, d.num_q_heads, d.num_index_heads, d.index_dim, d.top_k = R, num_q_heads, num_index_heads, ki_pool.shape[-1], top_k
+    assert ki_pool.dtype == torch.bfloat16 and ki_pool.stride(-1) == 1
+    d.ki_pool = ki_pool.data_ptr()
+    d.ki_stride_page, d.ki_stride_tok = ki_pool.stride(0), ki_pool.stride(1)
+    nbytes = int(lib().ls_dsa_gathered_bytes(pages.handle, C.byref(d)))
+    gathered = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=ki_pool.device)
+    d.gathered = gathered.data_ptr()
+    out = C.c_void_p()
+    _check(lib().ls_dsa_plan_create(pages.handle, C.byref(d), C.byref(out)), "ls_dsa_plan_create")
+    return DsaPlan(out, pages, ki_pool, gathered, d)
+
+
+def ls_dsa_index_scores(plan, q_index, w_index, scores=None, status=None):
+    """q_index [R, H_I, 128] bf16, w_index [R, H_I] fp32 -> scores [R, P] fp32."""
+    P = plan.pages.desc.prefix_len
+    if scores is None:
+        scores = torch.empty((plan.desc.R, P), dtype=torch.float32, device=q_index.device)
+    _check(lib().ls_dsa_index_scores(plan.handle, _ptr(q_index), _ptr(w_index), _ptr(scores), _ptr(status), _stream()),
+           "ls_dsa_index_scores")
+    return scores
+
+
+def ls_dsa_topk(plan, scores, sel=None):
+    """scores [R, P] fp32 -> sel [R, count] int32: the selected prefix positions, ascending."""
+    if sel is None:
+        sel = torch.empty((plan.desc.R, plan.count), dtype=torch.int32, device=scores.device)
+    _check(lib().ls_dsa_topk(plan.handle, _ptr(scores), _ptr(sel), _stream()), "ls_dsa_topk")
+    return sel
+
+
+def ls_dsa_attn_fwd(plan, sel, q, k_resp, v_resp, scale, status=None, workspace=None):
+    """Returns (o_bf16, o_f32, lse) of the sparse operator."""
+    R, Hq, _ = q.shape
+    dv = plan.pages.desc.dim_v
+    o_bf16 = torch.empty((R, Hq, dv), dtype=torch.bfloat16, device=q.device)
+    o_f32 = torch.empty((R, Hq, dv), dtype=torch.float32, device=q.device)
+    lse = torch.empty((R, Hq), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(int(lib().ls_dsa_workspace_bytes(plan.handle, LS_WORKSPACE_FWD)), dtype=torch.uint8,
+                                device=q.device)
+    _check(lib().ls_dsa_attn_fwd(plan.handle, _ptr(sel), float(scale), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_bf16),
+                                 _ptr(o_f32), _ptr(lse), _ptr(workspace), workspace.numel(), _ptr(status), _stream()),
+           "ls_dsa_attn_fwd")
+    return o_bf16, o_f32, lse
+
+
+def ls_dsa_attn_bwd(plan, q, k_resp, v_resp, o_f32, lse, d_o, scale, status=None, workspace=None):
+    """Returns (dq, dk_resp, dv_resp) with the selection of the plan's last forward held fixed."""
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k_resp), torch.empty_like(v_resp)
+    if workspace is None:
+        workspace = torch.empty(int(lib().ls_dsa_workspace_bytes(plan.handle, LS_WORKSPACE_BWD)), dtype=torch.uint8,
+                                device=q.device)
+    _check(lib().ls_dsa_attn_bwd(plan.handle, float(scale), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_f32), _ptr(lse),
+                                 _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace), workspace.numel(),
+                                 _ptr(status), _stream()), "ls_dsa_attn_bwd")
+    return dq, dk, dv

@@ -7,7 +7,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libls_replay.so")
-SOURCES = ["ls_pages.cu", "ls_merge.cu", "ls_fwd.cu", "ls_bwd.cu", "ls_bwd_mla.cu", "ls_bwd_mla_dq.cu"]
+SOURCES = ["ls_pages.cu", "ls_merge.cu", "ls_fwd.cu", "ls_bwd.cu", "ls_bwd_mla.cu", "ls_bwd_mla_dq.cu", "ls_dsa.cu"]
 
 
 def _nvcc():

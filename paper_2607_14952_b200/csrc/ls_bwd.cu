@@ -57,6 +57,7 @@ struct BwdParams {
   long long* timing;     // diagnostic builds only
   int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   int packed;    // dQ pass: one Q tile holds every (head, token) row of a KV group
+  int no_resp;   // dQ pass: the response block is left out
   // dK / dV pass: keys of a suffix block (1) read through pages [key_page_off, ..) of part_pages,
   // key_tokens of them, first gradient slot grad_slot0; or the response block (0)
   int keys_paged, key_page_off, key_tokens, grad_slot0;
@@ -585,7 +586,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = min(p.R, max(row0, row0_o) + 128);      // both CTAs walk the longer causal range
+    tokens = p.no_resp ? 0 : min(p.R, max(row0, row0_o) + 128);      // both CTAs walk the longer causal range
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -924,6 +925,10 @@ __global__ void dq_reduce_kernel(const float* __restrict__ dq_part, int parts, i
   }
 }
 
+void launch_delta(const void* d_o, const float* o_f32, int64_t rows, int dv, float* delta, cudaStream_t st) {
+  delta_kernel<<<(int)((rows + 7) / 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows, dv, delta);
+}
+
 template <int D, int MODE>
 static ls_status_t launch_kv(const BwdParams& prm, int grid, cudaStream_t st, bool timed) {
   using C = BwdCfg<D>;
@@ -1034,7 +1039,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = min(p.R, max(row0, row0_o) + 128);
+    tokens = p.no_resp ? 0 : min(p.R, max(row0, row0_o) + 128);
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -1338,7 +1343,10 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
                                           int32_t* status_dev, void* stream) {
   ls_status_t st = ls::check_handle(h, prm);
   if (st != LS_OK) return st;
-  if (!q || !k_resp || !v_resp || !o_f32 || !lse || !d_o || !dq || !dk_resp || !dv_resp) return LS_ERR_INVALID_ARG;
+  const bool no_resp = (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) != 0;
+  if (!q || !o_f32 || !lse || !d_o || !dq) return LS_ERR_INVALID_ARG;
+  if (!no_resp && (!k_resp || !v_resp || !dk_resp || !dv_resp)) return LS_ERR_INVALID_ARG;
+  if (no_resp) k_resp = v_resp = q;                    // response maps are encoded but never used
   const ls_pages_desc_t& d = h->desc;
   if (prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % d.num_kv_heads != 0) return LS_ERR_INVALID_ARG;
   if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;
@@ -1364,11 +1372,14 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   const int parts = h->num_parts();
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
-  ls::delta_kernel<<<(int)((rows + 7) / 8), 256, 0, cs>>>(static_cast<const __nv_bfloat16*>(d_o), o_f32, rows,
-                                                        d.dim_v, delta);
+  ls::launch_delta(d_o, o_f32, rows, d.dim_v, delta, cs);
 
   if (mla) {
     const bool mla_fast = ls::mla_dq_fast(h);
+    if (no_resp) {       // prefix parts only: the transposed kernel walks them all and writes dQ
+      if (!mla_fast) return LS_ERR_UNSUPPORTED_SHAPE;
+      return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, nullptr, dq, status_dev, cs);
+    }
     ls_status_t ms =
         ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_acc, dk_resp, dv_resp, mla_fast, status_dev, cs);
     if (ms != LS_OK) return ms;
@@ -1412,6 +1423,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   P.scale_log2 = prm->scale * ls::kLog2e;
 
   // ---- dQ: rows = queries, columns = keys of every part, summed through the running dQ
+  P.no_resp = no_resp ? 1 : 0;
   P.packed = 0;
   if (g > 1 && g * R <= 128) {           // short response: all rows of a KV group in one Q tile
     P.packed = 1;
@@ -1467,6 +1479,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
                     : ls::launch_kv<256, ls::MODE_DV>(P, grid_b, cs, false);
     if (st != LS_OK) return st;
   }
+  if (no_resp) return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
   // keys of the response block itself (causal); with LS_FLAG_ADD_SUFFIX_GRAD the gradient pages that later
   // blocks left for this block (its slots start where the suffix now ends) are added
   P.keys_paged = 0;

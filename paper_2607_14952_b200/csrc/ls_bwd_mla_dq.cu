@@ -40,7 +40,7 @@ struct MlaDqParams {
   const int64_t* shard_tokens;
   const float* lse;
   const float* delta;
-  const float* dq_resp;              // [R, Hq, 576] fp32, unscaled: the response block's part
+  const float* dq_resp;              // [R, Hq, 576] fp32, unscaled: the response block's part (NULL: none)
   __nv_bfloat16* dq;                 // [R, Hq, 576]
   int32_t* status;
   long long* timing;   // diagnostic builds only
@@ -403,7 +403,7 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
               const int r = row0 + half * 32 + j;
               if (r < p.R) {
                 const size_t idx = ((size_t)r * p.Hq + h) * 576 + ch;
-                p.dq[idx] = __float2bfloat16_rn((__uint_as_float(o[j]) + p.dq_resp[idx]) * p.scale);
+                p.dq[idx] = __float2bfloat16_rn((__uint_as_float(o[j]) + (p.dq_resp ? p.dq_resp[idx] : 0.f)) * p.scale);
               }
             }
           }

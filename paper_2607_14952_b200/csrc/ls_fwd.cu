@@ -54,6 +54,7 @@ struct FwdParams {
   long long* timing;   // diagnostic builds only
   int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   int chain_mode, fine;
+  int no_resp;    // 1: the response block is left out (its partial is written as empty)
   int dv_total;   // channels of one output row (DVT times the number of O tiles)
   int packed;     // 1: one Q tile holds every (head, token) row of a KV group (g * R <= 128 rows);
                   //    row r is head r / R, token r % R.  Lets a short response stream K/V once.
@@ -264,7 +265,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = min(p.R, t0 + 128);                       // keys 0 .. last row of this tile
+    tokens = p.no_resp ? 0 : min(p.R, t0 + 128);       // keys 0 .. last row of this tile (none when the block is left out)
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -506,7 +507,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         if (i == 0) {
           m_ref = (mx == -INFINITY) ? 0.f : mx;
-        } else if (__any_sync(0xffffffffu, mx > m_ref + thresh)) {
+        } else if (__any_sync(0xffffffffu, row_ok && mx > m_ref + thresh)) {   // (rows outside the tile hold stale bytes: they must not steer the warp)
           // rare: raise the reference maximum and rescale the running sum and O
           ok = LS_TWAIT(tw1, mbar_wait_warp(pv_done, (i - 1) & 1, abort_flag));
           if (!ok) break;
@@ -669,7 +670,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = min(p.R, max(t0, t0_o) + 128);          // both CTAs walk the longer causal range
+    tokens = p.no_resp ? 0 : min(p.R, max(t0, t0_o) + 128);   // both CTAs walk the longer causal range
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -847,7 +848,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
         const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         if (i == 0) {
           m_ref = (mx == -INFINITY) ? 0.f : mx;
-        } else if (__any_sync(0xffffffffu, mx > m_ref + thresh)) {
+        } else if (__any_sync(0xffffffffu, row_ok && mx > m_ref + thresh)) {   // (rows outside the tile hold stale bytes: they must not steer the warp)
           // rare: raise the reference maximum and rescale the running sum and O (this CTA's rows)
           ok = mbar_wait_warp(pv_done, (i - 1) & 1, abort_flag);
           if (!ok) break;
@@ -979,6 +980,7 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
   const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
   const bool small_pages = d.page_size == 64;
   const bool pair = d.dim_k == 256 && !f.packed;            // CTA pairs share every key tile between two Q tiles
+  if (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) k_resp = v_resp = q;   // the response maps are encoded but never used
   ls_status_t st = f.packed ? encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, R, f.g)
                             : encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, 128, 1);
   if (pair) {
@@ -1027,6 +1029,7 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.dv_total = d.dim_v;
   P.chain_mode = mode;
+  P.no_resp = (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) ? 1 : 0;
   P.fine = h->fine;
   P.ablate = prm->flags & LS_DBG_ABLATE_MASK;
   P.scale = prm->scale;
@@ -1051,7 +1054,8 @@ static ls_status_t check_forward_args(const ls_pages* h, const ls_attn_params_t*
                                       const void* k_resp, const void* v_resp) {
   ls_status_t st = check_handle(h, prm);
   if (st != LS_OK) return st;
-  if (!q || !k_resp || !v_resp) return LS_ERR_INVALID_ARG;
+  const bool no_resp = (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) != 0;
+  if (!q || (!no_resp && (!k_resp || !v_resp))) return LS_ERR_INVALID_ARG;
   const ls_pages_desc_t& d = h->desc;
   if (prm->R < 1 || prm->num_q_heads < 1 || prm->num_q_heads % d.num_kv_heads != 0) return LS_ERR_INVALID_ARG;
   if (!(prm->scale > 0.f)) return LS_ERR_INVALID_ARG;

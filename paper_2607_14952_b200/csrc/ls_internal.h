@@ -156,6 +156,9 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
 // True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix).
 bool mla_dq_fast(const ls_pages* h);
 
+// Delta[t,h] = dO[t,h] . O[t,h] (fp32), one warp per row.
+void launch_delta(const void* d_o, const float* o_f32, int64_t rows, int dv, float* delta, cudaStream_t st);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int pg_shift_of(int page_size) { return page_size == 64 ? 6 : page_size == 128 ? 7 : page_size == 256 ? 8 : 9; }

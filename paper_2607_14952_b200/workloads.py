@@ -138,6 +138,20 @@ def make_prefix(cfg, device="cpu", extra_phys_pages=0, permute=True):
     return k_pool, v_pool, table
 
 
+def make_index_inputs(cfg, num_index_heads, member=0, device="cpu", index_dim=128, num_phys_pages=None):
+    """Indexer side of the sparse (DSA) replay (Eq. dsa-index): indexer-key pages
+    [num_phys_pages, page_size, index_dim] bf16 (seed base+4; they follow the latent's page table),
+    the member's indexer queries [R, H_I, index_dim] bf16 and head weights [R, H_I] fp32."""
+    nphys = cfg.num_pages if num_phys_pages is None else num_phys_pages
+    ki_pool = _randn_bf16((nphys, cfg.page_size, index_dim), cfg.seed + 4, device)
+    s = member_seed(cfg, member)
+    q_index = _randn_bf16((cfg.R, num_index_heads, index_dim), s + 4, device)
+    g = torch.Generator(device=device)
+    g.manual_seed(s + 5)
+    w_index = torch.randn((cfg.R, num_index_heads), generator=g, device=device, dtype=torch.float32)
+    return ki_pool, q_index, w_index
+
+
 def bf16_bits(t):
     """torch bf16 tensor -> numpy uint16 bit patterns (host copy)."""
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view(np.uint16)

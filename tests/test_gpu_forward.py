@@ -93,6 +93,21 @@ def test_merged_forward_is_bit_reproducible_and_close_to_the_two_step_path():
         assert (a[0].float() - o_bf16.float()).abs().max() <= 2.0 ** -8 * o_bf16.float().abs().max()
 
 
+def test_packed_tiles_are_bit_reproducible_after_other_work():
+    # a packed short-response tile fills only g * R of the 128 Q rows; the rest of the tile holds
+    # whatever the previous CTA left in shared memory and must not influence the real rows
+    cfg = small("packed_det", P=4096, page_size=256, num_shards=4, R=3, Hq=24, Hkv=4)
+    case = parity.Case(cfg)
+    q, k, v, _ = case.member(0)
+    a = case.forward(q, k, v)
+    other = parity.Case(small("noise", P=2048, R=256, seed=5))      # different bytes through the same SMs
+    oq, ok_, ov, _ = other.member(0)
+    other.forward(oq * 37.0, ok_ * 11.0, ov)
+    b = case.forward(q, k, v)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
 def test_forward_split_count_does_not_change_the_merge():
     outs = []
     for S in (1, 2, 4, 8, 32):
