@@ -12,6 +12,7 @@ data path, weak scaling.  `--gpus N` without a torchrun environment starts the N
   --mode replay   forward (per-shard partials) + merge + backward              (default)
   --mode fused    forward with the merge folded in + backward
   --mode score    forward with the merge folded in only (a score-only pass)
+  --mode dsa      sparse replay over the 576/512 latent (index scores, top-2048, attention fwd + bwd)
   --blocks B      blockwise replay of the response in B blocks with a paged suffix: a no-grad
                   suffix pass (score + append per block), then the blocks in reverse (pop,
                   forward, backward with gradient pages)
@@ -365,6 +366,86 @@ def run_cuda(args):
         torch.distributed.destroy_process_group()
 
 
+def run_dsa(args):
+    """Sparse (DSA) replay over the shared latent: index scores -> global top-k -> attention over the
+    selected rows + the causal response block -> backward.  One step = one member; 1 GPU."""
+    from paper_2607_14952_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    cfg = W.CONFIGS["mla1m"]
+    if args.prefix:
+        cfg = W.scaled(cfg, name="%s-P%d" % (cfg.name, args.prefix), P=args.prefix)
+    HI, TOPK = 32, 2048
+    torch.cuda.reset_peak_memory_stats(dev)
+    k_pool, _, table = W.make_prefix(cfg, dev)
+    pages = B.ls_prefix_pages_build(cfg.P, cfg.page_size, cfg.num_shards, cfg.Hkv, cfg.Dk, cfg.Dv, k_pool.shape[0],
+                                    page_table=table, k_pool=k_pool, v_aliases_k=True)
+    members = []
+    for m in range(2):
+        ki_pool, q_index, w_index = W.make_index_inputs(cfg, HI, m, dev)
+        q, kr, _, d_o = W.make_member(cfg, m, dev)
+        members.append((q_index, w_index, q, kr, kr[..., :cfg.Dv].contiguous(), d_o))
+    plan = B.ls_dsa_plan_create(pages, ki_pool, cfg.R, cfg.Hq, HI, TOPK)
+    count = plan.count
+    scores = torch.empty((cfg.R, cfg.P), dtype=torch.float32, device=dev)
+    sel = torch.empty((cfg.R, count), dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws_f = torch.empty(int(B.lib().ls_dsa_workspace_bytes(plan.handle, B.LS_WORKSPACE_FWD)), dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(int(B.lib().ls_dsa_workspace_bytes(plan.handle, B.LS_WORKSPACE_BWD)), dtype=torch.uint8, device=dev)
+    names = ("index_scores", "topk", "attn_fwd", "attn_bwd")
+
+    def step(m, ev=None):
+        q_index, w_index, q, kr, vr, d_o = m
+        mark = (lambda i: ev[i].record()) if ev else (lambda i: None)
+        mark(0)
+        B.ls_dsa_index_scores(plan, q_index, w_index, scores=scores, status=status)
+        mark(1)
+        B.ls_dsa_topk(plan, scores, sel=sel)
+        mark(2)
+        _, o_f32, lse = B.ls_dsa_attn_fwd(plan, sel, q, kr, vr, cfg.scale, status=status, workspace=ws_f)
+        mark(3)
+        B.ls_dsa_attn_bwd(plan, q, kr, vr, o_f32, lse, d_o, cfg.scale, status=status, workspace=ws_b)
+        mark(4)
+
+    for w in range(args.warmup):
+        step(members[w % 2])
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    for i in range(args.steps):
+        step(members[i % 2], evs[i])
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if int(status.item()) != 0:
+        raise RuntimeError("device status %d" % int(status.item()))
+    phase_ms = {n: float(np.mean([e[j].elapsed_time(e[j + 1]) for e in evs])) for j, n in enumerate(names)}
+    step_ms = [e[0].elapsed_time(e[4]) for e in evs]
+    pairs = cfg.Hq * cfg.R * count + cfg.Hq * cfg.R * (cfg.R + 1) // 2
+    f_index = 2 * cfg.R * HI * cfg.P * 128
+    f_fwd = 2 * (cfg.Dk + cfg.Dv) * pairs
+    f_bwd = 2 * (2 * cfg.Dk + cfg.Dv) * pairs + 2 * (cfg.Dk + cfg.Dv) * cfg.Hq * cfg.R * (cfg.R + 1) // 2
+    flops = f_index + f_fwd + f_bwd
+    peaks = measured_peaks()
+    ms = float(np.mean(step_ms))
+    idx_tflops = f_index / (phase_ms["index_scores"] * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "ms_per_step_best": min(step_ms),
+        "ms_per_step_median": float(np.median(step_ms)), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "%s sparse: P=%d R=%d Hq=%d latent 576/512, %d index heads of 128, top-%d" % (
+            cfg.name, cfg.P, cfg.R, cfg.Hq, HI, TOPK), "mode": "dsa (index scores, top-k, sparse attention fwd + bwd)",
+            "flops_per_step": flops, "flops_index": f_index, "flops_attention": f_fwd + f_bwd, "phase_ms": phase_ms,
+            "l2": "indexer-key pages %.2f GiB + scores %.2f GiB streamed per step" % (
+                ki_pool.numel() * 2 / 2**30, scores.numel() * 4 / 2**30)},
+        "clocks": clocks, "gpu_launches": 11 * args.steps, "peak_device_bytes": torch.cuda.max_memory_allocated(dev),
+        "roofline": {"bound": "tensor", "kernel": "dsa_index_kernel (index scores, Eq. dsa-index)", "achieved": idx_tflops,
+                     "peak": peaks["bf16_tflops_sustained"], "unit": UNIT, "frac": idx_tflops / peaks["bf16_tflops_sustained"],
+                     "peak_source": "%s sustained bf16 cuBLAS" % peaks["source"], "ms_per_launch": phase_ms["index_scores"],
+                     "traffic": measured_traffic("dsa_index_kernel", cfg.name), "algorithmic_flops_per_launch": f_index}}))
+
+
 def _cpu_sample_inputs(cfg):
     """Inputs of ONE KV head on the host, drawn with the CPU generator (same distributions)."""
     one = W.scaled(cfg, Hkv=1, Hq=cfg.Hq // cfg.Hkv, needles=0)
@@ -445,13 +526,15 @@ def main():
     ap.add_argument("--prefix", type=int, default=0, help="override the workload's prefix length (profiling on a small case)")
     ap.add_argument("--stream-budget-kib", type=int, default=0,
                     help="K+V bytes of one (KV head, key range) stream, in KiB (0 = the library's default)")
-    ap.add_argument("--mode", default="replay", choices=["replay", "fused", "score"])
+    ap.add_argument("--mode", default="replay", choices=["replay", "fused", "score", "dsa"])
     ap.add_argument("--blocks", type=int, default=0, help="blockwise replay with a paged suffix in this many blocks")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "dsa":
+        run_dsa(args)
     elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(launch_ranks(args))
     else:

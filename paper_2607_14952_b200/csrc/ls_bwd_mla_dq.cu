@@ -45,6 +45,9 @@ struct MlaDqParams {
   int32_t* status;
   long long* timing;   // diagnostic builds only
   int R, Hq, g, nparts, pg_shift, tiles_per_head, num_phys_pages;
+  int packed;      // 1: a CTA's 64 rows are every (head, token) row of one KV group (g * R <= 64 rows; row r is
+                   //    head r / R, token r % R) instead of 64 tokens of one head
+  int qdo_bytes;   // bytes the Q and dO loads deliver
   int ablate;   // diagnostic builds only: 1 = no key loads, 2 = no tensor-core instructions
   float scale, scale_log2;
 };
@@ -93,8 +96,9 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   long long tw0 = 0, tw1 = 0, tw2 = 0, tw3 = 0;   // wait-time accumulators (only used with LS_TIMING)
   const long long t_begin = clock64();
-  const int h = blockIdx.x / p.tiles_per_head;
-  const int row0 = (blockIdx.x % p.tiles_per_head) * kTqRows;
+  // 64 tokens of one head, or (packed) all rows of one KV group
+  const int h = p.packed ? blockIdx.x * p.g : blockIdx.x / p.tiles_per_head;      // (first) head of the block
+  const int row0 = p.packed ? 0 : (blockIdx.x % p.tiles_per_head) * kTqRows;
   const int kvh = h / p.g;
 
   // key tiles of 128 over all partials (every role walks the same list)
@@ -117,7 +121,8 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
   }
   if (threadIdx.x >= 64 && threadIdx.x < 64 + kTqRows) {
     const int t = threadIdx.x - 64;
-    const size_t ri = (size_t)min(row0 + t, p.R - 1) * p.Hq + h;
+    const size_t ri = p.packed ? (size_t)(t % p.R) * p.Hq + h + min(t / p.R, p.g - 1)
+                               : (size_t)min(row0 + t, p.R - 1) * p.Hq + h;
     rowp[t] = make_float2(p.lse[ri] * kLog2eTq, p.delta[ri]);
   }
   if (warp == 1) {
@@ -138,7 +143,7 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
     // groups, one box) for dQ^T.  The dQ^T loads of tile i are interleaved one to one with the
     // [S^T | T^T] loads of tile i + 2, the order in which the two issuers consume them.
     if (lane == 0 && total_tiles > 0) {
-      mbar_arrive_expect_tx(a_full, kTqQdo);
+      mbar_arrive_expect_tx(a_full, p.qdo_bytes);
       for (int c = 0; c < 9; ++c) tma_load_5d(qdo + c * 16384, &p.q_map, a_full, 0, row0, c, h, 0);
       for (int c = 0; c < 8; ++c) tma_load_5d(qdo + c * 16384 + 8192, &p.do_map, a_full, 0, row0, c, h, 0);
 
@@ -400,9 +405,11 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
             tc_wait_ld32(o);
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int r = row0 + half * 32 + j;
-              if (r < p.R) {
-                const size_t idx = ((size_t)r * p.Hq + h) * 576 + ch;
+              const int rr = half * 32 + j;                    // row of the block
+              const int r = p.packed ? rr % p.R : row0 + rr;   // its token and head
+              const int hh = p.packed ? h + rr / p.R : h;
+              if (p.packed ? rr < p.g * p.R : r < p.R) {
+                const size_t idx = ((size_t)r * p.Hq + hh) * 576 + ch;
                 p.dq[idx] = __float2bfloat16_rn((__uint_as_float(o[j]) + (p.dq_resp ? p.dq_resp[idx] : 0.f)) * p.scale);
               }
             }
@@ -454,8 +461,15 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   P.timing = g_timing_buffer;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * kLog2eTq;
-  ls_status_t st = encode_map5(&P.q_map, q, 576, R, Hq, 1, (int64_t)Hq * 576, 576, (int64_t)R * Hq * 576, 64, 1);
-  if (st == LS_OK) st = encode_map5(&P.do_map, d_o, 512, R, Hq, 1, (int64_t)Hq * 512, 512, (int64_t)R * Hq * 512, 64, 1);
+  // a short response packs every (head, token) row of a KV group into the CTA's 64 rows
+  P.packed = (P.g > 1 && P.g * R <= kTqRows) ? 1 : 0;
+  const int rows_loaded = P.packed ? P.g * R : kTqRows;
+  P.qdo_bytes = (9 + 8) * rows_loaded * 128;
+  ls_status_t st = P.packed ? encode_map_rows(&P.q_map, q, 576, R, Hq, R, P.g)
+                            : encode_map5(&P.q_map, q, 576, R, Hq, 1, (int64_t)Hq * 576, 576, (int64_t)R * Hq * 576, 64, 1);
+  if (st == LS_OK)
+    st = P.packed ? encode_map_rows(&P.do_map, d_o, 512, R, Hq, R, P.g)
+                  : encode_map5(&P.do_map, d_o, 512, R, Hq, 1, (int64_t)Hq * 512, 512, (int64_t)R * Hq * 512, 64, 1);
   if (st == LS_OK) st = pool_map(&P.k_map, h, 0, 64, 1, false);
   if (st == LS_OK) st = pool_map(&P.k_tail, h, 0, 64, 1, true);
   if (st == LS_OK) st = pool_map(&P.k2_map, h, 0, 64, 2, false);
@@ -464,7 +478,7 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   static bool configured[64] = {};
   const ls_status_t cfg = configure_smem(bwd_mla_dq_kernel, kTqSmem, configured);
   if (cfg != LS_OK) return cfg;
-  const int64_t grid = (int64_t)Hq * P.tiles_per_head;
+  const int64_t grid = P.packed ? (int64_t)d.num_kv_heads : (int64_t)Hq * P.tiles_per_head;
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   profile_begin(LS_KERNEL_BWD_DQ, cs);
   bwd_mla_dq_kernel<<<(int)grid, kTqThreads, kTqSmem, cs>>>(P);

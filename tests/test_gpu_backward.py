@@ -44,6 +44,9 @@ def test_config1_tiny_full():
     small("short_r16", P=4096, page_size=256, num_shards=4, R=16, Hq=24, Hkv=4),
     small("short_r1", P=1500, page_size=64, num_shards=3, R=1, Hq=8, Hkv=2, Dk=128, Dv=128),
     small("short_r32_full_tile", P=2048, page_size=256, num_shards=2, R=32, Hq=8, Hkv=2),
+    small("mla_short_r3", Dk=576, Dv=512, v_aliases_k=True, Hq=16, Hkv=1, P=64 * 11 + 7, page_size=64, num_shards=2, R=3),
+    small("mla_short_r1_64heads", Dk=576, Dv=512, v_aliases_k=True, Hq=64, Hkv=1, P=256 * 5 + 9, page_size=256,
+          num_shards=3, R=1),
 ], ids=lambda c: c.name)
 def test_backward_small_cases(cfg):
     case = parity.Case(cfg, extra_phys_pages=2)
