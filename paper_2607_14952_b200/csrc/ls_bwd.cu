@@ -34,7 +34,11 @@ enum { MODE_DK = 1, MODE_DV = 2 };
 
 struct BwdParams {
   CUtensorMap a1_map, a2_map;                 // stationary rows: box 64 x 128 tokens x 1 group
-  CUtensorMap b1r_map, b2r_map, b3r_map;      // dK / dV pass: Q / dO / (Q | dO) as 128 columns x 128 channels
+  CUtensorMap b1r_map, b2r_map, b3r_map;      // dK / dV pass: Q / dO / (Q | dO) as 128 columns x 128 channels;
+                                              // single-CTA dQ pass: response K / V the same way
+  // single-CTA dQ pass: pool K and V as chunks of 128 keys x 128 channels (box 64 x 128 tokens x 2 groups,
+  // or 64 x 64 x 1 on 64-token pages: four boxes per chunk)
+  CUtensorMap bk_map, bk_tail, bv_map, bv_tail;
   // dQ pass on CTA pairs: each CTA loads half of every streamed operand.
   //   *_s: 64 columns x 128 channels (box 64 x 64 tokens x 2 groups)
   //   *_m: 128 columns x 64 channels (box 64 x 128 x 1, or 64 x 64 x 1 on 64-token pages)
@@ -885,6 +889,316 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   }
 }
 
+
+// ---------------------------------------------------------------------------------
+// dQ pass for short responses (g * R <= 128): every (head, token) row of a KV group sits in ONE
+// Q tile, so a (KV head, part) is one work item and its K/V pages are read once: the pass is
+// bound by HBM, not by the tensor pipe.  A single CTA per item (a pair would spend half of every
+// 256-row MMA on rows that do not exist), 128-key tiles, E written over T so that the tensor pipe
+// runs S(i+1) while the row threads form E(i):   S(0) T(0) | S(i+1)  ACC(i)  T(i+1) | ...
+// TMEM: ACC [0, D), S [D, D+128), T [D+128, D+256).  Chunks of 32 KB: 128 keys x 128 channels.
+// ---------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_constant__ BwdParams p) {
+  using C = BwdCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a1_smem = smem;
+  uint8_t* a2_smem = smem + C::SLABS * 16384;
+  uint8_t* ring = smem + C::A_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kBwdChunk);
+  uint64_t* a_full = bars;
+  uint64_t* full = bars + 1;
+  uint64_t* empty = full + C::RING;
+  uint64_t* s_full = empty + C::RING;    // S of a tile is in TMEM
+  uint64_t* s_read = s_full + 1;         // every row thread has pulled S
+  uint64_t* t_full = s_read + 1;         // T of a tile is in TMEM
+  uint64_t* e_full = t_full + 1;         // [4] quarter q of E is in TMEM
+  uint64_t* acc_final = e_full + 4;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* work_idx = const_cast<int*>(abort_flag) + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(a_full, 1);
+    for (int i = 0; i < C::RING; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    mbar_init(s_full, 1);
+    mbar_init(s_read, 256);
+    mbar_init(t_full, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 256);
+    mbar_init(acc_final, 1);
+    *abort_flag = 0;
+    *work_idx = atomicAdd(p.ctl, 1);      // work items in launch order of the CTAs that ask (see chain_wait)
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_holder, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const uint32_t tmem_acc = tmem_base;
+  const uint32_t tmem_s = tmem_base + D;
+  const uint32_t tmem_t = tmem_base + D + 128;
+
+  // ---- work item: (KV head, link); the one packed Q tile of the KV group
+  const DqItem it = dq_item(p, *work_idx, 1);
+  const int part = it.part, kvh = it.kvh;
+  const bool is_resp = it.is_resp;
+  const int h = kvh * p.g;
+  int64_t tokens;
+  int page_off = 0, n_pages = 0, tail_slot = -1;
+  if (is_resp) {
+    tokens = p.no_resp ? 0 : p.R;
+  } else {
+    tokens = p.part_tokens[part];
+    page_off = p.part_page_offset[part];
+    n_pages = p.part_page_offset[part + 1] - page_off;
+    tail_slot = p.part_tail_slot[part];
+  }
+  const int n_tiles = (int)((tokens + 127) / 128);
+
+  if (warp == 0) {
+    // =========================================================== producer (one thread)
+    if (lane == 0 && n_tiles > 0) {
+      mbar_arrive_expect_tx(a_full, 2 * C::SLABS * p.g * p.R * 128);
+      for (int c = 0; c < C::SLABS; ++c) {
+        tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, 0, c, h, 0);
+        tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, 0, c, h, 0);
+      }
+      const int32_t* pages = p.part_pages + page_off;
+      const int pg_mask = (1 << p.pg_shift) - 1;
+      const bool small_pages = !is_resp && p.pg_shift == 6;   // a 128-key tile spans two 64-token pages
+      auto fetch = [&](int ps) -> int {
+        if (is_resp) return 0;
+        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
+      };
+      uint32_t slot = 0, phase = 0, issued = 0;
+      bool ok = true;
+      // one chunk: 128 keys x channels [128 c, 128 c + 128) of K (which = 0) or V (1)
+      auto load = [&](int which, int i, int c, int pa, int pb) {
+        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
+        if (ok) {
+          mbar_arrive_expect_tx(&full[slot], kBwdChunk);
+          uint8_t* dst = ring + slot * kBwdChunk;
+          const int tok = i * 128;
+          if (is_resp) {
+            tma_load_5d(dst, which ? &p.b2r_map : &p.b1r_map, &full[slot], 0, tok, 2 * c, kvh, 0);
+          } else if (!small_pages) {
+            const bool tail = (tok >> p.pg_shift) == tail_slot;
+            const CUtensorMap* m = which ? (tail ? &p.bv_tail : &p.bv_map) : (tail ? &p.bk_tail : &p.bk_map);
+            tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 2 * c, kvh, pa);
+          } else {
+            const int sa = tok >> 6;
+            const CUtensorMap* ma = which ? (sa == tail_slot ? &p.bv_tail : &p.bv_map) : (sa == tail_slot ? &p.bk_tail : &p.bk_map);
+            const CUtensorMap* mb = which ? (sa + 1 == tail_slot ? &p.bv_tail : &p.bv_map)
+                                          : (sa + 1 == tail_slot ? &p.bk_tail : &p.bk_map);
+            for (int s2 = 0; s2 < 2; ++s2) {
+              tma_load_5d(dst + s2 * 16384, ma, &full[slot], 0, 0, 2 * c + s2, kvh, pa);
+              tma_load_5d(dst + s2 * 16384 + 8192, mb, &full[slot], 0, 0, 2 * c + s2, kvh, pb);
+            }
+          }
+        }
+        ++issued;
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      auto load_op = [&](int which, int i, int pa, int pb) {
+        for (int c = 0; c < C::NC; ++c) load(which, i, c, pa, pb);
+      };
+      const int sh = small_pages ? 1 : (p.pg_shift - 7);
+      auto slot_of = [&](int i) { return small_pages ? 2 * i : (i >> sh); };
+      int pa0 = fetch(slot_of(0)), pb0 = small_pages ? fetch(1) : pa0;
+      int pa1 = fetch(slot_of(1)), pb1 = small_pages ? fetch(3) : pa1;
+      // chunk order = consumption order: S(0) T(0) [S(i+1) ACC(i) T(i+1)] ...; ACC re-reads K
+      load_op(0, 0, pa0, pb0);
+      load_op(1, 0, pa0, pb0);
+      for (int i = 0; i < n_tiles; ++i) {
+        const int pa2 = fetch(slot_of(i + 2)), pb2 = small_pages ? fetch(2 * i + 5) : pa2;
+        if (i + 1 < n_tiles) load_op(0, i + 1, pa1, pb1);
+        load_op(0, i, pa0, pb0);
+        if (i + 1 < n_tiles) load_op(1, i + 1, pa1, pb1);
+        pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
+      }
+      if (*abort_flag) {   // aborted: wait (bounded) for the copies already started
+        for (uint32_t s2 = 0; s2 < (uint32_t)C::RING && s2 < issued; ++s2) {
+          const uint32_t last = ((issued - 1 - s2) / C::RING) * C::RING + s2;
+          const uint64_t t_start = globaltimer_ns();
+          while (!mbar_try_wait(&full[s2], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer (one thread)
+    if (lane == 0 && n_tiles > 0) {
+      constexpr uint32_t idesc_st = make_idesc(128, 128, 0, 0);
+      constexpr uint32_t idesc_acc = make_idesc(128, 128, 0, 1);
+      constexpr uint32_t hi = sdesc_hi(1024);
+      const uint32_t a1_lo = sdesc_lo(smem_u32(a1_smem), 16), a2_lo = sdesc_lo(smem_u32(a2_smem), 16);
+      const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);       // K-major view of a chunk
+      const uint32_t ring_m_lo = sdesc_lo(smem_u32(ring), 16384);    // MN-major view: 16 KB group pitch
+      uint32_t slot = 0, phase = 0;
+      bool ok = mbar_wait(a_full, 0, abort_flag);
+      auto advance = [&]() {
+        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+      };
+      auto issue_op = [&](int op) {       // S = Q K^T (0) or T = dO V^T (1)
+        const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
+        const uint32_t d = op == 0 ? tmem_s : tmem_t;
+#pragma unroll
+        for (int c = 0; c < C::NC; ++c) {
+          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
+          const uint32_t b_lo = ring_k_lo + slot * (kBwdChunk >> 4);
+#pragma unroll
+          for (int s2 = 0; s2 < 2; ++s2)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              mma_ss(d, sdesc(a_lo + (((2 * c + s2) * 16384 + k * 32) >> 4), hi),
+                     sdesc(b_lo + ((s2 * 16384 + k * 32) >> 4), hi), idesc_st, (c | s2 | k) != 0);
+          mma_commit(&empty[slot]);
+          advance();
+        }
+        mma_commit(op == 0 ? s_full : t_full);
+      };
+      auto issue_acc = [&](int i) {
+        uint32_t cs[C::NC], cph[C::NC];
+#pragma unroll
+        for (int c = 0; c < C::NC; ++c) {
+          cs[c] = slot;
+          cph[c] = phase;
+          advance();
+        }
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          ok = ok && mbar_wait(&e_full[qd], i & 1, abort_flag);
+          if (!ok) return;
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < C::NC; ++c) {
+            if (qd == 0) {
+              ok = ok && mbar_wait(&full[cs[c]], cph[c], abort_flag);
+              if (!ok) return;
+              tc_fence_after();
+            }
+            const uint32_t b_lo = ring_m_lo + cs[c] * (kBwdChunk >> 4);
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk)
+              mma_ts(tmem_acc + c * 128, tmem_t + (2 * qd + kk) * 8, sdesc(b_lo + (((2 * qd + kk) * 2048) >> 4), hi),
+                     idesc_acc, (i | qd | kk) != 0);
+            if (qd == 3) mma_commit(&empty[cs[c]]);
+          }
+        }
+        if (i == n_tiles - 1) mma_commit(acc_final);
+      };
+      if (ok) issue_op(0);
+      if (ok) issue_op(1);
+      for (int i = 0; i < n_tiles && ok; ++i) {
+        if (i + 1 < n_tiles) {
+          ok = ok && mbar_wait(s_read, i & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          issue_op(0);
+        }
+        if (ok) issue_acc(i);
+        if (ok && i + 1 < n_tiles) issue_op(1);
+      }
+    }
+  } else {
+    // =========================================================== elementwise + epilogue
+    const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const int row = quad * 32 + lane;
+    const int r_idx = row % p.R;                          // token of this packed row
+    const int hr = h + min(row / p.R, p.g - 1);           // and its head
+    const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
+    const bool row_ok = row < p.g * p.R;
+    const size_t ri = (size_t)r_idx * p.Hq + hr;
+    bool ok = true;
+    if (n_tiles > 0) {
+      const float lse2_row = p.lse[ri] * kLog2e;
+      const float delta_row = p.delta[ri];
+      const int64_t lim = is_resp ? (int64_t)r_idx : tokens - 1;
+      for (int i = 0; i < n_tiles; ++i) {
+        const int key0 = i * 128;
+        const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim);
+        // No thread leaves this loop on its own: a wait that gave up is remembered in `ok` and put
+        // to the vote at the tile's named barrier, where all 256 leave together.
+        ok = ok && mbar_wait(s_full, i & 1, abort_flag);
+        tc_fence_after();
+        uint32_t sr[64];
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr + 16 * qd);
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(sr + 16 * qd);
+        tc_fence_before();
+        mbar_arrive(s_read);                 // S is in registers: the next tile's S may overwrite the buffer
+        float pr[64];
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
+          if (edge && (int64_t)key0 + 32 * (j >> 4) + 16 * half + (j & 15) > lim) e = 0.f;
+          pr[j] = e;
+        }
+        ok = ok && mbar_wait(t_full, i & 1, abort_flag);
+        tc_fence_after();
+        uint32_t tr[64];
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr + 16 * qd);
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(tr + 16 * qd);
+        // E (bf16) goes over T's columns, which the row's other thread reads too: every T read of the
+        // CTA comes before any E write (named barrier 1, which also carries the vote)
+        ok = bar_and(1, 256, ok);
+        if (!ok) break;
+#pragma unroll
+        for (int qd = 0; qd < 4; ++qd) {
+          uint32_t pk[8];
+#pragma unroll
+          for (int j = 0; j < 16; j += 2)
+            pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[16 * qd + j]) - delta_row),
+                                   pr[16 * qd + j + 1] * (__uint_as_float(tr[16 * qd + j + 1]) - delta_row));
+          tmem_st8(tmem_t + lane_sel + 16 * qd + 8 * half, pk);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(&e_full[qd]);
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) ok = bwd_wait_warp(acc_final, 0, abort_flag);
+      if (ok) tc_fence_after();
+    }
+    // ---- epilogue: add this part's sum to the running dQ of the KV group's rows, in link order
+    const bool fold = it.link > 0, last = it.link == p.parts;
+    int* counter = p.ctl + kChainHeaderInts + kvh;
+    if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
+    if (ok)
+      dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, fold, last, p.scale,
+                          p.dq_acc + ri * D + half * (D / 2), p.dq + ri * D + half * (D / 2), row_ok);
+    const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
+    if (row == 0 && half == 0 && all_ok) chain_publish(counter, it.link + 1);
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+    st_relaxed_gpu(p.ctl + 1, 1);    // ends every other chain wait of this launch
+  }
+}
+
 // Delta[t,h] = sum_d dO[t,h,d] * O[t,h,d], one warp per row.
 __global__ void delta_kernel(const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ o, int64_t rows,
                              int dv, float* __restrict__ delta) {
@@ -1310,6 +1624,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   }
 }
 
+template <int D>
+static ls_status_t launch_dq1(const BwdParams& prm, int64_t grid, cudaStream_t st) {
+  using C = BwdCfg<D>;
+  static bool configured[64] = {};
+  if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
+  const ls_status_t cs = configure_smem(bwd_dq1_kernel<D>, C::SMEM_BYTES, configured);
+  if (cs != LS_OK) return cs;
+  profile_begin(LS_KERNEL_BWD_DQ, st);
+  bwd_dq1_kernel<D><<<(int)grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
+  profile_end(LS_KERNEL_BWD_DQ, st);
+  return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
 static ls_status_t launch_dq3(const BwdParams& prm, int64_t grid, cudaStream_t st) {
   static bool configured[64] = {};
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
@@ -1448,8 +1775,22 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   if (st == LS_OK) st = ls::pool_map(&P.pv_m_tail, h, 1, mbox, 1, true);
   if (st != LS_OK) return st;
   if (cudaMemsetAsync(ctl, 0, ctl_bytes, cs) != cudaSuccess) return LS_ERR_CUDA;
-  const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
-  st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq3(P, grid2, cs);
+  if (P.packed) {
+    // short response: one single-CTA work item per (KV head, part), K/V pages read once
+    const int pbox = small_pages ? 64 : 128, pgroups = small_pages ? 1 : 2;
+    st = dense_map(&P.b1r_map, k_resp, Hkv, 128, 2);
+    if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 128, 2);
+    if (st == LS_OK) st = ls::pool_map(&P.bk_map, h, 0, pbox, pgroups, false);
+    if (st == LS_OK) st = ls::pool_map(&P.bk_tail, h, 0, pbox, pgroups, true);
+    if (st == LS_OK) st = ls::pool_map(&P.bv_map, h, 1, pbox, pgroups, false);
+    if (st == LS_OK) st = ls::pool_map(&P.bv_tail, h, 1, pbox, pgroups, true);
+    if (st != LS_OK) return st;
+    const int64_t grid1 = (int64_t)Hkv * (parts + 1);
+    st = (D == 128) ? ls::launch_dq1<128>(P, grid1, cs) : ls::launch_dq1<256>(P, grid1, cs);
+  } else {
+    const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
+    st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq3(P, grid2, cs);
+  }
   if (st != LS_OK) return st;
 
   // ---- dK and dV: rows = keys, columns = queries of the KV group
