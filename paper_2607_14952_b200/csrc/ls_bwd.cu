@@ -1705,12 +1705,12 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     const bool mla_fast = ls::mla_dq_fast(h);
     if (no_resp) {       // prefix parts only: the transposed kernel walks them all and writes dQ
       if (!mla_fast) return LS_ERR_UNSUPPORTED_SHAPE;
-      return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, nullptr, dq, status_dev, cs);
+      return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, nullptr, dq_acc + rows * D, dq, status_dev, cs);
     }
     ls_status_t ms =
         ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_acc, dk_resp, dv_resp, mla_fast, status_dev, cs);
     if (ms != LS_OK) return ms;
-    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_acc, dq, status_dev, cs);
+    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_acc, dq_acc + rows * D, dq, status_dev, cs);
     const int64_t n4m = rows * D / 4;
     ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4m + 255) / 256, 148 * 16), 256, 0, cs>>>(
         dq_acc, parts + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));

@@ -48,6 +48,9 @@ struct MlaDqParams {
   int packed;      // 1: a CTA's 64 rows are every (head, token) row of one KV group (g * R <= 64 rows; row r is
                    //    head r / R, token r % R) instead of 64 tokens of one head
   int qdo_bytes;   // bytes the Q and dO loads deliver
+  int nsplit;      // packed: CTAs per KV group, each walking a contiguous range of the parts; with more than
+                   // one the fp32 sums go to dq_split [nsplit, R, Hq, 576] and a reduce kernel finishes
+  float* dq_split;
   int ablate;   // diagnostic builds only: 1 = no key loads, 2 = no tensor-core instructions
   float scale, scale_log2;
 };
@@ -97,13 +100,17 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
   long long tw0 = 0, tw1 = 0, tw2 = 0, tw3 = 0;   // wait-time accumulators (only used with LS_TIMING)
   const long long t_begin = clock64();
   // 64 tokens of one head, or (packed) all rows of one KV group
-  const int h = p.packed ? blockIdx.x * p.g : blockIdx.x / p.tiles_per_head;      // (first) head of the block
+  const int h = p.packed ? (blockIdx.x / p.nsplit) * p.g : blockIdx.x / p.tiles_per_head;   // (first) head of the block
   const int row0 = p.packed ? 0 : (blockIdx.x % p.tiles_per_head) * kTqRows;
   const int kvh = h / p.g;
+  // the parts this CTA walks: all of them, or (packed, several CTAs per KV group) a contiguous range
+  const int split = p.packed ? blockIdx.x % p.nsplit : 0;
+  const int part_lo = (int)((long long)split * p.nparts / p.nsplit);
+  const int part_hi = (int)((long long)(split + 1) * p.nparts / p.nsplit);
 
-  // key tiles of 128 over all partials (every role walks the same list)
+  // key tiles of 128 over those parts (every role walks the same list)
   int total_tiles = 0;
-  for (int r = 0; r < p.nparts; ++r) total_tiles += (int)((p.shard_tokens[r] + 127) >> 7);
+  for (int r = part_lo; r < part_hi; ++r) total_tiles += (int)((p.shard_tokens[r] + 127) >> 7);
 
   if (threadIdx.x == 0) {
     mbar_init(a_full, 1);
@@ -165,11 +172,11 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
       };
       auto next_tile = [&](Walk& w) {
         ++w.tile;
-        while (w.part < p.nparts && w.tile >= w.c_tiles) {
+        while (w.part < part_hi && w.tile >= w.c_tiles) {
           w.tile = 0;
-          if (w.part + 1 < p.nparts) open_part(w, w.part + 1); else ++w.part;
+          if (w.part + 1 < part_hi) open_part(w, w.part + 1); else ++w.part;
         }
-        if (w.part >= p.nparts) return;
+        if (w.part >= part_hi) return;
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           const int tok = w.tile * 128 + half * 64;
@@ -216,7 +223,7 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
       };
       Walk ws, wa;
       ws.tile = -1;
-      open_part(ws, 0);
+      open_part(ws, part_lo);
       wa = ws;
       next_tile(ws);
 #pragma unroll 1
@@ -339,7 +346,7 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
     const int sw = key & 7;
     if (total_tiles > 0) {
       bool ok = true;
-      int part = 0, tile = -1;
+      int part = part_lo, tile = -1;
       for (int i = 0; i < total_tiles && ok; ++i) {
         ++tile;
         while (tile >= (int)((p.shard_tokens[part] + 127) >> 7)) {
@@ -410,11 +417,21 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
               const int hh = p.packed ? h + rr / p.R : h;
               if (p.packed ? rr < p.g * p.R : r < p.R) {
                 const size_t idx = ((size_t)r * p.Hq + hh) * 576 + ch;
-                p.dq[idx] = __float2bfloat16_rn((__uint_as_float(o[j]) + (p.dq_resp ? p.dq_resp[idx] : 0.f)) * p.scale);
+                if (p.nsplit > 1)
+                  p.dq_split[(size_t)split * p.R * p.Hq * 576 + idx] = __uint_as_float(o[j]);
+                else
+                  p.dq[idx] = __float2bfloat16_rn((__uint_as_float(o[j]) + (p.dq_resp ? p.dq_resp[idx] : 0.f)) * p.scale);
               }
             }
           }
         }
+      }
+    } else if (p.nsplit > 1) {
+      // an empty range of parts still owes its (zero) partial to the reduce kernel
+      for (int m = 0; m < 5; ++m) {
+        if (m == 4 && quad >= 2) break;
+        for (int rr = 0; rr < p.g * p.R; ++rr)
+          p.dq_split[(size_t)split * p.R * p.Hq * 576 + ((size_t)(rr % p.R) * p.Hq + h + rr / p.R) * 576 + m * 128 + key] = 0.f;
       }
     }
   }
@@ -433,11 +450,35 @@ bool mla_dq_fast(const ls_pages* h) {
   return d.dim_k == 576 && d.dim_v == 512 && d.v_aliases_k && d.prefix_len > 0;
 }
 
+int mla_dq_splits(const ls_pages* h, int R, int Hq) {
+  const int Hkv = h->desc.num_kv_heads;
+  const int g = Hq / Hkv;
+  if (!(g > 1 && g * R <= kTqRows)) return 1;                    // not packed: one CTA per 64 rows walks every part
+  // packed: a KV group is one row block, so the parts are spread over enough CTAs to fill the GPU twice
+  return std::max(1, std::min(h->prefix_parts(), (148 * 2 + Hkv - 1) / Hkv));
+}
+
+// dq = scale * (sum of the split partials + the response block's partial), bf16
+__global__ void mla_dq_split_reduce_kernel(const float* __restrict__ part, int nsplit, const float* __restrict__ dq_resp,
+                                           int64_t n4, float scale, __nv_bfloat16* __restrict__ dq) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+    float4 acc = dq_resp ? *reinterpret_cast<const float4*>(dq_resp + i * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < nsplit; ++s) {
+      const float4 v = *reinterpret_cast<const float4*>(part + ((int64_t)s * n4 + i) * 4);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    uint2 pk;
+    pk.x = pack_bf16(acc.x * scale, acc.y * scale);
+    pk.y = pack_bf16(acc.z * scale, acc.w * scale);
+    *reinterpret_cast<uint2*>(dq + i * 4) = pk;
+  }
+}
+
 // dQ (bf16, final) of the 576/512 shape with V aliasing K: prefix part in this kernel, plus
 // dq_resp, the response block's unscaled fp32 part computed beforehand.
 ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
-                       const float* lse, const float* delta, const float* dq_resp, void* dq, int32_t* status_dev,
-                       cudaStream_t cs) {
+                       const float* lse, const float* delta, const float* dq_resp, float* dq_split, void* dq,
+                       int32_t* status_dev, cudaStream_t cs) {
   const ls_pages_desc_t& d = h->desc;
   const int R = prm->R, Hq = prm->num_q_heads;
   MlaDqParams P;
@@ -465,6 +506,9 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   P.packed = (P.g > 1 && P.g * R <= kTqRows) ? 1 : 0;
   const int rows_loaded = P.packed ? P.g * R : kTqRows;
   P.qdo_bytes = (9 + 8) * rows_loaded * 128;
+  P.nsplit = mla_dq_splits(h, R, Hq);
+  P.dq_split = dq_split;
+  if (P.nsplit > 1 && !dq_split) return LS_ERR_WORKSPACE;
   ls_status_t st = P.packed ? encode_map_rows(&P.q_map, q, 576, R, Hq, R, P.g)
                             : encode_map5(&P.q_map, q, 576, R, Hq, 1, (int64_t)Hq * 576, 576, (int64_t)R * Hq * 576, 64, 1);
   if (st == LS_OK)
@@ -478,10 +522,15 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   static bool configured[64] = {};
   const ls_status_t cfg = configure_smem(bwd_mla_dq_kernel, kTqSmem, configured);
   if (cfg != LS_OK) return cfg;
-  const int64_t grid = P.packed ? (int64_t)d.num_kv_heads : (int64_t)Hq * P.tiles_per_head;
+  const int64_t grid = P.packed ? (int64_t)d.num_kv_heads * P.nsplit : (int64_t)Hq * P.tiles_per_head;
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   profile_begin(LS_KERNEL_BWD_DQ, cs);
   bwd_mla_dq_kernel<<<(int)grid, kTqThreads, kTqSmem, cs>>>(P);
+  if (P.nsplit > 1) {
+    const int64_t n4 = (int64_t)R * Hq * 576 / 4;
+    mla_dq_split_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 8), 256, 0, cs>>>(
+        dq_split, P.nsplit, dq_resp, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
+  }
   profile_end(LS_KERNEL_BWD_DQ, cs);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }

@@ -1083,7 +1083,10 @@ extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_a
   const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes((int64_t)f.Hkv * f.g * f.tiles_per_head);
   if (f.mla && !ls::mla_dq_fast(h))     // 576/512 with a separate V pool: one fp32 dQ per partial
     return head + (size_t)(h->num_parts() + 1) * rows * d.dim_k * sizeof(float);
-  return head + rows * d.dim_k * sizeof(float);
+  // (short responses of the aliased 576/512 shape spread the parts of a KV group over several CTAs,
+  // each with an fp32 sum of its own)
+  const size_t splits = (f.mla && ls::mla_dq_fast(h)) ? (size_t)ls::mla_dq_splits(h, f.R, f.Hq) : 1;
+  return head + (1 + (splits > 1 ? splits : 0)) * rows * d.dim_k * sizeof(float);
 }
 
 extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_params_t* prm, const void* q,

@@ -150,9 +150,12 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
 
 // Prefix part of dQ for the 576/512 shape when V aliases K (ls_bwd_mla_dq.cu): every CTA walks
 // all partials, adds dq_resp (fp32, unscaled, [R, Hq, 576]) and writes the final bf16 dQ.
+// dq_split: fp32 scratch of mla_dq_splits() * R * Hq * 576 floats, needed when that count exceeds 1.
 ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
-                       const float* lse, const float* delta, const float* dq_resp, void* dq, int32_t* status_dev,
-                       cudaStream_t cs);
+                       const float* lse, const float* delta, const float* dq_resp, float* dq_split, void* dq,
+                       int32_t* status_dev, cudaStream_t cs);
+// CTAs per KV group of the packed (short-response) form of bwd_mla_dq; 1 otherwise.
+int mla_dq_splits(const ls_pages* h, int R, int Hq);
 // True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix).
 bool mla_dq_fast(const ls_pages* h);
 
