@@ -60,7 +60,8 @@ struct BwdParams {
   int32_t* status;
   long long* timing;     // diagnostic builds only
   int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
-  int packed;    // dQ pass: one Q tile holds every (head, token) row of a KV group
+  // dQ pass of a short response (single-CTA kernel): Q tiles of bt tokens x bh heads (RowTiling)
+  int bt, bh, tiles_tok;
   int no_resp;   // dQ pass: the response block is left out
   // dK / dV pass: keys of a suffix block (1) read through pages [key_page_off, ..) of part_pages,
   // key_tokens of them, first gradient slot grad_slot0; or the response block (0)
@@ -576,10 +577,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   const bool is_resp = it.is_resp;
   auto tile_of = [&](int qt, int& hh, int& r0) {
     if (qt < p.nq_tiles) {
-      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      hh = kvh * p.g + qt / p.tiles_per_head;
       r0 = (qt % p.tiles_per_head) * 128;
     } else {                                 // odd tile count: the pair's second CTA works on zero rows
-      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      hh = kvh * p.g + p.g - 1;
       r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
     }
   };
@@ -602,7 +603,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
-      const int a_rows = p.packed ? p.g * p.R : 128;
+      const int a_rows = 128;
       if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * a_rows * 128);
       for (int c = 0; c < C::SLABS; ++c) {
         tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
@@ -788,12 +789,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;
-    // this thread's (token, head): 128 tokens of one head, or all rows of a KV group when packed
-    const int r_idx = p.packed ? row0 + row % p.R : row0 + row;
-    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
+    // this thread's (token, head): 128 tokens of one head
+    const int r_idx = row0 + row;
+    const int hr = h;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const bool tile_ok = qtile < p.nq_tiles;
-    const bool row_ok = tile_ok && r_idx < p.R && (!p.packed || row < p.g * p.R);
+    const bool row_ok = tile_ok && r_idx < p.R;
     const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
     bool ok = true;
     if (n_tiles > 0) {
@@ -948,15 +949,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
   const uint32_t tmem_s = tmem_base + D;
   const uint32_t tmem_t = tmem_base + D + 128;
 
-  // ---- work item: (KV head, link); the one packed Q tile of the KV group
-  const DqItem it = dq_item(p, *work_idx, 1);
-  const int part = it.part, kvh = it.kvh;
+  // ---- work item: (KV head, link, Q tile of bt tokens x bh heads of the KV group)
+  const DqItem it = dq_item(p, *work_idx, p.nq_tiles);
+  const int part = it.part, kvh = it.kvh, qtile = it.pairi;
   const bool is_resp = it.is_resp;
-  const int h = kvh * p.g;
+  const int h = kvh * p.g + (qtile / p.tiles_tok) * p.bh;
+  const int t0 = (qtile % p.tiles_tok) * p.bt;
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = p.no_resp ? 0 : p.R;
+    tokens = p.no_resp ? 0 : min(p.R, t0 + p.bt);
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -968,10 +970,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
   if (warp == 0) {
     // =========================================================== producer (one thread)
     if (lane == 0 && n_tiles > 0) {
-      mbar_arrive_expect_tx(a_full, 2 * C::SLABS * p.g * p.R * 128);
+      mbar_arrive_expect_tx(a_full, 2 * C::SLABS * p.bt * p.bh * 128);
       for (int c = 0; c < C::SLABS; ++c) {
-        tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, 0, c, h, 0);
-        tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, 0, c, h, 0);
+        tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, t0, c, h, 0);
+        tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, t0, c, h, 0);
       }
       const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
@@ -1117,10 +1119,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
     const int row = quad * 32 + lane;
-    const int r_idx = row % p.R;                          // token of this packed row
-    const int hr = h + min(row / p.R, p.g - 1);           // and its head
+    const int hj = row / p.bt;                            // head and token of this row of the tile
+    const int r_tok = t0 + row - hj * p.bt;
+    const bool row_ok = hj < p.bh && r_tok < p.R && h + hj < (kvh + 1) * p.g;
+    const int r_idx = min(r_tok, p.R - 1);
+    const int hr = min(h + hj, p.Hq - 1);
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    const bool row_ok = row < p.g * p.R;
     const size_t ri = (size_t)r_idx * p.Hq + hr;
     bool ok = true;
     if (n_tiles > 0) {
@@ -1178,7 +1182,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
     }
     // ---- epilogue: add this part's sum to the running dQ of the KV group's rows, in link order
     const bool fold = it.link > 0, last = it.link == p.parts;
-    int* counter = p.ctl + kChainHeaderInts + kvh;
+    int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + qtile;
     if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
     if (ok)
       dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, fold, last, p.scale,
@@ -1339,10 +1343,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   const bool is_resp = it.is_resp;
   auto tile_of = [&](int qt, int& hh, int& r0) {
     if (qt < p.nq_tiles) {
-      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
+      hh = kvh * p.g + qt / p.tiles_per_head;
       r0 = (qt % p.tiles_per_head) * 128;
     } else {
-      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
+      hh = kvh * p.g + p.g - 1;
       r0 = p.tiles_per_head * 128;
     }
   };
@@ -1365,7 +1369,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
-      const int a_rows = p.packed ? p.g * p.R : 128;
+      const int a_rows = 128;
       if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * a_rows * 128);
       for (int c = 0; c < C::SLABS; ++c) {
         tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
@@ -1515,11 +1519,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
     const int quad = warp & 3;
     const int sub = (warp - 2) >> 2;                // which 32 of every 64-column quarter this thread owns (2 threads per row)
     const int row = quad * 32 + lane;
-    const int r_idx = p.packed ? row0 + row % p.R : row0 + row;
-    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
+    const int r_idx = row0 + row;
+    const int hr = h;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const bool tile_ok = qtile < p.nq_tiles;
-    const bool row_ok = tile_ok && r_idx < p.R && (!p.packed || row < p.g * p.R);
+    const bool row_ok = tile_ok && r_idx < p.R;
     const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
     bool ok = true;
     if (n_tiles > 0) {
@@ -1751,12 +1755,14 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
 
   // ---- dQ: rows = queries, columns = keys of every part, summed through the running dQ
   P.no_resp = no_resp ? 1 : 0;
-  P.packed = 0;
-  if (g > 1 && g * R <= 128) {           // short response: all rows of a KV group in one Q tile
-    P.packed = 1;
-    P.nq_tiles = 1;
-    st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, R, g);
-    if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, R, g);
+  const ls::RowTiling rt = ls::row_tiling(R, g, 128);
+  P.bt = rt.bt;
+  P.bh = rt.bh;
+  P.tiles_tok = rt.tiles_tok;
+  if (rt.packed) {                       // short response: rows of several heads share a Q tile
+    P.nq_tiles = rt.nq_tiles;
+    st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, rt.bt, rt.bh);
+    if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, rt.bt, rt.bh);
   } else {
     st = dense_map(&P.a1_map, q, Hq, 128, 1);
     if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128, 1);
@@ -1775,8 +1781,8 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   if (st == LS_OK) st = ls::pool_map(&P.pv_m_tail, h, 1, mbox, 1, true);
   if (st != LS_OK) return st;
   if (cudaMemsetAsync(ctl, 0, ctl_bytes, cs) != cudaSuccess) return LS_ERR_CUDA;
-  if (P.packed) {
-    // short response: one single-CTA work item per (KV head, part), K/V pages read once
+  if (rt.packed) {
+    // short response: one single-CTA work item per (KV head, part, Q tile); K/V pages come from DRAM once
     const int pbox = small_pages ? 64 : 128, pgroups = small_pages ? 1 : 2;
     st = dense_map(&P.b1r_map, k_resp, Hkv, 128, 2);
     if (st == LS_OK) st = dense_map(&P.b2r_map, v_resp, Hkv, 128, 2);
@@ -1785,7 +1791,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     if (st == LS_OK) st = ls::pool_map(&P.bv_map, h, 1, pbox, pgroups, false);
     if (st == LS_OK) st = ls::pool_map(&P.bv_tail, h, 1, pbox, pgroups, true);
     if (st != LS_OK) return st;
-    const int64_t grid1 = (int64_t)Hkv * (parts + 1);
+    const int64_t grid1 = (int64_t)Hkv * (parts + 1) * rt.nq_tiles;
     st = (D == 128) ? ls::launch_dq1<128>(P, grid1, cs) : ls::launch_dq1<256>(P, grid1, cs);
   } else {
     const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;

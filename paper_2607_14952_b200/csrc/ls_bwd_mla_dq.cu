@@ -44,12 +44,13 @@ struct MlaDqParams {
   __nv_bfloat16* dq;                 // [R, Hq, 576]
   int32_t* status;
   long long* timing;   // diagnostic builds only
-  int R, Hq, g, nparts, pg_shift, tiles_per_head, num_phys_pages;
-  int packed;      // 1: a CTA's 64 rows are every (head, token) row of one KV group (g * R <= 64 rows; row r is
-                   //    head r / R, token r % R) instead of 64 tokens of one head
+  int R, Hq, g, nparts, pg_shift, num_phys_pages;
+  // Row blocks of a KV group (RowTiling with 64-row tiles): block q covers bt tokens from (q % tiles_tok) * bt
+  // of bh heads from (q / tiles_tok) * bh; its row r is head r / bt, token r % bt.  Long responses: 64 x 1.
+  int bt, bh, tiles_tok, nq_tiles;
   int qdo_bytes;   // bytes the Q and dO loads deliver
-  int nsplit;      // packed: CTAs per KV group, each walking a contiguous range of the parts; with more than
-                   // one the fp32 sums go to dq_split [nsplit, R, Hq, 576] and a reduce kernel finishes
+  int nsplit;      // CTAs per row block, each walking a contiguous range of the parts; with more than one
+                   // the fp32 sums go to dq_split [nsplit, R, Hq, 576] and a reduce kernel finishes
   float* dq_split;
   int ablate;   // diagnostic builds only: 1 = no key loads, 2 = no tensor-core instructions
   float scale, scale_log2;
@@ -99,12 +100,13 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   long long tw0 = 0, tw1 = 0, tw2 = 0, tw3 = 0;   // wait-time accumulators (only used with LS_TIMING)
   const long long t_begin = clock64();
-  // 64 tokens of one head, or (packed) all rows of one KV group
-  const int h = p.packed ? (blockIdx.x / p.nsplit) * p.g : blockIdx.x / p.tiles_per_head;   // (first) head of the block
-  const int row0 = p.packed ? 0 : (blockIdx.x % p.tiles_per_head) * kTqRows;
-  const int kvh = h / p.g;
-  // the parts this CTA walks: all of them, or (packed, several CTAs per KV group) a contiguous range
-  const int split = p.packed ? blockIdx.x % p.nsplit : 0;
+  // work item: row block (fastest, so that the CTAs in flight share the same keys), range of parts, KV head
+  const int qtile = blockIdx.x % p.nq_tiles;
+  const int split = (blockIdx.x / p.nq_tiles) % p.nsplit;
+  const int kvh = blockIdx.x / (p.nq_tiles * p.nsplit);
+  const int h = kvh * p.g + (qtile / p.tiles_tok) * p.bh;     // first head and token of the block
+  const int row0 = (qtile % p.tiles_tok) * p.bt;
+  // the parts this CTA walks: all of them, or (several CTAs per row block) a contiguous range
   const int part_lo = (int)((long long)split * p.nparts / p.nsplit);
   const int part_hi = (int)((long long)(split + 1) * p.nparts / p.nsplit);
 
@@ -128,8 +130,8 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
   }
   if (threadIdx.x >= 64 && threadIdx.x < 64 + kTqRows) {
     const int t = threadIdx.x - 64;
-    const size_t ri = p.packed ? (size_t)(t % p.R) * p.Hq + h + min(t / p.R, p.g - 1)
-                               : (size_t)min(row0 + t, p.R - 1) * p.Hq + h;
+    const int hj = t / p.bt;
+    const size_t ri = (size_t)min(row0 + t - hj * p.bt, p.R - 1) * p.Hq + min(h + hj, p.Hq - 1);
     rowp[t] = make_float2(p.lse[ri] * kLog2eTq, p.delta[ri]);
   }
   if (warp == 1) {
@@ -410,12 +412,15 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
             uint32_t o[32];
             tmem_ld32(tmem_acc + lane_sel + m * 64 + half * 32, o);
             tc_wait_ld32(o);
+            int hj = (half * 32) / p.bt, tk = half * 32 - hj * p.bt;   // head and token of row half * 32 + j
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int rr = half * 32 + j;                    // row of the block
-              const int r = p.packed ? rr % p.R : row0 + rr;   // its token and head
-              const int hh = p.packed ? h + rr / p.R : h;
-              if (p.packed ? rr < p.g * p.R : r < p.R) {
+              const int r = row0 + tk, hh = h + hj;
+              if (++tk == p.bt) {
+                tk = 0;
+                ++hj;
+              }
+              if (hh - h < p.bh && r < p.R && hh < (kvh + 1) * p.g) {
                 const size_t idx = ((size_t)r * p.Hq + hh) * 576 + ch;
                 if (p.nsplit > 1)
                   p.dq_split[(size_t)split * p.R * p.Hq * 576 + idx] = __uint_as_float(o[j]);
@@ -430,8 +435,11 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
       // an empty range of parts still owes its (zero) partial to the reduce kernel
       for (int m = 0; m < 5; ++m) {
         if (m == 4 && quad >= 2) break;
-        for (int rr = 0; rr < p.g * p.R; ++rr)
-          p.dq_split[(size_t)split * p.R * p.Hq * 576 + ((size_t)(rr % p.R) * p.Hq + h + rr / p.R) * 576 + m * 128 + key] = 0.f;
+        for (int rr = 0; rr < p.bt * p.bh; ++rr) {
+          const int r = row0 + rr % p.bt, hh = h + rr / p.bt;
+          if (r < p.R && hh < (kvh + 1) * p.g)
+            p.dq_split[(size_t)split * p.R * p.Hq * 576 + ((size_t)r * p.Hq + hh) * 576 + m * 128 + key] = 0.f;
+        }
       }
     }
   }
@@ -452,10 +460,10 @@ bool mla_dq_fast(const ls_pages* h) {
 
 int mla_dq_splits(const ls_pages* h, int R, int Hq) {
   const int Hkv = h->desc.num_kv_heads;
-  const int g = Hq / Hkv;
-  if (!(g > 1 && g * R <= kTqRows)) return 1;                    // not packed: one CTA per 64 rows walks every part
-  // packed: a KV group is one row block, so the parts are spread over enough CTAs to fill the GPU twice
-  return std::max(1, std::min(h->prefix_parts(), (148 * 2 + Hkv - 1) / Hkv));
+  const int64_t blocks = (int64_t)Hkv * row_tiling(R, Hq / Hkv, kTqRows).nq_tiles;
+  if (blocks >= 148) return 1;                 // enough row blocks: every CTA walks all parts
+  // few rows: the parts are spread over enough CTAs to fill the GPU twice
+  return std::max(1, std::min(h->prefix_parts(), (int)((148 * 2 + blocks - 1) / blocks)));
 }
 
 // dq = scale * (sum of the split partials + the response block's partial), bf16
@@ -497,23 +505,21 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   P.nparts = h->prefix_parts();
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.pg_shift = pg_shift_of(d.page_size);
-  P.tiles_per_head = (R + kTqRows - 1) / kTqRows;
   P.ablate = (prm->flags & LS_DBG_ABLATE_LOADS ? 1 : 0) | (prm->flags & LS_DBG_ABLATE_MMA ? 2 : 0);
   P.timing = g_timing_buffer;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * kLog2eTq;
-  // a short response packs every (head, token) row of a KV group into the CTA's 64 rows
-  P.packed = (P.g > 1 && P.g * R <= kTqRows) ? 1 : 0;
-  const int rows_loaded = P.packed ? P.g * R : kTqRows;
-  P.qdo_bytes = (9 + 8) * rows_loaded * 128;
-  P.nsplit = mla_dq_splits(h, R, Hq);
+  // a short response packs rows of several heads of a KV group into a CTA's 64 rows
+  const RowTiling rt = row_tiling(R, P.g, kTqRows);
+  P.bt = rt.bt;
+  P.bh = rt.bh;
+  P.tiles_tok = rt.tiles_tok;
+  P.nq_tiles = rt.nq_tiles;
+  P.qdo_bytes = (9 + 8) * rt.bt * rt.bh * 128;
+  P.nsplit = dq_split ? mla_dq_splits(h, R, Hq) : 1;     // without scratch every CTA walks all parts
   P.dq_split = dq_split;
-  if (P.nsplit > 1 && !dq_split) return LS_ERR_WORKSPACE;
-  ls_status_t st = P.packed ? encode_map_rows(&P.q_map, q, 576, R, Hq, R, P.g)
-                            : encode_map5(&P.q_map, q, 576, R, Hq, 1, (int64_t)Hq * 576, 576, (int64_t)R * Hq * 576, 64, 1);
-  if (st == LS_OK)
-    st = P.packed ? encode_map_rows(&P.do_map, d_o, 512, R, Hq, R, P.g)
-                  : encode_map5(&P.do_map, d_o, 512, R, Hq, 1, (int64_t)Hq * 512, 512, (int64_t)R * Hq * 512, 64, 1);
+  ls_status_t st = encode_map_rows(&P.q_map, q, 576, R, Hq, rt.bt, rt.bh);
+  if (st == LS_OK) st = encode_map_rows(&P.do_map, d_o, 512, R, Hq, rt.bt, rt.bh);
   if (st == LS_OK) st = pool_map(&P.k_map, h, 0, 64, 1, false);
   if (st == LS_OK) st = pool_map(&P.k_tail, h, 0, 64, 1, true);
   if (st == LS_OK) st = pool_map(&P.k2_map, h, 0, 64, 2, false);
@@ -522,7 +528,7 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   static bool configured[64] = {};
   const ls_status_t cfg = configure_smem(bwd_mla_dq_kernel, kTqSmem, configured);
   if (cfg != LS_OK) return cfg;
-  const int64_t grid = P.packed ? (int64_t)d.num_kv_heads * P.nsplit : (int64_t)Hq * P.tiles_per_head;
+  const int64_t grid = (int64_t)d.num_kv_heads * rt.nq_tiles * P.nsplit;
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   profile_begin(LS_KERNEL_BWD_DQ, cs);
   bwd_mla_dq_kernel<<<(int)grid, kTqThreads, kTqSmem, cs>>>(P);

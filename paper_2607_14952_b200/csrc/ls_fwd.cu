@@ -52,12 +52,13 @@ struct FwdParams {
   int* ctl;            // hand-over control words (ticket, abort, counters) or NULL
   int32_t* status;
   long long* timing;   // diagnostic builds only
-  int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
+  int R, Hq, Hkv, g, parts, pg_shift, nq_tiles, num_phys_pages;
+  // Q tiles of a KV group (RowTiling): tile q covers bt tokens from (q % tiles_tok) * bt of bh heads from
+  // (q / tiles_tok) * bh; its row r is head r / bt, token r % bt.  Long responses: bt = 128, bh = 1.
+  int bt, bh, tiles_tok;
   int chain_mode, fine;
   int no_resp;    // 1: the response block is left out (its partial is written as empty)
   int dv_total;   // channels of one output row (DVT times the number of O tiles)
-  int packed;     // 1: one Q tile holds every (head, token) row of a KV group (g * R <= 128 rows);
-                  //    row r is head r / R, token r % R.  Lets a short response stream K/V once.
   int q_bytes;    // bytes the Q loads deliver
   int ablate;     // diagnostic builds only (LS_DBG_ABLATE_*)
   float scale, scale_log2;
@@ -258,14 +259,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
   idx /= NDV;
   const FwdItem it = fwd_item(p, idx, p.nq_tiles);
   const int qtile = it.qunit, part = it.part, kvh = it.kvh;
-  const int h = kvh * p.g + qtile / p.tiles_per_head;
-  const int ttile = qtile % p.tiles_per_head;
-  const int t0 = ttile * 128;
+  const int h = kvh * p.g + (qtile / p.tiles_tok) * p.bh;      // first head and token of the tile
+  const int t0 = (qtile % p.tiles_tok) * p.bt;
   const bool is_resp = it.is_resp;
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = p.no_resp ? 0 : min(p.R, t0 + 128);       // keys 0 .. last row of this tile (none when the block is left out)
+    tokens = p.no_resp ? 0 : min(p.R, t0 + p.bt);      // keys 0 .. last row of this tile (none when the block is left out)
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -456,10 +456,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
     // =========================================================== softmax + epilogue
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    // this thread's (token, head): a tile is 128 tokens of one head, or all rows of a KV group
-    const int t = p.packed ? row % p.R : t0 + row;
-    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
-    const bool row_ok = p.packed ? row < p.g * p.R : t < p.R;
+    // this thread's (token, head) inside the tile of bt tokens x bh heads
+    const int hj = row / p.bt;
+    const int t = t0 + row - hj * p.bt;
+    const bool row_ok = hj < p.bh && t < p.R && h + hj < (kvh + 1) * p.g;
+    const int hr = min(h + hj, p.Hq - 1);
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const size_t out_row = ((size_t)fwd_out_part(p, it) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
     const bool to_resp = is_resp && p.chain_mode != 2;
@@ -656,11 +657,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   const bool is_resp = it.is_resp;
   auto tile_of = [&](int qt, int& hh, int& r0) {
     if (qt < p.nq_tiles) {
-      hh = kvh * p.g + (p.packed ? 0 : qt / p.tiles_per_head);
-      r0 = (qt % p.tiles_per_head) * 128;
+      hh = kvh * p.g + qt / p.tiles_tok;     // (this kernel serves tiles of 128 tokens of one head only)
+      r0 = (qt % p.tiles_tok) * 128;
     } else {                                 // odd tile count: the pair's second CTA works on zero rows
-      hh = kvh * p.g + (p.packed ? 0 : p.g - 1);
-      r0 = p.tiles_per_head * 128;           // token coordinate past R: TMA delivers zeros
+      hh = kvh * p.g + p.g - 1;
+      r0 = p.tiles_tok * 128;                // token coordinate past R: TMA delivers zeros
     }
   };
   const int qtile = 2 * pairi + (int)rank;
@@ -805,10 +806,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     // =========================================================== softmax + epilogue (both CTAs)
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    const int t = p.packed ? t0 + row % p.R : t0 + row;
-    const int hr = p.packed ? h + min(row / p.R, p.g - 1) : h;
+    const int t = t0 + row;
+    const int hr = h;
     const bool tile_ok = qtile < p.nq_tiles;
-    const bool row_ok = tile_ok && t < p.R && (!p.packed || row < p.g * p.R);
+    const bool row_ok = tile_ok && t < p.R;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const size_t out_row = ((size_t)fwd_out_part(p, it) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
     const bool to_resp = is_resp && p.chain_mode != 2;
@@ -944,7 +945,8 @@ static ls_status_t launch_fwd(const FwdParams& prm, int64_t grid, cudaStream_t s
 
 // Shape facts shared by the entry points.
 struct FwdShape {
-  int R, Hq, Hkv, g, dk, dv, nq_tiles, tiles_per_head, ndv;
+  int R, Hq, Hkv, g, dk, dv, nq_tiles, ndv;
+  RowTiling rt;
   bool mla, packed;
 };
 static FwdShape fwd_shape(const ls_pages* h, const ls_attn_params_t* prm) {
@@ -957,9 +959,9 @@ static FwdShape fwd_shape(const ls_pages* h, const ls_attn_params_t* prm) {
   f.dk = d.dim_k;
   f.dv = d.dim_v;
   f.mla = d.dim_k == 576;
-  f.packed = f.g * f.R <= 128 && f.g > 1;      // short response: every row of a KV group in one Q tile
-  f.tiles_per_head = (f.R + 127) / 128;
-  f.nq_tiles = f.packed ? 1 : f.g * f.tiles_per_head;
+  f.rt = row_tiling(f.R, f.g, 128);            // short response: rows of several heads share a Q tile
+  f.packed = f.rt.packed;
+  f.nq_tiles = f.rt.nq_tiles;
   f.ndv = f.mla ? 2 : 1;
   return f;
 }
@@ -981,8 +983,7 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
   const bool small_pages = d.page_size == 64;
   const bool pair = d.dim_k == 256 && !f.packed;            // CTA pairs share every key tile between two Q tiles
   if (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) k_resp = v_resp = q;   // the response maps are encoded but never used
-  ls_status_t st = f.packed ? encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, R, f.g)
-                            : encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, 128, 1);
+  ls_status_t st = encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, f.rt.bt, f.rt.bh);
   if (pair) {
     if (st == LS_OK) st = encode_map5(&P.rk2, k_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
     if (st == LS_OK) st = encode_map5(&P.rv2, v_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
@@ -1022,10 +1023,11 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
   P.g = f.g;
   P.parts = parts;
   P.pg_shift = pg_shift_of(d.page_size);
-  P.tiles_per_head = f.tiles_per_head;
   P.nq_tiles = f.nq_tiles;
-  P.packed = f.packed ? 1 : 0;
-  P.q_bytes = (d.dim_k / 64) * (f.packed ? f.g * R : 128) * 128;
+  P.bt = f.rt.bt;
+  P.bh = f.rt.bh;
+  P.tiles_tok = f.rt.tiles_tok;
+  P.q_bytes = (d.dim_k / 64) * f.rt.bt * f.rt.bh * 128;
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.dv_total = d.dim_v;
   P.chain_mode = mode;
@@ -1080,7 +1082,7 @@ extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_a
     return ls::ctl_bytes((int64_t)f.Hkv * f.nq_tiles * f.ndv) + (f.mla ? rows * sizeof(float) : 0);
   if (which != LS_WORKSPACE_BWD) return 0;
   // backward: Delta (fp32) + hand-over counters + the fp32 dQ that the partials are summed into
-  const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes((int64_t)f.Hkv * f.g * f.tiles_per_head);
+  const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes((int64_t)f.Hkv * f.g * ((f.R + 127) / 128));
   if (f.mla && !ls::mla_dq_fast(h))     // 576/512 with a separate V pool: one fp32 dQ per partial
     return head + (size_t)(h->num_parts() + 1) * rows * d.dim_k * sizeof(float);
   // (short responses of the aliased 576/512 shape spread the parts of a KV group over several CTAs,

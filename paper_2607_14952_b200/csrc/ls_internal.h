@@ -150,17 +150,51 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
 
 // Prefix part of dQ for the 576/512 shape when V aliases K (ls_bwd_mla_dq.cu): every CTA walks
 // all partials, adds dq_resp (fp32, unscaled, [R, Hq, 576]) and writes the final bf16 dQ.
-// dq_split: fp32 scratch of mla_dq_splits() * R * Hq * 576 floats, needed when that count exceeds 1.
+// dq_split: fp32 scratch of mla_dq_splits() * R * Hq * 576 floats that lets a launch with few row blocks
+// spread the parts over several CTAs per block (NULL: every CTA walks all parts).
 ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
                        const float* lse, const float* delta, const float* dq_resp, float* dq_split, void* dq,
                        int32_t* status_dev, cudaStream_t cs);
-// CTAs per KV group of the packed (short-response) form of bwd_mla_dq; 1 otherwise.
+// CTAs per row block of bwd_mla_dq when the launch has fewer row blocks than SMs; 1 otherwise.
 int mla_dq_splits(const ls_pages* h, int R, int Hq);
 // True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix).
 bool mla_dq_fast(const ls_pages* h);
 
 // Delta[t,h] = dO[t,h] . O[t,h] (fp32), one warp per row.
 void launch_delta(const void* d_o, const float* o_f32, int64_t rows, int dv, float* delta, cudaStream_t st);
+
+// How the (token, head) rows of one KV group (R tokens x g heads) are cut into Q tiles of at most
+// tile_rows rows.  A tile covers bt consecutive tokens of bh consecutive heads; its row r is head
+// r / bt, token r % bt (the order in which one TMA box of bt tokens x bh heads lands in shared
+// memory).  Long responses use tiles of tile_rows tokens of one head.  A response shorter than a
+// tile packs the rows of several heads into one tile whenever that needs fewer tiles, so that the
+// K/V pages of the group are streamed once per tile of FULL rows instead of once per head.
+struct RowTiling {
+  int bt, bh, tiles_tok, tiles_head, nq_tiles;
+  bool packed;
+};
+inline RowTiling row_tiling(int R, int g, int tile_rows) {
+  RowTiling t;
+  t.bt = tile_rows;
+  t.bh = 1;
+  t.tiles_tok = (R + tile_rows - 1) / tile_rows;
+  t.tiles_head = g;
+  t.packed = false;
+  if (g > 1 && R < tile_rows) {
+    const int bh = g < tile_rows ? g : tile_rows;
+    const int bt = R < tile_rows / bh ? R : tile_rows / bh;
+    const int tt = (R + bt - 1) / bt, th = (g + bh - 1) / bh;
+    if (tt * th < g) {
+      t.bt = bt;
+      t.bh = bh;
+      t.tiles_tok = tt;
+      t.tiles_head = th;
+      t.packed = true;
+    }
+  }
+  t.nq_tiles = t.tiles_tok * t.tiles_head;
+  return t;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -47,6 +47,16 @@ def test_config1_tiny_full():
     small("mla_short_r3", Dk=576, Dv=512, v_aliases_k=True, Hq=16, Hkv=1, P=64 * 11 + 7, page_size=64, num_shards=2, R=3),
     small("mla_short_r1_64heads", Dk=576, Dv=512, v_aliases_k=True, Hq=64, Hkv=1, P=256 * 5 + 9, page_size=256,
           num_shards=3, R=1),
+    # responses shorter than a Q tile whose KV group needs several tiles of (tokens x heads) rows
+    small("short_r40_two_tiles", P=2048 + 77, page_size=256, num_shards=3, R=40, Hq=8, Hkv=2),
+    small("short_r30_g6", P=1900, page_size=128, num_shards=2, R=30, Hq=12, Hkv=2),
+    small("short_r100_d128", Dk=128, Dv=128, P=64 * 21 + 3, page_size=64, num_shards=4, R=100, Hq=16, Hkv=2),
+    small("mla_short_r5_64heads", Dk=576, Dv=512, v_aliases_k=True, Hq=64, Hkv=1, P=64 * 23 + 11, page_size=64,
+          num_shards=4, R=5),
+    small("mla_short_r2_128heads", Dk=576, Dv=512, v_aliases_k=True, Hq=128, Hkv=1, P=256 * 4 + 100, page_size=256,
+          num_shards=2, R=2),
+    small("mla_short_r20_8heads", Dk=576, Dv=512, v_aliases_k=True, Hq=8, Hkv=1, P=64 * 17, page_size=64,
+          num_shards=3, R=20),
 ], ids=lambda c: c.name)
 def test_backward_small_cases(cfg):
     case = parity.Case(cfg, extra_phys_pages=2)

@@ -40,6 +40,11 @@ def test_config1_tiny_full():
     small("short_r16", P=4096, page_size=256, num_shards=4, R=16, Hq=24, Hkv=4),
     small("short_r1", P=1500, page_size=64, num_shards=3, R=1, Hq=8, Hkv=2, Dk=128, Dv=128),
     small("short_r32_full_tile", P=2048, page_size=256, num_shards=2, R=32, Hq=8, Hkv=2),
+    # responses shorter than a Q tile whose KV group needs several tiles of (tokens x heads) rows
+    small("short_r40_two_tiles", P=2048 + 77, page_size=256, num_shards=3, R=40, Hq=8, Hkv=2),
+    small("short_r100_d128", Dk=128, Dv=128, P=64 * 21 + 3, page_size=64, num_shards=4, R=100, Hq=16, Hkv=2),
+    small("mla_short_r5_64heads", Dk=576, Dv=512, v_aliases_k=True, Hq=64, Hkv=1, P=64 * 23 + 11, page_size=64,
+          num_shards=4, R=5),
 ], ids=lambda c: c.name)
 def test_forward_small_cases(cfg):
     case = parity.Case(cfg, extra_phys_pages=2)
