@@ -2,25 +2,34 @@
 // channels of the 576-channel key page (Sec. "GLM page payloads"; dense form):
 //   dQ_th = scale * sum_j p_tj (dO_th . v_j - Delta_th) k_j,   p_tj = exp(scale q_th . k_j - LSE_th).
 //
-// The products are formed TRANSPOSED, keys on the tensor core's M side, so that a CTA can
-// keep only 64 rows (Q 72 KB + dO 64 KB) and still fill every 128-row instruction:
-//   [S^T | T^T] (128 keys x 128) = K_c (128 keys x 64 ch)  x  [Q_c ; dO_c]^T   c = 0..7
-//        Q and dO of the same 64-channel group lie back to back in shared memory, so one
-//        128x128x16 instruction yields 64 columns of S^T and 64 of T^T (V = K[:, :512]);
-//   S^T += K_8 x Q_8^T  (rope channels, N = 64);
-//   E^T  = p (T^T - Delta) : one thread per key, written to shared memory as bf16, keys x 64 rows;
-//   dQ^T (576 ch x 64 rows) += K^T (128 ch x 16 keys, MN-major view of the same slabs) x E^T.
-// The 576 x 64 fp32 accumulator is five 128-lane tiles of 64 TMEM columns (320 columns; the
-// upper half of the fifth is unused), [S^T | T^T] one buffer of 128 columns.  Every CTA walks
-// ALL prefix partials in order and keeps accumulating, which is Eq. qwen-dq-reduce carried out
-// in the accumulator; the causal response block (whose V is a separate tensor) arrives as an
-// fp32 partial from the generic kernel and is added in the epilogue, which writes bf16 dQ.
+// The products are formed TRANSPOSED, keys on the tensor core's M side, so that 64 rows (Q 72 KB,
+// dO 64 KB) still fill every 128-row instruction, and on CTA PAIRS (cta_group::2): the even CTA
+// keeps Q of the 64 rows, the odd CTA keeps dO, and a step covers 256 keys, 128 per CTA.
+//   [S^T | T^T] (256 keys x 128) = K_c (this CTA's 128 keys x 64 ch) x [Q_c ; dO_c]^T   c = 0..7
+//        the B operand of a pair instruction is split along N between the two CTAs, so the Q half
+//        yields 64 columns of S^T and the dO half 64 columns of T^T (V = K[:, :512]) in BOTH CTAs'
+//        TMEM, each for its own keys;
+//   S^T += K_8 x Q_8^T  (rope channels, N = 64: each CTA contributes 32 rows of Q_8, of which both
+//        hold a copy);
+//   E^T  = p (T^T - Delta) : one thread per key.  dQ^T is split along the channels (M) between the
+//        CTAs, and its B operand E^T along the rows (N): a thread writes rows 0-31 of its key into
+//        the even CTA's shared memory and rows 32-63 into the odd CTA's (st.shared::cluster), as
+//        bf16 in MN-major 64-byte lines;
+//   dQ^T (this CTA's 128 of 256 channels x 64 rows) += K^T (MN-major, 16 keys) x E^T, for the keys
+//        of either CTA.  Channel block m = groups 4m, 4m+1 (even CTA) and 4m+2, 4m+3 (odd CTA);
+//        block 2 is the 64 rope channels in the even CTA alone.
+// TMEM per CTA: two [S^T | T^T] buffers of 128 columns and three accumulator tiles of 64 columns.
+// Every pair walks ALL prefix partials in order and keeps accumulating, which is Eq. qwen-dq-reduce
+// carried out in the accumulator; the causal response block (whose V is a separate tensor) arrives
+// as an fp32 partial from the generic kernel and is added in the epilogue, which writes bf16 dQ.
 //
-// Every key tile streams through shared memory twice, in 16 KB slots of two small rings: as
-// nine K-major slabs (128 keys x one channel group) for [S^T | T^T], and as ten MN-major
-// slots (64 keys x two channel groups; the missing partner of the rope group reads as zeros)
-// for dQ^T.  Two threads issue the two kinds of products, so that dQ^T of tile i overlaps
-// [S^T | T^T] of tile i + 2 while the key threads work on tile i + 1.
+// Every key tile streams through shared memory twice, in 16 KB slots of two rings with a producer
+// thread each: K-major slabs (this CTA's 128 keys x one channel group) for [S^T | T^T], and
+// MN-major slots (64 keys of either CTA's tile x two of this CTA's channel groups) for dQ^T.  Two
+// threads of the even CTA issue the two kinds of products, so that dQ^T of step i overlaps
+// [S^T | T^T] of step i + 1 while the key threads of both CTAs work between them; E^T and
+// [S^T | T^T] are double-buffered.  What bounds it at full size is the stream itself: every 64-row
+// block pulls 2.3 KB per key out of L2 (about 7.5 TB/s over the launch).
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -68,62 +77,82 @@ struct MlaDqParams {
 #define LS_TQABLATE(bit) false
 #endif
 
-constexpr int kTqThreads = 224;   // producer, [S^T|T^T] issuer, 4 warps of key threads, dQ^T issuer
+constexpr int kTqThreads = 256;   // K-major producer, [S^T|T^T] issuer, 4 warps of key threads, dQ^T issuer, MN-major producer
 constexpr int kTqSlab = 16384;                 // 128 keys x 128 B
-constexpr int kTqRing = 4;                   // ring slots of 16 KB:
-constexpr int kTqStSlots = 2;                //   [S^T | T^T] slabs
-constexpr int kTqAccSlots = kTqRing - kTqStSlots;   //   dQ^T slots
+constexpr int kTqStSlots = 3;                  // ring slots of 16 KB: [S^T | T^T] slabs
+constexpr int kTqAccSlots = 4;                 //                      dQ^T slots
+constexpr int kTqRing = kTqStSlots + kTqAccSlots;
 constexpr int kTqRows = 64;
-constexpr int kTqQdo = 8 * 16384 + 8192;       // [Q_c | dO_c] c = 0..7, then Q_8
-constexpr int kTqSmem = 1024 + kTqQdo + kTqRing * kTqSlab + kTqSlab + 512 + 256;
+// Row operands of a CTA: eight 8 KB slabs (64 rows x 64 channels) -- Q_c in the even CTA, dO_c in
+// the odd one -- and the rope slab Q_8 of all 64 rows, placed so that the half of its rows a CTA
+// contributes (rows 0-31 even, 32-63 odd) starts at the same offset kTqRope in both.
+constexpr int kTqRope = 8 * 8192 + 4096;
+constexpr int kTqB = kTqRope + 8192;
+constexpr int kTqE = 2 * 8192;                 // E^T of the even and of the odd CTA's keys: this CTA's 32 rows of each
+constexpr int kTqEBufs = 2;                    // E^T buffers: step i + 1 is written while dQ^T of step i reads
+constexpr int kTqSmem = 1024 + kTqB + kTqRing * kTqSlab + kTqEBufs * kTqE + 512 + 256;
 constexpr float kLog2eTq = 1.4426950408889634f;
 
-__global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_constant__ MlaDqParams p) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
+    bwd_mla_dq_kernel(const __grid_constant__ MlaDqParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* qdo = smem;
-  uint8_t* ring = qdo + kTqQdo;
+  uint8_t* bop = smem;
+  uint8_t* ring = bop + kTqB;
   uint8_t* e_smem = ring + kTqRing * kTqSlab;
-  float2* rowp = reinterpret_cast<float2*>(e_smem + kTqSlab);     // (LSE * log2 e, Delta) of the 64 rows
-  uint64_t* bars = reinterpret_cast<uint64_t*>(e_smem + kTqSlab + 512);
-  uint64_t* a_full = bars;
-  uint64_t* full = bars + 1;
-  uint64_t* empty = full + kTqRing;
-  uint64_t* st_full = empty + kTqRing;
-  uint64_t* s_read = st_full + 1;
-  uint64_t* e_full = s_read + 1;
-  uint64_t* e_free = e_full + 1;
-  uint64_t* acc_final = e_free + 1;
+  float2* rowp = reinterpret_cast<float2*>(e_smem + kTqEBufs * kTqE);        // (LSE * log2 e, Delta) of the 64 rows
+  uint64_t* bars = reinterpret_cast<uint64_t*>(e_smem + kTqEBufs * kTqE + 512);
+  uint64_t* a_full = bars;               // (even CTA) the row operands of both CTAs landed
+  uint64_t* full = bars + 1;             // (even CTA) both CTAs' halves of a slot landed
+  uint64_t* empty = full + kTqRing;      // (each CTA)
+  uint64_t* st_full = empty + kTqRing;   // [2] (each CTA) one per [S^T | T^T] buffer
+  uint64_t* s_read = st_full + 2;        // [2] (even CTA) 8 warp arrivals: both CTAs hold the buffer's tile in registers
+  uint64_t* e_full = s_read + 2;         // [2] (even CTA) 8 warp arrivals: E^T of both CTAs' keys is written to the buffer
+  uint64_t* e_free = e_full + 2;         // [2] (each CTA) one per E^T buffer
+  uint64_t* acc_final = e_free + 2;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
   long long tw0 = 0, tw1 = 0, tw2 = 0, tw3 = 0;   // wait-time accumulators (only used with LS_TIMING)
   const long long t_begin = clock64();
-  // work item: row block (fastest, so that the CTAs in flight share the same keys), range of parts, KV head
-  const int qtile = blockIdx.x % p.nq_tiles;
-  const int split = (blockIdx.x / p.nq_tiles) % p.nsplit;
-  const int kvh = blockIdx.x / (p.nq_tiles * p.nsplit);
+  (void)tw0; (void)tw1; (void)tw2; (void)tw3; (void)t_begin;
+  // work item of the pair: row block (fastest, so that the pairs in flight share the same keys),
+  // range of parts, KV head
+  const int work = (int)(blockIdx.x >> 1);
+  const int qtile = work % p.nq_tiles;
+  const int split = (work / p.nq_tiles) % p.nsplit;
+  const int kvh = work / (p.nq_tiles * p.nsplit);
   const int h = kvh * p.g + (qtile / p.tiles_tok) * p.bh;     // first head and token of the block
   const int row0 = (qtile % p.tiles_tok) * p.bt;
-  // the parts this CTA walks: all of them, or (several CTAs per row block) a contiguous range
+  // the parts this pair walks: all of them, or (several pairs per row block) a contiguous range
   const int part_lo = (int)((long long)split * p.nparts / p.nsplit);
   const int part_hi = (int)((long long)(split + 1) * p.nparts / p.nsplit);
 
-  // key tiles of 128 over those parts (every role walks the same list)
-  int total_tiles = 0;
-  for (int r = part_lo; r < part_hi; ++r) total_tiles += (int)((p.shard_tokens[r] + 127) >> 7);
+  // steps of 256 keys over those parts: the even CTA takes the first 128-key tile of a step, the odd
+  // CTA the second (past a part's last tile: zeros, masked).  Every role walks the same list.
+  int total_steps = 0;
+  for (int r = part_lo; r < part_hi; ++r) total_steps += (int)((((p.shard_tokens[r] + 127) >> 7) + 1) >> 1);
 
   if (threadIdx.x == 0) {
     mbar_init(a_full, 1);
+    // A dQ^T slot completes only when BOTH producers have passed their wait for it (two arrivals): the
+    // odd CTA loads nothing for channel block 2, and without its arrival such a slot could be filled,
+    // consumed and released twice while that producer still waits for the first release.
     for (int i = 0; i < kTqRing; ++i) {
-      mbar_init(&full[i], 1);
+      mbar_init(&full[i], i < kTqStSlots ? 1 : 2);
       mbar_init(&empty[i], 1);
     }
-    mbar_init(st_full, 1);
-    mbar_init(s_read, 128);
-    mbar_init(e_full, 128);
-    mbar_init(e_free, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&st_full[i], 1);
+      mbar_init(&s_read[i], 8);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&e_full[i], 8);
+      mbar_init(&e_free[i], 1);
+    }
     mbar_init(acc_final, 1);
     *abort_flag = 0;
     fence_barrier_init();
@@ -135,148 +164,147 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
     rowp[t] = make_float2(p.lse[ri] * kLog2eTq, p.delta[ri]);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_holder, 512);
-    tmem_relinquish();
+    tmem_alloc_pair(tmem_holder, 512);
+    tmem_relinquish_pair();
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();                      // both CTAs' barriers exist before any remote signal
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
-  const uint32_t tmem_acc = tmem_base;          // 5 x 64 columns
-  const uint32_t tmem_st = tmem_base + 320;     // S^T [0,64) | T^T [64,128)
+  const uint32_t tmem_st = tmem_base;           // two buffers of S^T [0,64) | T^T [64,128) of this CTA's 128 keys
+  const uint32_t tmem_acc = tmem_base + 256;    // 3 x 64 columns: this CTA's 128 channels of each block
 
-  if (warp == 0) {
-    // =========================================================== producer (one thread)
-    // Two rings: slots [0, kTqStSlots) carry K-major slabs (128 keys x one channel group, two
-    // 64-token boxes) for [S^T | T^T]; the rest carry MN-major slots (64 keys x two channel
-    // groups, one box) for dQ^T.  The dQ^T loads of tile i are interleaved one to one with the
-    // [S^T | T^T] loads of tile i + 2, the order in which the two issuers consume them.
-    if (lane == 0 && total_tiles > 0) {
-      mbar_arrive_expect_tx(a_full, p.qdo_bytes);
-      for (int c = 0; c < 9; ++c) tma_load_5d(qdo + c * 16384, &p.q_map, a_full, 0, row0, c, h, 0);
-      for (int c = 0; c < 8; ++c) tma_load_5d(qdo + c * 16384 + 8192, &p.do_map, a_full, 0, row0, c, h, 0);
-
+  if (warp == 0 || warp == 7) {
+    // =========================================================== producers (two threads per CTA)
+    // Two rings, one producer thread each (a single thread issues a TMA instruction every ~200
+    // cycles, too slow for both): slots [0, kTqStSlots) carry K-major slabs (this CTA's 128 keys x
+    // one channel group, two 64-token boxes) for [S^T | T^T], filled by warp 0; the rest carry
+    // MN-major slots (64 keys of either CTA's tile x two of THIS CTA's channel groups, one box) for
+    // dQ^T, filled by warp 7.  Every load credits the even CTA's barrier of the slot.
+    if (lane == 0 && total_steps > 0) {
+      const bool st_role = warp == 0;
+      if (st_role) {
+        if (leader) mbar_arrive_expect_tx(a_full, p.qdo_bytes);
+        if (leader) {
+          for (int c = 0; c < 8; ++c) tma_load_5d_pair(bop + c * 8192, &p.q_map, a_full, 0, row0, c, h, 0);
+          tma_load_5d_pair(bop + kTqRope, &p.q_map, a_full, 0, row0, 8, h, 0);
+        } else {
+          for (int c = 0; c < 8; ++c) tma_load_5d_pair(bop + c * 8192, &p.do_map, a_full, 0, row0, c, h, 0);
+          tma_load_5d_pair(bop + kTqRope - 4096, &p.q_map, a_full, 0, row0, 8, h, 0);
+        }
+      }
       const int pg_mask = (1 << p.pg_shift) - 1;
       bool ok = true;
-      // A walk over the key tiles of all partials; everything that needs global memory (the two
-      // 64-token boxes of a tile) is resolved once per tile.
-      struct Walk {
-        int part, tile, c_off, c_pages, c_tail, c_tiles;
-        int page[2], tok[2];
-        bool tail[2];
-      };
-      auto open_part = [&](Walk& w, int r) {
-        w.part = r;
-        w.c_off = p.shard_page_offset[r];
-        w.c_pages = p.shard_page_offset[r + 1] - w.c_off;
-        w.c_tail = p.shard_tail_slot[r];
-        w.c_tiles = (int)((p.shard_tokens[r] + 127) >> 7);
-      };
-      auto next_tile = [&](Walk& w) {
-        ++w.tile;
-        while (w.part < part_hi && w.tile >= w.c_tiles) {
-          w.tile = 0;
-          if (w.part + 1 < part_hi) open_part(w, w.part + 1); else ++w.part;
-        }
-        if (w.part >= part_hi) return;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const int tok = w.tile * 128 + half * 64;
-          const int ps = tok >> p.pg_shift;
-          // past the part's last page: a coordinate beyond the pool, where TMA fills zeros (the bytes of
-          // an arbitrary page could be NaN patterns, and 0 * NaN would poison dQ^T)
-          w.page[half] = ps < w.c_pages ? __ldg(p.shard_phys_pages + w.c_off + ps) : p.num_phys_pages;
-          w.tok[half] = tok & pg_mask;
-          w.tail[half] = ps == w.c_tail;
+      // a walk over the 256-key steps of the parts; a step is four 64-token boxes, resolved by `box`
+      int part = part_lo, step = -1;
+      int c_off = p.shard_page_offset[part], c_pages = p.shard_page_offset[part + 1] - c_off;
+      int c_tail = p.shard_tail_slot[part], c_steps = (int)((((p.shard_tokens[part] + 127) >> 7) + 1) >> 1);
+      auto next_step = [&]() {
+        ++step;
+        while (step >= c_steps) {          // (the caller stops after total_steps steps)
+          ++part;
+          step = 0;
+          c_off = p.shard_page_offset[part];
+          c_pages = p.shard_page_offset[part + 1] - c_off;
+          c_tail = p.shard_tail_slot[part];
+          c_steps = (int)((((p.shard_tokens[part] + 127) >> 7) + 1) >> 1);
         }
       };
-      uint32_t s_seq = 0, a_seq = 0, issued_s = 0, issued_a = 0;
-      auto load_st = [&](const Walk& w, int c) {          // channel group c of the tile
-        const uint32_t slot = s_seq % kTqStSlots, lap = s_seq / kTqStSlots;
-        ok = ok && LS_TQWAIT(tw0, mbar_wait(&empty[slot], (lap & 1) ^ 1, abort_flag));
-        if (ok) {
-          uint8_t* dst = ring + slot * kTqSlab;
-          if (LS_TQABLATE(1)) {
-            mbar_arrive(&full[slot]);
-          } else {
-            mbar_arrive_expect_tx(&full[slot], kTqSlab);
-            tma_load_5d(dst, w.tail[0] ? &p.k_tail : &p.k_map, &full[slot], 0, w.tok[0], c, kvh, w.page[0]);
-            tma_load_5d(dst + 8192, w.tail[1] ? &p.k_tail : &p.k_map, &full[slot], 0, w.tok[1], c, kvh, w.page[1]);
-          }
-          ++issued_s;
-        }
-        ++s_seq;
+      // box q of the step: physical page, first token inside it, and whether it is the pool's partly
+      // filled last page.  Past the part's last page: a coordinate beyond the pool, where TMA fills zeros
+      // (the bytes of an arbitrary page could be NaN patterns, and 0 * NaN would poison dQ^T).
+      auto box = [&](int q, int& page, int& tok, bool& tail) {
+        const int t = step * 256 + q * 64;
+        const int ps = t >> p.pg_shift;
+        page = ps < c_pages ? __ldg(p.shard_phys_pages + c_off + ps) : p.num_phys_pages;
+        tok = t & pg_mask;
+        tail = ps == c_tail;
       };
-      auto load_acc = [&](const Walk& w, int k) {         // k = half * 5 + channel-group pair
-        const uint32_t slot = kTqStSlots + a_seq % kTqAccSlots, lap = a_seq / kTqAccSlots;
-        ok = ok && LS_TQWAIT(tw1, mbar_wait(&empty[slot], (lap & 1) ^ 1, abort_flag));
-        if (ok) {
-          const int half = k >= 5 ? 1 : 0, m = k - half * 5;
-          if (LS_TQABLATE(1)) {
-            mbar_arrive(&full[slot]);
-          } else {
-            mbar_arrive_expect_tx(&full[slot], kTqSlab);
-            tma_load_5d(ring + slot * kTqSlab, w.tail[half] ? &p.k2_tail : &p.k2_map, &full[slot], 0, w.tok[half],
-                        2 * m, kvh, w.page[half]);
-          }
-          ++issued_a;
-        }
-        ++a_seq;
-      };
-      Walk ws, wa;
-      ws.tile = -1;
-      open_part(ws, part_lo);
-      wa = ws;
-      next_tile(ws);
+      uint32_t seq = 0, issued = 0;
+      if (st_role) {
+        for (int i = 0; i < total_steps && ok; ++i) {
+          next_step();
+          int pg0, pg1, tk0, tk1;
+          bool tl0, tl1;
+          box(2 * (int)rank, pg0, tk0, tl0);
+          box(2 * (int)rank + 1, pg1, tk1, tl1);
+          const CUtensorMap* m0 = tl0 ? &p.k_tail : &p.k_map;
+          const CUtensorMap* m1 = tl1 ? &p.k_tail : &p.k_map;
 #pragma unroll 1
-      for (int c = 0; c < 9; ++c) load_st(ws, c);          // tile 0
-      if (total_tiles > 1) {
-        next_tile(ws);
-#pragma unroll 1
-        for (int c = 0; c < 9; ++c) load_st(ws, c);        // tile 1
-      }
-      for (int i = 0; i < total_tiles && ok; ++i) {
-        const bool has_st = i + 2 < total_tiles;
-        if (has_st) next_tile(ws);
-        next_tile(wa);
-#pragma unroll
-        for (int k = 0; k < 10; ++k) {
-          if (has_st && k < 9) load_st(ws, k);
-          load_acc(wa, k);
+          for (int c = 0; c < 9; ++c) {          // channel group c of this CTA's tile of the step
+            const uint32_t slot = seq % kTqStSlots, lap = seq / kTqStSlots;
+            ok = ok && LS_TQWAIT(tw0, mbar_wait(&empty[slot], (lap & 1) ^ 1, abort_flag));
+            if (!ok) break;
+            uint8_t* dst = ring + slot * kTqSlab;
+            if (leader) mbar_arrive_expect_tx(&full[slot], 2 * kTqSlab);
+            tma_load_5d_pair(dst, m0, &full[slot], 0, tk0, c, kvh, pg0);
+            tma_load_5d_pair(dst + 8192, m1, &full[slot], 0, tk1, c, kvh, pg1);
+            ++issued;
+            ++seq;
+          }
         }
+        LS_TQDUMP(0, tw0);
+        LS_TQDUMP(1, clock64() - t_begin);
+      } else {
+        const uint32_t full_remote = mapa_u32(smem_u32(&full[kTqStSlots]), 0);
+        for (int i = 0; i < total_steps && ok; ++i) {
+          next_step();
+          int pg[4], tk[4];
+          bool tl[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) box(q, pg[q], tk[q], tl[q]);
+          // k = (tile of the step) * 6 + (channel block) * 2 + (64-key half): channel block m is groups
+          // 4m, 4m+1 in the even CTA (group 9 does not exist and reads as zeros) and 4m+2, 4m+3 in the
+          // odd CTA, which has nothing to load for block 2.
+#pragma unroll
+          for (int k = 0; k < 12; ++k) {
+            const int j = k / 6, m = (k % 6) >> 1, q = 2 * j + (k & 1);
+            const uint32_t sl = seq % kTqAccSlots, lap = seq / kTqAccSlots;
+            const uint32_t slot = kTqStSlots + sl;
+            ok = ok && LS_TQWAIT(tw1, mbar_wait(&empty[slot], (lap & 1) ^ 1, abort_flag));
+            if (!ok) break;
+            if (leader) mbar_arrive_expect_tx(&full[slot], m < 2 ? 2 * kTqSlab : kTqSlab / 2);
+            else mbar_arrive_cluster(full_remote + sl * 8);
+            if (m < 2)
+              tma_load_5d_pair(ring + slot * kTqSlab, tl[q] ? &p.k2_tail : &p.k2_map, &full[slot], 0, tk[q],
+                               4 * m + 2 * (int)rank, kvh, pg[q]);
+            else if (leader)      // the rope group alone: the other half of the slot feeds accumulator lanes nobody reads
+              tma_load_5d_pair(ring + slot * kTqSlab, tl[q] ? &p.k_tail : &p.k_map, &full[slot], 0, tk[q], 8, kvh,
+                               pg[q]);
+            ++issued;
+            ++seq;
+          }
+        }
+        LS_TQDUMP(2, tw1);
+        LS_TQDUMP(3, clock64() - t_begin);
       }
-      LS_TQDUMP(0, tw0);
-      LS_TQDUMP(2, tw1);
-      LS_TQDUMP(1, clock64() - t_begin);
-      if (*abort_flag) {   // aborted: wait (bounded) for the copies already started
-        for (int s = 0; s < kTqRing; ++s) {
-          const bool st_ring = s < kTqStSlots;
-          const uint32_t n = st_ring ? issued_s : issued_a, per = st_ring ? kTqStSlots : kTqAccSlots;
-          const uint32_t idx = st_ring ? s : s - kTqStSlots;
-          if (n <= idx) continue;
-          const uint32_t last_lap = (n - 1 - idx) / per;
+      if (*abort_flag && leader) {   // aborted: wait (bounded) for the copies credited to this CTA's barriers
+        const uint32_t per = st_role ? kTqStSlots : kTqAccSlots, first = st_role ? 0 : kTqStSlots;
+        for (uint32_t idx = 0; idx < per && idx < issued; ++idx) {
+          const uint32_t last_lap = (issued - 1 - idx) / per;
           const uint64_t t_start = globaltimer_ns();
-          while (!mbar_try_wait(&full[s], last_lap & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
+          while (!mbar_try_wait(&full[first + idx], last_lap & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
           }
         }
       }
     }
   } else if (warp == 1) {
-    // =========================================================== [S^T | T^T] issuer (one thread)
+    // =========================================================== [S^T | T^T] issuer (one thread of the even CTA)
     // The two kinds of products are issued by two threads (this one and one of warp 6), each
     // from its own ring: they write disjoint TMEM columns and each thread's own instructions
     // stay in order, so the per-slot bookkeeping of one overlaps the other's.
-    if (lane == 0 && total_tiles > 0) {
-      constexpr uint32_t idesc_st = make_idesc(128, 128, 0, 0);
-      constexpr uint32_t idesc_rope = make_idesc(128, 64, 0, 0);
+    if (leader && lane == 0 && total_steps > 0) {
+      constexpr uint32_t idesc_st = make_idesc(256, 128, 0, 0);
+      constexpr uint32_t idesc_rope = make_idesc(256, 64, 0, 0);
       constexpr uint32_t hi = sdesc_hi(1024);
-      const uint32_t qdo_lo = sdesc_lo(smem_u32(qdo), 16);
+      const uint32_t b_lo = sdesc_lo(smem_u32(bop), 16);
       const uint32_t ring_k_lo = sdesc_lo(smem_u32(ring), 16);          // K-major: 128 keys x 64 channels
       bool ok = mbar_wait(a_full, 0, abort_flag);
       uint32_t seq = 0;
-      for (int i = 0; i < total_tiles && ok; ++i) {
-        if (i > 0) {
-          ok = LS_TQWAIT(tw2, mbar_wait(s_read, (i - 1) & 1, abort_flag));   // tile i - 1 is in registers
+      for (int i = 0; i < total_steps && ok; ++i) {
+        if (i > 1) {      // the buffer's previous tile (step i - 2) is in registers
+          ok = LS_TQWAIT(tw2, mbar_wait(&s_read[i & 1], ((i >> 1) - 1) & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
         }
@@ -289,35 +317,36 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
           const uint32_t a_lo = ring_k_lo + slot * (kTqSlab >> 4);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            if (!LS_TQABLATE(2))
-              mma_ss(tmem_st, sdesc(a_lo + ((k * 32) >> 4), hi), sdesc(qdo_lo + ((c * 16384 + k * 32) >> 4), hi),
-                     c < 8 ? idesc_st : idesc_rope, (c | k) != 0);
-          mma_commit(&empty[slot]);
+            mma_ss_pair(tmem_st + (i & 1) * 128, sdesc(a_lo + ((k * 32) >> 4), hi),
+                        sdesc(b_lo + (((c < 8 ? c * 8192 : kTqRope) + k * 32) >> 4), hi),
+                        c < 8 ? idesc_st : idesc_rope, (c | k) != 0);
+          mma_commit_pair(&empty[slot]);
           ++seq;
         }
         if (!ok) break;
-        mma_commit(st_full);
+        mma_commit_pair(&st_full[i & 1]);
       }
       LS_TQDUMP(8, tw0);
       LS_TQDUMP(10, tw2);
       LS_TQDUMP(12, clock64() - t_begin);
     }
   } else if (warp == 6) {
-    // =========================================================== dQ^T issuer (one thread)
-    if (lane == 0 && total_tiles > 0) {
-      constexpr uint32_t idesc_acc = make_idesc(128, 64, 1, 1);
+    // =========================================================== dQ^T issuer (one thread of the even CTA)
+    if (leader && lane == 0 && total_steps > 0) {
+      constexpr uint32_t idesc_acc = make_idesc(256, 64, 1, 1);
       constexpr uint32_t hi = sdesc_hi(1024);
+      constexpr uint32_t hi_e = sdesc_hi_sw64(512);
       const uint32_t ring_m_lo = sdesc_lo(smem_u32(ring), 8192);        // MN-major: 64 keys x two channel groups
-      const uint32_t e_lo = sdesc_lo(smem_u32(e_smem), 16);             // MN-major: keys x 64 rows
+      const uint32_t e_lo = sdesc_lo(smem_u32(e_smem), 512);            // MN-major, 64-byte lines: 128 keys x 32 rows per tile
       bool ok = true;
       uint32_t seq = 0;
-      for (int i = 0; i < total_tiles && ok; ++i) {
-        ok = LS_TQWAIT(tw3, mbar_wait(e_full, i & 1, abort_flag));
+      for (int i = 0; i < total_steps && ok; ++i) {
+        ok = LS_TQWAIT(tw3, mbar_wait_cluster(&e_full[i & 1], (i >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < 10; ++k) {
-          const int half = k >= 5 ? 1 : 0, m = k - half * 5;
+        for (int k = 0; k < 12; ++k) {
+          const int j = k / 6, m = (k % 6) >> 1, kh = k & 1;
           const uint32_t slot = kTqStSlots + seq % kTqAccSlots, lap = seq / kTqAccSlots;
           ok = ok && LS_TQWAIT(tw1, mbar_wait(&full[slot], lap & 1, abort_flag));
           if (!ok) break;
@@ -325,15 +354,15 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
           const uint32_t a_lo = ring_m_lo + slot * (kTqSlab >> 4);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)
-            if (!LS_TQABLATE(2))
-              mma_ss(tmem_acc + m * 64, sdesc(a_lo + ((kk * 2048) >> 4), hi),
-                     sdesc(e_lo + ((half * 8192 + kk * 2048) >> 4), hi), idesc_acc, (i | half | kk) != 0);
-          mma_commit(&empty[slot]);
+            mma_ss_pair(tmem_acc + m * 64, sdesc(a_lo + ((kk * 2048) >> 4), hi),
+                        sdesc(e_lo + (((i & 1) * kTqE + j * 8192 + kh * 4096 + kk * 1024) >> 4), hi_e), idesc_acc,
+                        (i | j | kh | kk) != 0);
+          mma_commit_pair(&empty[slot]);
           ++seq;
         }
         if (!ok) break;
-        mma_commit(e_free);
-        if (i == total_tiles - 1) mma_commit(acc_final);
+        mma_commit_pair(&e_free[i & 1]);
+        if (i == total_steps - 1) mma_commit_pair(acc_final);
       }
       LS_TQDUMP(9, tw1);
       LS_TQDUMP(11, tw3);
@@ -342,34 +371,42 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
   } else {
     // =========================================================== one thread per key: E^T, epilogue
     const int quad = warp & 3;
-    const int key = quad * 32 + lane;                      // TMEM lane = key of the tile
+    const int key = quad * 32 + lane;                      // TMEM lane = key of this CTA's tile
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
-    uint8_t* e_row = e_smem + key * 128;
-    const int sw = key & 7;
-    if (total_tiles > 0) {
+    // E^T of this CTA's keys, MN-major [key][row] in 64-byte lines (64-byte swizzle): rows 0-31 go
+    // to the even CTA's copy, rows 32-63 to the odd CTA's, each at offset rank * 8 KB of the E^T area
+    const uint32_t e_mine = smem_u32(e_smem) + rank * 8192 + (key >> 3) * 512 + (key & 7) * 64;
+    const uint32_t e_dst[2] = {mapa_u32(e_mine, 0), mapa_u32(e_mine, 1)};
+    const uint32_t sw = (uint32_t)(key & 7) >> 1;
+    const uint32_t s_read_remote[2] = {mapa_u32(smem_u32(&s_read[0]), 0), mapa_u32(smem_u32(&s_read[1]), 0)};
+    const uint32_t e_full_remote[2] = {mapa_u32(smem_u32(&e_full[0]), 0), mapa_u32(smem_u32(&e_full[1]), 0)};
+    if (total_steps > 0) {
       bool ok = true;
-      int part = part_lo, tile = -1;
-      for (int i = 0; i < total_tiles && ok; ++i) {
-        ++tile;
-        while (tile >= (int)((p.shard_tokens[part] + 127) >> 7)) {
+      int part = part_lo, step = -1;
+      for (int i = 0; i < total_steps && ok; ++i) {
+        ++step;
+        while (step >= (int)((((p.shard_tokens[part] + 127) >> 7) + 1) >> 1)) {
           ++part;
-          tile = 0;
+          step = 0;
         }
-        const bool valid = (int64_t)tile * 128 + key < p.shard_tokens[part];
-        ok = LS_TQWAIT(tw0, mbar_wait(st_full, i & 1, abort_flag));
+        const bool valid = ((int64_t)(2 * step + (int)rank)) * 128 + key < p.shard_tokens[part];
+        ok = LS_TQWAIT(tw0, mbar_wait(&st_full[i & 1], (i >> 1) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t tst = tmem_st + (i & 1) * 128 + lane_sel;
         uint32_t pk[32];
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
           uint32_t sr[32], tr[32];
-          tmem_ld32(tmem_st + lane_sel + half * 32, sr);
-          tmem_ld32(tmem_st + lane_sel + 64 + half * 32, tr);
+          tmem_ld32(tst + half * 32, sr);
+          tmem_ld32(tst + 64 + half * 32, tr);
           tc_wait_ld32(sr);
           tc_wait_ld32(tr);
-          if (half == 1) {          // the whole buffer is in registers: the next tile may overwrite it
+          if (half == 1) {          // the whole buffer is in registers: the next step may overwrite it
             tc_fence_before();
-            mbar_arrive(s_read);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(s_read_remote[i & 1]);
           }
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
@@ -384,16 +421,20 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
 #pragma unroll
           for (int j = 0; j < 32; ++j) pk[j] = 0u;
         }
-        if (i > 0) {
-          ok = LS_TQWAIT(tw1, mbar_wait(e_free, (i - 1) & 1, abort_flag));   // the previous tile's dQ^T instructions have read E^T
+        if (i > 1) {      // the dQ^T instructions of step i - 2 have read this E^T buffer
+          ok = LS_TQWAIT(tw1, mbar_wait(&e_free[i & 1], ((i >> 1) - 1) & 1, abort_flag));
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-          *reinterpret_cast<uint4*>(e_row + ((j ^ sw) << 4)) =
-              make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-        fence_proxy_async();
-        mbar_arrive(e_full);
+        for (int c = 0; c < 2; ++c)          // destination CTA = half of the rows
+#pragma unroll
+          for (int q = 0; q < 4; ++q)        // 16-byte chunk: rows 32 c + 8 q .. + 7
+            st_shared_cluster_v4(e_dst[c] + (i & 1) * kTqE + (((uint32_t)q ^ sw) << 4), pk[16 * c + 4 * q], pk[16 * c + 4 * q + 1],
+                                 pk[16 * c + 4 * q + 2], pk[16 * c + 4 * q + 3]);
+        fence_proxy_async_all();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster_release(e_full_remote[i & 1]);
       }
       if (threadIdx.x == 64) {
         LS_TQDUMP(16, tw0);
@@ -401,12 +442,13 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
         LS_TQDUMP(18, clock64() - t_begin);
       }
       if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
 #pragma unroll 1
-        for (int m = 0; m < 5; ++m) {
-          if (m == 4 && quad >= 2) break;                   // channels 576.. do not exist
-          const int ch = m * 128 + key;
+        for (int m = 0; m < 3; ++m) {
+          if (m == 2 && (!leader || quad >= 2)) break;      // block 2 is the 64 rope channels, in the even CTA
+          const int ch = m * 256 + (int)rank * 128 + key;
 #pragma unroll 1
           for (int half = 0; half < 2; ++half) {
             uint32_t o[32];
@@ -433,12 +475,13 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
       }
     } else if (p.nsplit > 1) {
       // an empty range of parts still owes its (zero) partial to the reduce kernel
-      for (int m = 0; m < 5; ++m) {
-        if (m == 4 && quad >= 2) break;
+      for (int m = 0; m < 3; ++m) {
+        if (m == 2 && (!leader || quad >= 2)) break;
+        const int ch = m * 256 + (int)rank * 128 + key;
         for (int rr = 0; rr < p.bt * p.bh; ++rr) {
           const int r = row0 + rr % p.bt, hh = h + rr / p.bt;
           if (r < p.R && hh < (kvh + 1) * p.g)
-            p.dq_split[(size_t)split * p.R * p.Hq * 576 + ((size_t)r * p.Hq + hh) * 576 + m * 128 + key] = 0.f;
+            p.dq_split[(size_t)split * p.R * p.Hq * 576 + ((size_t)r * p.Hq + hh) * 576 + ch] = 0.f;
         }
       }
     }
@@ -446,9 +489,10 @@ __global__ void __launch_bounds__(kTqThreads, 1) bwd_mla_dq_kernel(const __grid_
 
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();          // neither CTA leaves while the other may still touch its shared memory
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc_pair(tmem_base, 512);
   }
   if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
 }
@@ -461,9 +505,9 @@ bool mla_dq_fast(const ls_pages* h) {
 int mla_dq_splits(const ls_pages* h, int R, int Hq) {
   const int Hkv = h->desc.num_kv_heads;
   const int64_t blocks = (int64_t)Hkv * row_tiling(R, Hq / Hkv, kTqRows).nq_tiles;
-  if (blocks >= 148) return 1;                 // enough row blocks: every CTA walks all parts
-  // few rows: the parts are spread over enough CTAs to fill the GPU twice
-  return std::max(1, std::min(h->prefix_parts(), (int)((148 * 2 + blocks - 1) / blocks)));
+  if (blocks >= 74) return 1;                  // enough row blocks for every CTA pair: each walks all parts
+  // few rows: the parts are spread over enough CTA pairs to fill the GPU twice
+  return std::max(1, std::min(h->prefix_parts(), (int)((148 + blocks - 1) / blocks)));
 }
 
 // dq = scale * (sum of the split partials + the response block's partial), bf16
@@ -515,7 +559,7 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   P.bh = rt.bh;
   P.tiles_tok = rt.tiles_tok;
   P.nq_tiles = rt.nq_tiles;
-  P.qdo_bytes = (9 + 8) * rt.bt * rt.bh * 128;
+  P.qdo_bytes = (9 + 9) * rt.bt * rt.bh * 128;      // Q (even CTA), dO and the rope slab of Q (odd CTA)
   P.nsplit = dq_split ? mla_dq_splits(h, R, Hq) : 1;     // without scratch every CTA walks all parts
   P.dq_split = dq_split;
   ls_status_t st = encode_map_rows(&P.q_map, q, 576, R, Hq, rt.bt, rt.bh);
@@ -528,7 +572,7 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   static bool configured[64] = {};
   const ls_status_t cfg = configure_smem(bwd_mla_dq_kernel, kTqSmem, configured);
   if (cfg != LS_OK) return cfg;
-  const int64_t grid = (int64_t)d.num_kv_heads * rt.nq_tiles * P.nsplit;
+  const int64_t grid = (int64_t)d.num_kv_heads * rt.nq_tiles * P.nsplit * 2;     // CTA pairs
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   profile_begin(LS_KERNEL_BWD_DQ, cs);
   bwd_mla_dq_kernel<<<(int)grid, kTqThreads, kTqSmem, cs>>>(P);

@@ -39,6 +39,8 @@ struct FwdParams {
   CUtensorMap kr_map, vr_map;      // response K (64 x 128 x KSLABS) and V (64 x VKEYS x DVT/64)
   // CTA-pair variant (D = 256): every box is 64 channels x 64 tokens x 2 groups (16 KB)
   CUtensorMap pk2, pk2_tail, pv2, pv2_tail, rk2, rv2;
+  // the odd ninth channel group of the 576-wide key: 64 channels x 64 tokens x 1 group (8 KB)
+  CUtensorMap pk1, pk1_tail, rk1;
   const int32_t* part_pages;
   const int32_t* part_page_offset;
   const int32_t* part_tail_slot;
@@ -582,24 +584,30 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_kernel(const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------
-// Forward on CTA pairs (cta_group::2), head dim 256.  Two neighbouring SMs take two Q tiles of
-// the same (KV head, partial) and stream the keys once between them: for S each CTA loads 64
-// of the 128 keys of a tile, for P V each loads 128 of the 256 value channels, so shared-memory
-// writes and L2 reads halve and the ring covers two tiles.  One thread of the even CTA issues
-// all MMAs (256 rows); completions are multicast to both CTAs' barriers; the odd CTA's softmax
-// warps report P to the even CTA's barrier.  Chunks are 16 KB: 64 tokens x 128 channels.
+// Forward on CTA pairs (cta_group::2), head dim 256 and the 576/512 shape.  Two neighbouring SMs
+// take two Q tiles of the same (KV head, partial) and stream the keys once between them: for S
+// each CTA loads 64 of the 128 keys of a tile, for P V each loads 128 of the 256 value channels,
+// so shared-memory writes and L2 reads halve and the ring covers more tiles.  One thread of the
+// even CTA issues all MMAs (256 rows); completions are multicast to both CTAs' barriers; the odd
+// CTA's softmax warps report P to the even CTA's barrier.  Chunks are 16 KB: 64 tokens x 128
+// channels (the ninth 64-channel group of a 576-wide key travels alone, 8 KB in a slot of its own).
+// With 512 value channels a pair of Q tiles is NDV = 2 work items, one per 256-channel half of O
+// (O of 128 rows x 512 channels alone would fill the 512 TMEM columns).
 // ---------------------------------------------------------------------------------
+template <int DK>
 struct Fwd2Cfg {
-  static constexpr int D = 256;
+  static constexpr int KG = DK / 64;                  // 64-channel groups of a key
+  static constexpr int NKC = (KG + 1) / 2;            // key chunks per tile and CTA
   static constexpr int CHUNK = 16384;
-  static constexpr int RING = 8;
-  static constexpr int Q_BYTES = 4 * 16384;
+  static constexpr int RING = DK == 256 ? 8 : 5;
+  static constexpr int Q_BYTES = KG * 16384;
   static constexpr int SMEM_BYTES = 1024 + Q_BYTES + RING * CHUNK + 512;
 };
 
+template <int DK, int NDV>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     fwd2_kernel(const __grid_constant__ FwdParams p) {
-  using C = Fwd2Cfg;
+  using C = Fwd2Cfg<DK>;
   constexpr int DV = 256;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -618,6 +626,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   int* work_idx = const_cast<int*>(abort_flag) + 1;   // (even CTA) the pair's work item
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  long long tw0 = 0, tw1 = 0, tw2 = 0;   // wait-time accumulators (only used with LS_TIMING)
+  const long long t_begin = clock64();
+  (void)tw0; (void)tw1; (void)tw2; (void)t_begin;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
 
@@ -652,7 +663,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
 
   // ---- work item of the pair, and this CTA's Q tile
   const int npairs = (p.nq_tiles + 1) / 2;
-  const FwdItem it = fwd_item(p, (int)ld_shared_cluster_u32(mapa_u32(smem_u32(work_idx), 0)), npairs);
+  int widx = (int)ld_shared_cluster_u32(mapa_u32(smem_u32(work_idx), 0));
+  const int dvh = widx % NDV;           // which 256-wide slice of the value channels
+  widx /= NDV;
+  const FwdItem it = fwd_item(p, widx, npairs);
   const int pairi = it.qunit, part = it.part, kvh = it.kvh;
   const bool is_resp = it.is_resp;
   auto tile_of = [&](int qt, int& hh, int& r0) {
@@ -684,7 +698,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
       if (leader) mbar_arrive_expect_tx(q_full, 2 * p.q_bytes);
-      for (int c = 0; c < 4; ++c) tma_load_5d_pair(q_smem + c * 16384, &p.q_map, q_full, 0, t0, c, h, 0);
+      for (int c = 0; c < C::KG; ++c) tma_load_5d_pair(q_smem + c * 16384, &p.q_map, q_full, 0, t0, c, h, 0);
       const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
       auto page_at = [&](int tok) -> int {
@@ -694,34 +708,37 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
       };
       uint32_t slot = 0, phase = 0, issued = 0;
       bool ok = true;
-      // one chunk: 64 tokens starting at `tok` x channel groups [grp, grp + 2) of K (which = 0) or V
-      auto load = [&](int which, int tok, int grp, int page) {
-        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
+      // one chunk: 64 tokens starting at `tok` x channel groups [grp, grp + 2) of K (which = 0) or V;
+      // single: the lone last group of an odd group count (8 KB)
+      auto load = [&](int which, int tok, int grp, int page, bool single) {
+        ok = ok && LS_TWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
         if (ok) {
-          if (leader) mbar_arrive_expect_tx(&full[slot], 2 * C::CHUNK);
+          if (leader) mbar_arrive_expect_tx(&full[slot], single ? C::CHUNK : 2 * C::CHUNK);
           uint8_t* dst = ring + slot * C::CHUNK;
           if (is_resp) {
-            tma_load_5d_pair(dst, which ? &p.rv2 : &p.rk2, &full[slot], 0, tok, grp, kvh, 0);
+            tma_load_5d_pair(dst, which ? &p.rv2 : (single ? &p.rk1 : &p.rk2), &full[slot], 0, tok, grp, kvh, 0);
           } else {
             const bool tail = (tok >> p.pg_shift) == tail_slot;
-            const CUtensorMap* m = which ? (tail ? &p.pv2_tail : &p.pv2) : (tail ? &p.pk2_tail : &p.pk2);
+            const CUtensorMap* m = which    ? (tail ? &p.pv2_tail : &p.pv2)
+                                   : single ? (tail ? &p.pk1_tail : &p.pk1)
+                                            : (tail ? &p.pk2_tail : &p.pk2);
             tma_load_5d_pair(dst, m, &full[slot], 0, tok & pg_mask, grp, kvh, page);
           }
         }
         ++issued;
         if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
       };
-      // K of tile i for S: this CTA's 64 keys, two chunks of 128 channels.
-      // V of tile i for P V: both 64-key halves, this CTA's 128 channels.
+      // K of tile i for S: this CTA's 64 keys, chunks of 128 channels.
+      // V of tile i for P V: both 64-key halves, this CTA's 128 of the work item's 256 channels.
       auto load_k = [&](int i, int pa, int pb) {
         const int tok = i * 128 + (int)rank * 64;
         const int pg = rank ? pb : pa;
-        load(0, tok, 0, pg);
-        load(0, tok, 2, pg);
+#pragma unroll
+        for (int c = 0; c < C::NKC; ++c) load(0, tok, 2 * c, pg, 2 * c + 1 == C::KG);
       };
       auto load_v = [&](int i, int pa, int pb) {
-        load(1, i * 128, 2 * (int)rank, pa);
-        load(1, i * 128 + 64, 2 * (int)rank, pb);
+        load(1, i * 128, 4 * dvh + 2 * (int)rank, pa, false);
+        load(1, i * 128 + 64, 4 * dvh + 2 * (int)rank, pb, false);
       };
       // pages of the two 64-key halves of tile i (equal unless the pages hold 64 tokens)
       int pa0 = page_at(0), pb0 = page_at(64), pa1 = page_at(128), pb1 = page_at(192);
@@ -733,6 +750,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
         load_v(i, pa0, pb0);
         pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
       }
+      LS_TDUMP(0, tw0);
+      LS_TDUMP(1, clock64() - t_begin);
       if (*abort_flag && leader) {   // aborted: wait (bounded) for the copies credited to this CTA's barriers
         for (uint32_t s2 = 0; s2 < (uint32_t)C::RING && s2 < issued; ++s2) {
           const uint32_t last = ((issued - 1 - s2) / C::RING) * C::RING + s2;
@@ -759,17 +778,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
       auto issue_s = [&](int tile) {
         const uint32_t d = tmem_s0 + (tile & 1) * 128;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+        for (int c = 0; c < C::NKC; ++c) {
+          ok = ok && LS_TWAIT(tw1, mbar_wait(&full[slot], phase, abort_flag));
           if (!ok) return;
           tc_fence_after();
           const uint32_t b_lo = ring_k_lo + slot * (C::CHUNK >> 4);
 #pragma unroll
-          for (int s2 = 0; s2 < 2; ++s2)
+          for (int s2 = 0; s2 < 2; ++s2) {
+            if (2 * c + s2 >= C::KG) break;
 #pragma unroll
             for (int k = 0; k < 4; ++k)
               mma_ss_pair(d, sdesc(q_lo + (((2 * c + s2) * 16384 + k * 32) >> 4), hi),
                           sdesc(b_lo + ((s2 * 8192 + k * 32) >> 4), hi), idesc_s, (c | s2 | k) != 0);
+          }
           mma_commit_pair(&empty[slot]);
           advance();
         }
@@ -779,7 +800,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
         const uint32_t a_base = tmem_s0 + (tile & 1) * 128;   // P over the S columns
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+          ok = ok && LS_TWAIT(tw1, mbar_wait(&full[slot], phase, abort_flag));
           if (!ok) return;
           tc_fence_after();
           const uint32_t b_lo = ring_v_lo + slot * (C::CHUNK >> 4);
@@ -796,11 +817,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
       if (ok) issue_s(0);
       for (int i = 0; i < n_tiles && ok; ++i) {
         if (i + 1 < n_tiles) issue_s(i + 1);
-        ok = ok && mbar_wait(&p_full[i & 1], (i >> 1) & 1, abort_flag);
+        ok = ok && LS_TWAIT(tw2, mbar_wait(&p_full[i & 1], (i >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         issue_pv(i);
       }
+      LS_TDUMP(9, tw1);
+      LS_TDUMP(10, tw2);
+      LS_TDUMP(11, clock64() - t_begin);
+      LS_TDUMP(12, n_tiles);
     }
   } else {
     // =========================================================== softmax + epilogue (both CTAs)
@@ -813,8 +838,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const size_t out_row = ((size_t)fwd_out_part(p, it) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
     const bool to_resp = is_resp && p.chain_mode != 2;
-    float* o_dst = (to_resp ? p.o_resp : p.o_out) + out_row * p.dv_total;
+    float* o_dst = (to_resp ? p.o_resp : p.o_out) + out_row * p.dv_total + dvh * DV;
     float* lse_dst = (to_resp ? p.lse_resp : p.lse_out) + out_row;
+    if (dvh != 0 && it.chained) lse_dst = p.lse_aux + out_row;     // the second O half's chain keeps its own copy of l
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     if (n_tiles > 0) {
@@ -823,7 +849,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
       const uint32_t p_remote[2] = {mapa_u32(smem_u32(&p_full[0]), 0), mapa_u32(smem_u32(&p_full[1]), 0)};
       for (int i = 0; i < n_tiles && ok; ++i) {
         const uint32_t ts = tmem_s0 + (i & 1) * 128 + lane_sel;
-        ok = mbar_wait_warp(&s_full[i & 1], (i >> 1) & 1, abort_flag);
+        ok = LS_TWAIT(tw0, mbar_wait_warp(&s_full[i & 1], (i >> 1) & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         uint32_t sr[128];
@@ -888,17 +914,22 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(p_remote[i & 1]);   // one arrival per warp, at the even CTA
       }
+      if (threadIdx.x == 64) {
+        LS_TDUMP(16, tw0);
+        LS_TDUMP(18, clock64() - t_begin);
+      }
       if (ok) ok = mbar_wait_warp(o_final, 0, abort_flag);
       if (ok) tc_fence_after();
     }
     // ---- epilogue: store this partial, or fold it into the running value of its chain
     const bool chained = it.chained && tile_ok;
-    int* counter = chained ? p.ctl + kChainHeaderInts + fwd_chain_index(p, it, qtile) : nullptr;
+    int* counter = chained ? p.ctl + kChainHeaderInts + fwd_chain_index(p, it, qtile) * NDV + dvh : nullptr;
     const bool fold = chained && !it.first;
     if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
     if (ok)
-      fwd_store_row<DV>(tmem_o + lane_sel, n_tiles > 0, l, m_ref * p.scale, fold, o_dst, lse_dst, true,
-                        (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total : nullptr, row_ok, chained,
+      fwd_store_row<DV>(tmem_o + lane_sel, n_tiles > 0, l, m_ref * p.scale, fold, o_dst, lse_dst,
+                        dvh == 0 || chained,
+                        (it.last && p.o_bf16) ? p.o_bf16 + out_row * p.dv_total + dvh * DV : nullptr, row_ok, chained,
                         chained && (p.chain_mode == 2 ? it.last : it.link == p.fine - 1));
     if (chained) {
       const bool all_ok = bar_and(2, 128, ok);     // every row of the tile is written
@@ -919,13 +950,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   }
 }
 
+template <int DK, int NDV>
 static ls_status_t launch_fwd2(const FwdParams& prm, int64_t grid, cudaStream_t st) {
+  using C = Fwd2Cfg<DK>;
   static bool configured[64] = {};
+  grid *= NDV;
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  const ls_status_t cs = configure_smem(fwd2_kernel, Fwd2Cfg::SMEM_BYTES, configured);
+  const ls_status_t cs = configure_smem(fwd2_kernel<DK, NDV>, C::SMEM_BYTES, configured);
   if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_FWD, st);
-  fwd2_kernel<<<(int)grid, kFwdThreads, Fwd2Cfg::SMEM_BYTES, st>>>(prm);
+  fwd2_kernel<DK, NDV><<<(int)grid, kFwdThreads, C::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_FWD, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
@@ -981,12 +1015,20 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
   const int dvt = f.mla ? 256 : d.dim_v;                    // O channels per CTA
   const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
   const bool small_pages = d.page_size == 64;
-  const bool pair = d.dim_k == 256 && !f.packed;            // CTA pairs share every key tile between two Q tiles
+  const bool pair = (d.dim_k == 256 || f.mla) && !f.packed;  // CTA pairs share every key tile between two Q tiles
   if (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) k_resp = v_resp = q;   // the response maps are encoded but never used
   ls_status_t st = encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, f.rt.bt, f.rt.bh);
   if (pair) {
-    if (st == LS_OK) st = encode_map5(&P.rk2, k_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
-    if (st == LS_OK) st = encode_map5(&P.rv2, v_resp, 256, R, Hkv, 1, (int64_t)Hkv * 256, 256, (int64_t)R * Hkv * 256, 64, 2);
+    if (st == LS_OK)
+      st = encode_map5(&P.rk2, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k, (int64_t)R * Hkv * d.dim_k, 64, 2);
+    if (st == LS_OK)
+      st = encode_map5(&P.rv2, v_resp, d.dim_v, R, Hkv, 1, (int64_t)Hkv * d.dim_v, d.dim_v, (int64_t)R * Hkv * d.dim_v, 64, 2);
+    if (f.mla) {
+      if (st == LS_OK)
+        st = encode_map5(&P.rk1, k_resp, d.dim_k, R, Hkv, 1, (int64_t)Hkv * d.dim_k, d.dim_k, (int64_t)R * Hkv * d.dim_k, 64, 1);
+      if (st == LS_OK) st = pool_map(&P.pk1, h, 0, 64, 1, false);
+      if (st == LS_OK) st = pool_map(&P.pk1_tail, h, 0, 64, 1, true);
+    }
     if (st == LS_OK) st = pool_map(&P.pk2, h, 0, 64, 2, false);
     if (st == LS_OK) st = pool_map(&P.pk2_tail, h, 0, 64, 2, true);
     if (st == LS_OK) st = pool_map(&P.pv2, h, 1, 64, 2, false);
@@ -1046,7 +1088,10 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
     P.lse_aux = reinterpret_cast<float*>(static_cast<char*>(workspace) + cb);
     if (cudaMemsetAsync(workspace, 0, cb, cs) != cudaSuccess) return LS_ERR_CUDA;
   }
-  if (pair) return launch_fwd2(P, (int64_t)Hkv * (parts + 1) * ((f.nq_tiles + 1) / 2) * 2, cs);
+  if (pair) {
+    const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((f.nq_tiles + 1) / 2) * 2;
+    return f.mla ? launch_fwd2<576, 2>(P, grid2, cs) : launch_fwd2<256, 1>(P, grid2, cs);
+  }
   const int64_t grid = (int64_t)Hkv * (parts + 1) * f.nq_tiles;
   return f.mla ? launch_fwd<576, 256, 2>(P, grid, cs)
                : d.dim_k == 128 ? launch_fwd<128, 128, 1>(P, grid, cs) : launch_fwd<256, 256, 1>(P, grid, cs);

@@ -123,11 +123,17 @@ def test_workspace_sizes():
     assert B.ls_replay_attn_workspace_bytes(many, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == head + rows * 256 * 4
     # a tiny stream budget walks every shard as sub-ranges: the forward then needs its counters, nothing more
     cut = B.ls_prefix_pages_build(256 * 12, 256, 3, 2, 256, 256, 12, stream_budget_kib=512)
-    assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_FWD) == _ctl(2 * 3 * 4)
+    # (R = 96 < 128 with 4 heads per KV head: 3 Q tiles of 32 tokens x 4 heads per KV head, not 4 of one head)
+    assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_FWD) == _ctl(2 * 3 * 3)
     assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == head + rows * 256 * 4
     mla = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=True)
-    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + rows * 576 * 4
-    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_FWD_MERGED) == _ctl(Hq * 2) + rows * 4
+    # 16 row blocks of 64 are too few to fill the GPU: the 4 parts go to 4 CTA pairs per block, each with an
+    # fp32 sum of its own beside the response block's
+    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + (1 + 4) * rows * 576 * 4
+    assert B.ls_replay_attn_workspace_bytes(mla, 4096, 64, 1 / 24, B.LS_WORKSPACE_BWD) == \
+        4096 * 64 * 4 + _ctl(64 * 32) + 4096 * 64 * 576 * 4
+    # forward: 6 Q tiles of 16 tokens x 8 heads, two 256-channel halves of O each
+    assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_FWD_MERGED) == _ctl(6 * 2) + rows * 4
     sep = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=False)
     assert B.ls_replay_attn_workspace_bytes(sep, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + (4 + 1) * rows * 576 * 4
     empty = B.ls_prefix_pages_build(0, 64, 1, 1, 576, 512, 1, v_aliases_k=True)
