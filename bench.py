@@ -40,6 +40,25 @@ UNIT = "TFLOP/s"
 DQ_KERNEL_NAME = {(256, 256): "bwd_dq3_kernel", (128, 128): "bwd_dq2_kernel", (576, 512): "bwd_mla_dq_kernel"}
 
 
+def packed_tiles(cfg, tile_rows=128):
+    """True when the library packs rows of several heads of a KV group into one Q tile (a response
+    shorter than a tile, and fewer tiles that way): which kernels run depends on it."""
+    g = cfg.Hq // cfg.Hkv
+    if g <= 1 or cfg.R >= tile_rows:
+        return False
+    bh = min(g, tile_rows)
+    bt = min(cfg.R, tile_rows // bh)
+    return -(-cfg.R // bt) * -(-g // bh) < g
+
+
+def kernel_names(cfg):
+    """(forward kernel, query-gradient kernel) the library launches for this workload."""
+    packed = packed_tiles(cfg)
+    fwd = "fwd2_kernel" if (cfg.Dk in (256, 576) and not packed) else "fwd_kernel"
+    dq = "bwd_dq1_kernel" if (packed and cfg.Dk != 576) else DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv))
+    return fwd, dq
+
+
 def measured_traffic(kernel, workload):
     """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel` at `workload`, from the
     committed ncu capture records (a JSON list of {kernel, workload, dram_bytes_per_launch, ...});
@@ -324,19 +343,20 @@ def run_cuda(args):
     }
     if mode in ("replay", "fused"):
         dq_tflops = dq_f / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e12
-        kname = DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv))
+        kname = kernel_names(cfg)[1]
         out["roofline"] = {"bound": "tensor", "kernel": "%s (query-gradient pass over all parts)" % kname,
                            "achieved": dq_tflops, "peak": peak, "unit": UNIT, "frac": dq_tflops / peak,
                            "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
                            "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
                            "traffic": measured_traffic(kname, cfg.name),
                            "algorithmic_flops_per_launch": dq_f,
-                           "fwd_kernel": {"achieved": fwd_tflops, "frac": fwd_tflops / peak,
-                                          "ms_per_launch": k_ms[B.LS_KERNEL_FWD]},
+                           "fwd_kernel": {"kernel": kernel_names(cfg)[0], "achieved": fwd_tflops, "frac": fwd_tflops / peak,
+                                          "ms_per_launch": k_ms[B.LS_KERNEL_FWD],
+                                          "traffic": measured_traffic(kernel_names(cfg)[0], cfg.name)},
                            "whole_step_frac": value / world / peak,
                            "frac_of_nominal_2250": value / world / 2250.0}
     elif mode == "score":
-        kname = "fwd2_kernel" if cfg.Dk == 256 else "fwd_kernel"
+        kname = kernel_names(cfg)[0]
         out["roofline"] = {"bound": "tensor", "kernel": "%s (forward with the merge folded in)" % kname,
                            "achieved": fwd_tflops, "peak": peak, "unit": UNIT, "frac": fwd_tflops / peak,
                            "peak_source": "%s sustained bf16 cuBLAS (burst %.1f)" % (peaks["source"], peaks["bf16_tflops"]),
@@ -349,7 +369,7 @@ def run_cuda(args):
     if args.small_r and mode != "blocks":
         kv_bytes = pool_bytes
         fwd_gbs = kv_bytes / (k_ms[B.LS_KERNEL_FWD] * 1e-3) / 1e9
-        fname = "fwd_kernel" if cfg.Hq // cfg.Hkv * cfg.R <= 128 or cfg.Dk != 256 else "fwd2_kernel"
+        fname, dqname = kernel_names(cfg)
         out["roofline"] = {"bound": "hbm", "kernel": "%s (K and V pages streamed once per launch)" % fname,
                            "achieved": fwd_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": fwd_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
@@ -357,8 +377,9 @@ def run_cuda(args):
                            "algorithmic_bytes_per_launch": kv_bytes, "frac_of_nominal_8000": fwd_gbs / 8000.0}
         if B.LS_KERNEL_BWD_DQ in k_ms:
             dq_gbs = kv_bytes / (k_ms[B.LS_KERNEL_BWD_DQ] * 1e-3) / 1e9
-            out["roofline"]["dq_kernel"] = {"achieved": dq_gbs, "frac": dq_gbs / peaks["hbm_gbs"],
-                                            "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ]}
+            out["roofline"]["dq_kernel"] = {"kernel": dqname, "achieved": dq_gbs, "frac": dq_gbs / peaks["hbm_gbs"],
+                                            "ms_per_launch": k_ms[B.LS_KERNEL_BWD_DQ],
+                                            "traffic": measured_traffic(dqname, cfg.name)}
     if not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, seconds_target=15.0)
     print(json.dumps(out))

@@ -1,7 +1,7 @@
 """fp64 oracle for sparse (DSA) response replay over the shared latent.
 
-Test infrastructure only; shares no code with the CUDA library.  No kernel exists for this
-operator yet: the oracle and its pins come first.
+Test infrastructure only; shares no code with the CUDA library (whose sparse path the GPU
+tests compare against these functions).
 
 What is computed (Sec. "GLM Attention: MLA, DSA, and IndexShare", Eq. dsa-index,
 Eq. dsa-attention; Sec. "Predecessor CP-Local 2M Diagnostic", Eq. glm-global-dsa):

@@ -1698,7 +1698,9 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   float* delta = static_cast<float*>(workspace);
   const size_t delta_bytes = ((size_t)rows * sizeof(float) + 15) & ~(size_t)15;
   int* ctl = reinterpret_cast<int*>(static_cast<char*>(workspace) + delta_bytes);
-  const size_t ctl_bytes = ((size_t)(ls::kChainHeaderInts + (int64_t)Hkv * g * tiles_per_head) * sizeof(int) + 15) & ~(size_t)15;
+  int64_t chains = (int64_t)Hkv * g * tiles_per_head;
+  if (mla && ls::mla_dq_fast(h)) chains = std::max(chains, ls::mla_dq_blocks(h, R, Hq));
+  const size_t ctl_bytes = ((size_t)(ls::kChainHeaderInts + chains) * sizeof(int) + 15) & ~(size_t)15;
   float* dq_acc = reinterpret_cast<float*>(reinterpret_cast<char*>(ctl) + ctl_bytes);
   const int parts = h->num_parts();
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
@@ -1709,12 +1711,15 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     const bool mla_fast = ls::mla_dq_fast(h);
     if (no_resp) {       // prefix parts only: the transposed kernel walks them all and writes dQ
       if (!mla_fast) return LS_ERR_UNSUPPORTED_SHAPE;
-      return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, nullptr, dq_acc + rows * D, dq, status_dev, cs);
+      // (no response partial: the first fp32 region is the running dQ of a chained launch, the split
+      // partials follow it)
+      return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, nullptr,
+                            ls::mla_dq_split(h, R, Hq).chain ? dq_acc : dq_acc + rows * D, ctl, dq, status_dev, cs);
     }
     ls_status_t ms =
         ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_acc, dk_resp, dv_resp, mla_fast, status_dev, cs);
     if (ms != LS_OK) return ms;
-    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_acc, dq_acc + rows * D, dq, status_dev, cs);
+    if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_acc, dq_acc + rows * D, ctl, dq, status_dev, cs);
     const int64_t n4m = rows * D / 4;
     ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4m + 255) / 256, 148 * 16), 256, 0, cs>>>(
         dq_acc, parts + 1, n4m, prm->scale, static_cast<__nv_bfloat16*>(dq));

@@ -29,7 +29,8 @@
 // threads of the even CTA issue the two kinds of products, so that dQ^T of step i overlaps
 // [S^T | T^T] of step i + 1 while the key threads of both CTAs work between them; E^T and
 // [S^T | T^T] are double-buffered.  What bounds it at full size is the stream itself: every 64-row
-// block pulls 2.3 KB per key out of L2 (about 7.5 TB/s over the launch).
+// block pulls 2.3 KB per key out of L2, and beside the resident rows only seven ring slots (112 KB
+// of loads in flight per SM) fit in shared memory.
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -61,6 +62,14 @@ struct MlaDqParams {
   int nsplit;      // CTAs per row block, each walking a contiguous range of the parts; with more than one
                    // the fp32 sums go to dq_split [nsplit, R, Hq, 576] and a reduce kernel finishes
   float* dq_split;
+  // chain != 0 (many row blocks): the pairs of one range of parts run together (work items handed out by
+  // ticket, range-major) so that its keys stay in L2, and the ranges' sums of a row block meet in ONE
+  // running fp32 dQ, dq_acc [R, Hq, 576], in range order (ordered hand-over: ctl[0] ticket, ctl[1] abort,
+  // ctl[4 + row block] completed CTAs); acc_init: dq_acc already holds the response block's partial.
+  int chain, acc_init;
+  int* ctl;
+  float* dq_acc;
+  int num_kv_heads;
   int ablate;   // diagnostic builds only: 1 = no key loads, 2 = no tensor-core instructions
   float scale, scale_log2;
 };
@@ -112,6 +121,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
   uint64_t* acc_final = e_free + 2;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* work_idx = const_cast<int*>(abort_flag) + 1;   // (even CTA) the pair's work item
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -119,12 +129,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
   long long tw0 = 0, tw1 = 0, tw2 = 0, tw3 = 0;   // wait-time accumulators (only used with LS_TIMING)
   const long long t_begin = clock64();
   (void)tw0; (void)tw1; (void)tw2; (void)tw3; (void)t_begin;
-  // work item of the pair: row block (fastest, so that the pairs in flight share the same keys),
-  // range of parts, KV head
-  const int work = (int)(blockIdx.x >> 1);
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    // chained: work items in launch order of the pairs that ask, so that a link only waits for links some pair has started
+    if (leader) *work_idx = p.chain ? atomicAdd(p.ctl, 1) : (int)(blockIdx.x >> 1);
+  }
+  cluster_sync_all();
+  // work item of the pair: row block (fastest, so that the pairs in flight share the same keys), then
+  // KV head and range of parts (chained: range slowest)
+  const int work = (int)ld_shared_cluster_u32(mapa_u32(smem_u32(work_idx), 0));
   const int qtile = work % p.nq_tiles;
-  const int split = (work / p.nq_tiles) % p.nsplit;
-  const int kvh = work / (p.nq_tiles * p.nsplit);
+  const int split = p.chain ? work / (p.nq_tiles * p.num_kv_heads) : (work / p.nq_tiles) % p.nsplit;
+  const int kvh = p.chain ? (work / p.nq_tiles) % p.num_kv_heads : work / (p.nq_tiles * p.nsplit);
   const int h = kvh * p.g + (qtile / p.tiles_tok) * p.bh;     // first head and token of the block
   const int row0 = (qtile % p.tiles_tok) * p.bt;
   // the parts this pair walks: all of them, or (several pairs per row block) a contiguous range
@@ -154,7 +170,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
       mbar_init(&e_free[i], 1);
     }
     mbar_init(acc_final, 1);
-    *abort_flag = 0;
     fence_barrier_init();
   }
   if (threadIdx.x >= 64 && threadIdx.x < 64 + kTqRows) {
@@ -380,6 +395,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
     const uint32_t sw = (uint32_t)(key & 7) >> 1;
     const uint32_t s_read_remote[2] = {mapa_u32(smem_u32(&s_read[0]), 0), mapa_u32(smem_u32(&s_read[1]), 0)};
     const uint32_t e_full_remote[2] = {mapa_u32(smem_u32(&e_full[0]), 0), mapa_u32(smem_u32(&e_full[1]), 0)};
+    bool key_ok = true;
     if (total_steps > 0) {
       bool ok = true;
       int part = part_lo, step = -1;
@@ -443,47 +459,62 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
       }
       if (ok) ok = mbar_wait(acc_final, 0, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
-        tc_fence_after();
+      if (ok) tc_fence_after();
+      key_ok = ok;
+    }
+    // ---- epilogue: this CTA's channels of the 64 rows.  Alone (one range of parts): scale, add the response
+    // block's partial, write bf16.  Split: the fp32 sum goes to the range's scratch partial.  Chained: it is
+    // added to the running dQ once the previous range's pair has published, and the last range writes bf16.
+    const bool have_acc = total_steps > 0;
+    const bool last = p.chain && split == p.nsplit - 1;
+    const bool fold = p.chain && (split > 0 || p.acc_init);
+    int* counter = p.chain ? p.ctl + kChainHeaderInts + kvh * p.nq_tiles + qtile : nullptr;
+    if (key_ok && p.chain && split > 0)
+      key_ok = __all_sync(0xffffffffu, chain_wait(counter, 2 * split, p.ctl, abort_flag));
+    if (key_ok && (have_acc || p.nsplit > 1)) {
+      const uint64_t pol = l2_policy_evict_first();     // the running dQ passes through L2 once per range
 #pragma unroll 1
-        for (int m = 0; m < 3; ++m) {
-          if (m == 2 && (!leader || quad >= 2)) break;      // block 2 is the 64 rope channels, in the even CTA
-          const int ch = m * 256 + (int)rank * 128 + key;
+      for (int m = 0; m < 3; ++m) {
+        if (m == 2 && (!leader || quad >= 2)) break;      // block 2 is the 64 rope channels, in the even CTA
+        const int ch = m * 256 + (int)rank * 128 + key;
 #pragma unroll 1
-          for (int half = 0; half < 2; ++half) {
-            uint32_t o[32];
+        for (int half = 0; half < 2; ++half) {
+          uint32_t o[32];
+          if (have_acc) {
             tmem_ld32(tmem_acc + lane_sel + m * 64 + half * 32, o);
             tc_wait_ld32(o);
-            int hj = (half * 32) / p.bt, tk = half * 32 - hj * p.bt;   // head and token of row half * 32 + j
+          } else {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int r = row0 + tk, hh = h + hj;
-              if (++tk == p.bt) {
-                tk = 0;
-                ++hj;
-              }
-              if (hh - h < p.bh && r < p.R && hh < (kvh + 1) * p.g) {
-                const size_t idx = ((size_t)r * p.Hq + hh) * 576 + ch;
-                if (p.nsplit > 1)
-                  p.dq_split[(size_t)split * p.R * p.Hq * 576 + idx] = __uint_as_float(o[j]);
-                else
-                  p.dq[idx] = __float2bfloat16_rn((__uint_as_float(o[j]) + (p.dq_resp ? p.dq_resp[idx] : 0.f)) * p.scale);
+            for (int j = 0; j < 32; ++j) o[j] = 0u;
+          }
+          int hj = (half * 32) / p.bt, tk = half * 32 - hj * p.bt;   // head and token of row half * 32 + j
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int r = row0 + tk, hh = h + hj;
+            if (++tk == p.bt) {
+              tk = 0;
+              ++hj;
+            }
+            if (hh - h < p.bh && r < p.R && hh < (kvh + 1) * p.g) {
+              const size_t idx = ((size_t)r * p.Hq + hh) * 576 + ch;
+              float v = __uint_as_float(o[j]);
+              if (p.chain) {
+                if (fold) v += ld_cg_hint_f32(p.dq_acc + idx, pol);
+                if (last) p.dq[idx] = __float2bfloat16_rn(v * p.scale);
+                else st_hint_f32(p.dq_acc + idx, v, pol);
+              } else if (p.nsplit > 1) {
+                p.dq_split[(size_t)split * p.R * p.Hq * 576 + idx] = v;
+              } else {
+                p.dq[idx] = __float2bfloat16_rn((v + (p.dq_resp ? p.dq_resp[idx] : 0.f)) * p.scale);
               }
             }
           }
         }
       }
-    } else if (p.nsplit > 1) {
-      // an empty range of parts still owes its (zero) partial to the reduce kernel
-      for (int m = 0; m < 3; ++m) {
-        if (m == 2 && (!leader || quad >= 2)) break;
-        const int ch = m * 256 + (int)rank * 128 + key;
-        for (int rr = 0; rr < p.bt * p.bh; ++rr) {
-          const int r = row0 + rr % p.bt, hh = h + rr / p.bt;
-          if (r < p.R && hh < (kvh + 1) * p.g)
-            p.dq_split[(size_t)split * p.R * p.Hq * 576 + ((size_t)r * p.Hq + hh) * 576 + ch] = 0.f;
-        }
-      }
+    }
+    if (p.chain) {
+      const bool all_ok = bar_and(1, 128, key_ok);      // every row of this CTA's channels is written
+      if (key == 0 && all_ok) chain_publish_add(counter);
     }
   }
 
@@ -494,7 +525,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
     tc_fence_after();
     tmem_dealloc_pair(tmem_base, 512);
   }
-  if (threadIdx.x == 0 && *abort_flag && p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+  if (threadIdx.x == 0 && *abort_flag) {
+    if (p.status) atomicExch(p.status, (int)LS_ERR_TIMEOUT);
+    if (p.chain) st_relaxed_gpu(p.ctl + 1, 1);    // ends every other chain wait of this launch
+  }
 }
 
 bool mla_dq_fast(const ls_pages* h) {
@@ -502,12 +536,27 @@ bool mla_dq_fast(const ls_pages* h) {
   return d.dim_k == 576 && d.dim_v == 512 && d.v_aliases_k && d.prefix_len > 0;
 }
 
-int mla_dq_splits(const ls_pages* h, int R, int Hq) {
+int64_t mla_dq_blocks(const ls_pages* h, int R, int Hq) {
+  const int Hkv = h->desc.num_kv_heads;
+  return (int64_t)Hkv * row_tiling(R, Hq / Hkv, kTqRows).nq_tiles;
+}
+
+MlaDqSplit mla_dq_split(const ls_pages* h, int R, int Hq) {
   const int Hkv = h->desc.num_kv_heads;
   const int64_t blocks = (int64_t)Hkv * row_tiling(R, Hq / Hkv, kTqRows).nq_tiles;
-  if (blocks >= 74) return 1;                  // enough row blocks for every CTA pair: each walks all parts
-  // few rows: the parts are spread over enough CTA pairs to fill the GPU twice
-  return std::max(1, std::min(h->prefix_parts(), (int)((148 + blocks - 1) / blocks)));
+  const int parts = h->prefix_parts();
+  MlaDqSplit sp;
+  if (blocks >= 74) {
+    // a row block for every CTA pair of the GPU and more: one range per part, the pairs of a range run together
+    // (its keys, at most the stream budget, stay in L2 while every row block passes over them)
+    sp.count = parts;
+    sp.chain = parts > 1;
+  } else {
+    // few rows: the parts are spread over enough CTA pairs to fill the GPU twice, all running at once
+    sp.count = std::max(1, std::min(parts, (int)((148 + blocks - 1) / blocks)));
+    sp.chain = false;
+  }
+  return sp;
 }
 
 // dq = scale * (sum of the split partials + the response block's partial), bf16
@@ -529,7 +578,7 @@ __global__ void mla_dq_split_reduce_kernel(const float* __restrict__ part, int n
 // dQ (bf16, final) of the 576/512 shape with V aliasing K: prefix part in this kernel, plus
 // dq_resp, the response block's unscaled fp32 part computed beforehand.
 ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
-                       const float* lse, const float* delta, const float* dq_resp, float* dq_split, void* dq,
+                       const float* lse, const float* delta, float* dq_resp, float* scratch, int* ctl, void* dq,
                        int32_t* status_dev, cudaStream_t cs) {
   const ls_pages_desc_t& d = h->desc;
   const int R = prm->R, Hq = prm->num_q_heads;
@@ -560,8 +609,19 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   P.tiles_tok = rt.tiles_tok;
   P.nq_tiles = rt.nq_tiles;
   P.qdo_bytes = (9 + 9) * rt.bt * rt.bh * 128;      // Q (even CTA), dO and the rope slab of Q (odd CTA)
-  P.nsplit = dq_split ? mla_dq_splits(h, R, Hq) : 1;     // without scratch every CTA walks all parts
-  P.dq_split = dq_split;
+  MlaDqSplit sp = mla_dq_split(h, R, Hq);
+  if (!scratch || !ctl) sp = MlaDqSplit{1, false};         // without scratch every pair walks all parts
+  P.nsplit = sp.count;
+  P.dq_split = scratch;
+  P.chain = sp.chain ? 1 : 0;
+  P.ctl = ctl;
+  P.num_kv_heads = d.num_kv_heads;
+  // chained: the running dQ starts as the response block's partial where there is one
+  P.acc_init = dq_resp ? 1 : 0;
+  P.dq_acc = dq_resp ? dq_resp : scratch;
+  if (P.chain &&
+      cudaMemsetAsync(ctl, 0, (kChainHeaderInts + (size_t)d.num_kv_heads * rt.nq_tiles) * sizeof(int), cs) != cudaSuccess)
+    return LS_ERR_CUDA;
   ls_status_t st = encode_map_rows(&P.q_map, q, 576, R, Hq, rt.bt, rt.bh);
   if (st == LS_OK) st = encode_map_rows(&P.do_map, d_o, 512, R, Hq, rt.bt, rt.bh);
   if (st == LS_OK) st = pool_map(&P.k_map, h, 0, 64, 1, false);
@@ -576,10 +636,10 @@ ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const voi
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
   profile_begin(LS_KERNEL_BWD_DQ, cs);
   bwd_mla_dq_kernel<<<(int)grid, kTqThreads, kTqSmem, cs>>>(P);
-  if (P.nsplit > 1) {
+  if (P.nsplit > 1 && !P.chain) {
     const int64_t n4 = (int64_t)R * Hq * 576 / 4;
     mla_dq_split_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 8), 256, 0, cs>>>(
-        dq_split, P.nsplit, dq_resp, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
+        scratch, P.nsplit, dq_resp, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
   }
   profile_end(LS_KERNEL_BWD_DQ, cs);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;

@@ -554,5 +554,5 @@ extern "C" ls_status_t ls_dsa_attn_bwd(const ls_dsa_plan_t* p, float scale, cons
   pg.R = 1;
   pg.num_q_heads = (int32_t)rows;
   pg.scale = scale;
-  return ls::bwd_mla_dq(p->gathered, &pg, q, d_o, lse, delta, dq_resp, nullptr, dq, status_dev, cs);
+  return ls::bwd_mla_dq(p->gathered, &pg, q, d_o, lse, delta, dq_resp, nullptr, nullptr, dq, status_dev, cs);
 }

@@ -1127,13 +1127,20 @@ extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_a
     return ls::ctl_bytes((int64_t)f.Hkv * f.nq_tiles * f.ndv) + (f.mla ? rows * sizeof(float) : 0);
   if (which != LS_WORKSPACE_BWD) return 0;
   // backward: Delta (fp32) + hand-over counters + the fp32 dQ that the partials are summed into
-  const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes((int64_t)f.Hkv * f.g * ((f.R + 127) / 128));
-  if (f.mla && !ls::mla_dq_fast(h))     // 576/512 with a separate V pool: one fp32 dQ per partial
+  const bool mla_fast = f.mla && ls::mla_dq_fast(h);
+  int64_t chains = (int64_t)f.Hkv * f.g * ((f.R + 127) / 128);
+  if (mla_fast) chains = std::max(chains, ls::mla_dq_blocks(h, f.R, f.Hq));     // its row blocks are 64 rows
+  const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes(chains);
+  if (f.mla && !mla_fast)     // 576/512 with a separate V pool: one fp32 dQ per partial
     return head + (size_t)(h->num_parts() + 1) * rows * d.dim_k * sizeof(float);
-  // (short responses of the aliased 576/512 shape spread the parts of a KV group over several CTAs,
+  // (short responses of the aliased 576/512 shape spread the parts over several CTA pairs per row block,
   // each with an fp32 sum of its own)
-  const size_t splits = (f.mla && ls::mla_dq_fast(h)) ? (size_t)ls::mla_dq_splits(h, f.R, f.Hq) : 1;
-  return head + (1 + (splits > 1 ? splits : 0)) * rows * d.dim_k * sizeof(float);
+  size_t partials = 0;
+  if (mla_fast) {
+    const ls::MlaDqSplit sp = ls::mla_dq_split(h, f.R, f.Hq);
+    if (sp.count > 1 && !sp.chain) partials = (size_t)sp.count;
+  }
+  return head + (1 + partials) * rows * d.dim_k * sizeof(float);
 }
 
 extern "C" ls_status_t ls_replay_attn_fwd(const ls_pages_t* h, const ls_attn_params_t* prm, const void* q,

@@ -148,15 +148,26 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
                     void* dk_resp, void* dv_resp, bool dq_resp_only, int32_t* status_dev, cudaStream_t cs);
 
-// Prefix part of dQ for the 576/512 shape when V aliases K (ls_bwd_mla_dq.cu): every CTA walks
-// all partials, adds dq_resp (fp32, unscaled, [R, Hq, 576]) and writes the final bf16 dQ.
-// dq_split: fp32 scratch of mla_dq_splits() * R * Hq * 576 floats that lets a launch with few row blocks
-// spread the parts over several CTAs per block (NULL: every CTA walks all parts).
+// Prefix part of dQ for the 576/512 shape when V aliases K (ls_bwd_mla_dq.cu): CTA pairs walk the
+// prefix parts, add dq_resp (fp32, unscaled, [R, Hq, 576]; NULL: none) and write the final bf16 dQ.
+// How the parts are spread is mla_dq_split(): with more than one range per row block the sums meet
+// either in `scratch` (count partials of R * Hq * 576 floats, then a reduce kernel) or, chained, in
+// ONE running fp32 dQ -- dq_resp itself, or the first R * Hq * 576 floats of scratch when there is
+// no response partial -- through the control words `ctl` (kChainHeaderInts + one per 64-row block).
+// Without scratch or ctl every pair walks all parts.
 ls_status_t bwd_mla_dq(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* d_o,
-                       const float* lse, const float* delta, const float* dq_resp, float* dq_split, void* dq,
+                       const float* lse, const float* delta, float* dq_resp, float* scratch, int* ctl, void* dq,
                        int32_t* status_dev, cudaStream_t cs);
-// CTAs per row block of bwd_mla_dq when the launch has fewer row blocks than SMs; 1 otherwise.
-int mla_dq_splits(const ls_pages* h, int R, int Hq);
+// count: ranges of parts per row block; chain: many row blocks -- the pairs of one range run together
+// (its keys stay in L2) and the ranges fold into one running dQ in order; otherwise (few row blocks) all
+// pairs run at once, each with a scratch partial.
+struct MlaDqSplit {
+  int count;
+  bool chain;
+};
+MlaDqSplit mla_dq_split(const ls_pages* h, int R, int Hq);
+// 64-row blocks of bwd_mla_dq for this call (one hand-over counter each).
+int64_t mla_dq_blocks(const ls_pages* h, int R, int Hq);
 // True when bwd_mla_dq serves this handle (576/512, V aliasing K, non-empty prefix).
 bool mla_dq_fast(const ls_pages* h);
 

@@ -172,10 +172,25 @@ __device__ __forceinline__ void st_hint(float4* ptr, float4 v, uint64_t pol) {
                "f"(v.w), "l"(pol)
                : "memory");
 }
+__device__ __forceinline__ float ld_cg_hint_f32(const float* ptr, uint64_t pol) {
+  float v;
+  asm volatile("ld.global.cg.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(ptr), "l"(pol) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_hint_f32(float* ptr, float v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(ptr), "f"(v), "l"(pol) : "memory");
+}
 // Called by ONE thread after a CTA-level barrier that all writers of the running value passed.
 __device__ __forceinline__ void chain_publish(int* counter, int value) {
   __threadfence();
   st_release_gpu(counter, value);
+}
+
+// The same for a link that several CTAs complete together (each adds one after its own barrier);
+// the successor waits for the sum.
+__device__ __forceinline__ void chain_publish_add(int* counter) {
+  __threadfence();
+  asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(counter) : "memory");
 }
 
 // ------------------------------------------------------------------ TMA
