@@ -11,9 +11,10 @@
 //      indexer-key pages through a ring; D = kI qI^T lands in TMEM (128 keys x 256 columns, two
 //      buffers), and one thread per key folds its row: relu, weight, sum over the H_I heads of a
 //      token -- a reduction along the thread's own registers, written coalesced along the keys.
-//   2. top-k: one CTA per query row, 8-bit radix select on order-preserving keys (4 passes), then an
-//      ordered pass that emits the selected positions in ascending order and breaks ties at the
-//      threshold by position.  Integer work: bit-exact against the rule, whatever the scheduling.
+//   2. top-k: one CTA per query row, radix select on order-preserving keys (digits of 11, 11 and 10
+//      bits: three passes over the row, 16-byte loads), then an ordered pass that emits the selected
+//      positions in ascending order and breaks ties at the threshold by position.  Integer work:
+//      bit-exact against the rule, whatever the scheduling.
 //   3. gather: the selected latent rows are copied into a pool whose "KV head" index is the query
 //      token: [k / 64 pages, 64, R, 576].  On that pool the dense kernels of this library compute
 //      exactly the sparse operator: KV head t = token t's selected keys, its H heads = the query
@@ -246,67 +247,162 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 constexpr int kTopkThreads = 1024;
+constexpr int kTopkBins = 2048;            // radix digits of 11, 11 and 10 bits
 
-__global__ void __launch_bounds__(kTopkThreads) dsa_topk_kernel(const float* __restrict__ scores, long long P, int k,
-                                                                int32_t* __restrict__ sel) {
-  const float* s = scores + (long long)blockIdx.x * P;
-  const int count = (int)min((long long)k, P);
-  int32_t* out = sel + (long long)blockIdx.x * count;
+// Warp 0: the digit d with  #(digit > d) < need <= #(digit >= d)  in the histogram, and #(digit > d).
+// Each lane sums 64 bins, the lanes scan from the top; the lane that holds d writes the results.
+__device__ __forceinline__ void topk_find_digit(const uint32_t* hist, uint32_t need, int lane, uint32_t* d_out,
+                                                uint32_t* above_out) {
+  constexpr int kPer = kTopkBins / 32;
+  uint32_t mine = 0;
+  for (int b = 0; b < kPer; ++b) mine += hist[lane * kPer + b];
+  uint32_t above = 0;                                     // bins of higher lanes
+  for (int l = 31; l > 0; --l) {
+    const uint32_t v = __shfl_sync(0xffffffffu, mine, l);
+    if (lane < l) above += v;
+  }
+  if (above < need && above + mine >= need) {             // exactly one lane
+    uint32_t cum = above;
+    int d = lane * kPer + kPer - 1;
+    for (; d > lane * kPer; --d) {
+      if (cum + hist[d] >= need) break;
+      cum += hist[d];
+    }
+    *d_out = (uint32_t)d;
+    *above_out = cum;
+  }
+}
+
+// One histogram sweep over positions [begin, end) of a row: scores whose key, shifted down to the
+// current digit, lies in [lo_full, lo_full + span] are counted under their digit.  The body runs on
+// 16-byte loads (the row's first `peel` positions bring it to a 16-byte boundary), four in flight per thread.
+__device__ __forceinline__ void topk_count(const float* __restrict__ s, int begin, int end, int peel, bool vec,
+                                           int shift, uint32_t dmask, uint32_t lo_full, uint32_t span,
+                                           uint32_t* hist, int tid) {
+  auto count = [&](float f) {
+    const uint32_t kh = order_key(f) >> shift;
+    if (kh - lo_full <= span) atomicAdd(&hist[kh & dmask], 1u);
+  };
+  int body0 = begin, body1 = begin;                       // [body0, body1): whole aligned float4 groups
+  if (vec) {
+    body0 = begin <= peel ? peel : peel + ((begin - peel + 3) & ~3);
+    body1 = body0 + (end > body0 ? ((end - body0) & ~3) : 0);
+    if (body0 > end) body0 = body1 = end;
+  }
+  for (int i = begin + tid; i < body0; i += kTopkThreads) count(__ldg(s + i));
+  const float4* s4 = reinterpret_cast<const float4*>(s + body0);
+  const int n4 = (body1 - body0) >> 2;
+  int i = tid;
+  for (; i + 3 * kTopkThreads < n4; i += 4 * kTopkThreads) {
+    const float4 a = __ldg(s4 + i), b = __ldg(s4 + i + kTopkThreads), c = __ldg(s4 + i + 2 * kTopkThreads),
+                 d = __ldg(s4 + i + 3 * kTopkThreads);
+    count(a.x); count(a.y); count(a.z); count(a.w);
+    count(b.x); count(b.y); count(b.z); count(b.w);
+    count(c.x); count(c.y); count(c.z); count(c.w);
+    count(d.x); count(d.y); count(d.z); count(d.w);
+  }
+  for (; i < n4; i += kTopkThreads) {
+    const float4 a = __ldg(s4 + i);
+    count(a.x); count(a.y); count(a.z); count(a.w);
+  }
+  for (int j = body1 + tid; j < end; j += kTopkThreads) count(__ldg(s + j));
+}
+
+__global__ void __launch_bounds__(kTopkThreads, 2) dsa_topk_kernel(const float* __restrict__ scores, long long P64, int k,
+                                                                   int32_t* __restrict__ sel) {
+  const float* s = scores + (long long)blockIdx.x * P64;
+  const int P = (int)P64;                                   // positions are int32
+  const int count_sel = min(k, P);
+  int32_t* out = sel + (long long)blockIdx.x * count_sel;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   if (P <= k) {
-    for (long long i = tid; i < P; i += kTopkThreads) out[i] = (int32_t)i;
+    for (int i = tid; i < P; i += kTopkThreads) out[i] = i;
     return;
   }
-  __shared__ uint32_t hist[256];
-  __shared__ uint32_t sh_prefix, sh_need;
+  __shared__ uint32_t hist[kTopkBins];
+  __shared__ uint32_t sh_digit, sh_above;
   __shared__ uint32_t warp_gt[32], warp_eq[32];
   __shared__ uint32_t base_gt, base_eq;
+  // 16-byte loads need the scores buffer on a 16-byte boundary; a row then starts 0..3 floats past one
+  const bool vec = (reinterpret_cast<uintptr_t>(scores) & 15) == 0;
+  const int peel = vec ? (int)((4 - (((long long)blockIdx.x * P64) & 3)) & 3) : 0;
   // ---- radix select: the key of the k-th largest score, and how many scores equal to it to take
-  uint32_t prefix = 0, mask = 0, need = (uint32_t)k;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
-    if (tid < 256) hist[tid] = 0;
+  uint32_t prefix = 0, need = (uint32_t)k;
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : pass == 1 ? 10 : 0;
+    const uint32_t dmask = pass == 2 ? 1023u : 2047u;
+    for (int b = tid; b < kTopkBins; b += kTopkThreads) hist[b] = 0;
     __syncthreads();
-    for (long long i = tid; i < P; i += kTopkThreads) {
-      const uint32_t key = order_key(s[i]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    // Pass 0 would send every score of the row through a shared-memory atomic.  Its first 64K positions
+    // alone already hold `need` scores whose digit is at least some d0, so no score with a smaller digit
+    // can be selected: once d0 is known the rest of the row only counts digits >= d0 (a few per cent).
+    uint32_t lo = 0;
+    const int head = (pass == 0 && P > 8 * 65536 && need <= 16384) ? 65536 : 0;
+    if (head) {
+      topk_count(s, 0, head, peel, vec, shift, dmask, 0u, dmask, hist, tid);
+      __syncthreads();
+      if (wid == 0) topk_find_digit(hist, need, lane, &sh_digit, &sh_above);
+      __syncthreads();
+      lo = sh_digit;
+      __syncthreads();
     }
+    topk_count(s, head, P, peel, vec, shift, dmask, (prefix >> shift) + lo, dmask - lo, hist, tid);
     __syncthreads();
-    if (tid == 0) {
-      uint32_t cum = 0;
-      int d = 255;
-      for (; d > 0; --d) {
-        if (cum + hist[d] >= need) break;
-        cum += hist[d];
-      }
-      sh_prefix = prefix | ((uint32_t)d << shift);
-      sh_need = need - cum;
-    }
+    if (wid == 0) topk_find_digit(hist, need, lane, &sh_digit, &sh_above);
     __syncthreads();
-    prefix = sh_prefix;
-    need = sh_need;
-    mask |= 255u << shift;
+    prefix |= sh_digit << shift;
+    need -= sh_above;
+    __syncthreads();
   }
-  // ---- ordered pass: positions in ascending order; among scores equal to the threshold the
-  // lower positions are taken
+  // ---- ordered pass: positions in ascending order; among scores equal to the threshold the lower
+  // positions are taken.  A thread owns 16 consecutive positions of a 16384-position tile; it first
+  // counts (greater, equal), and only a thread that owns a selected position reads its scores again.
   const uint32_t thr = prefix;
   if (tid == 0) { base_gt = 0; base_eq = 0; }
   __syncthreads();
-  for (long long start = 0; start < P; start += kTopkThreads) {
-    const long long i = start + tid;
-    uint32_t key = 0;
-    const bool in = i < P;
-    if (in) key = order_key(s[i]);
-    const bool gt = in && key > thr, eq = in && key == thr;
-    const uint32_t m_gt = __ballot_sync(0xffffffffu, gt), m_eq = __ballot_sync(0xffffffffu, eq);
-    const uint32_t lt = (1u << lane) - 1u;
-    if (lane == 0) { warp_gt[wid] = __popc(m_gt); warp_eq[wid] = __popc(m_eq); }
+  for (int start = 0; start < P; start += 16 * kTopkThreads) {
+    const int i0 = start + 16 * tid;
+    uint32_t n_gt = 0, n_eq = 0;
+    if (i0 < P) {
+      if (vec && i0 >= peel && ((i0 - peel) & 3) == 0 && i0 + 16 <= P) {
+        const float4* s4 = reinterpret_cast<const float4*>(s + i0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float4 v = __ldg(s4 + j);
+          const uint32_t k0 = order_key(v.x), k1 = order_key(v.y), k2 = order_key(v.z), k3 = order_key(v.w);
+          n_gt += (k0 > thr) + (k1 > thr) + (k2 > thr) + (k3 > thr);
+          n_eq += (k0 == thr) + (k1 == thr) + (k2 == thr) + (k3 == thr);
+        }
+      } else {
+        for (int e = 0; e < 16 && i0 + e < P; ++e) {
+          const uint32_t key = order_key(__ldg(s + i0 + e));
+          n_gt += key > thr;
+          n_eq += key == thr;
+        }
+      }
+    }
+    uint32_t ex_gt = n_gt, ex_eq = n_eq;                     // inclusive prefix over the lanes
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t a = __shfl_up_sync(0xffffffffu, ex_gt, o), b = __shfl_up_sync(0xffffffffu, ex_eq, o);
+      if (lane >= o) { ex_gt += a; ex_eq += b; }
+    }
+    if (lane == 31) { warp_gt[wid] = ex_gt; warp_eq[wid] = ex_eq; }
+    ex_gt -= n_gt;
+    ex_eq -= n_eq;
     __syncthreads();
-    uint32_t ex_gt = __popc(m_gt & lt), ex_eq = __popc(m_eq & lt);
-    for (int w = 0; w < wid; ++w) { ex_gt += warp_gt[w]; ex_eq += warp_eq[w]; }
     const uint32_t bg = base_gt, be = base_eq;
-    const uint32_t eq_before = be + ex_eq;
-    if (gt || (eq && eq_before < need)) out[bg + ex_gt + min(eq_before, need)] = (int32_t)i;
+    if (n_gt | n_eq) {
+      for (int w = 0; w < wid; ++w) { ex_gt += warp_gt[w]; ex_eq += warp_eq[w]; }
+      uint32_t g_before = bg + ex_gt, e_before = be + ex_eq;
+      for (int e = 0; e < 16 && i0 + e < P; ++e) {
+        const uint32_t key = order_key(__ldg(s + i0 + e));
+        const bool gt = key > thr, eq = key == thr;
+        if (gt || (eq && e_before < need)) out[g_before + min(e_before, need)] = i0 + e;
+        g_before += gt;
+        e_before += eq;
+      }
+    }
     __syncthreads();
     if (tid == 0) {
       uint32_t tg = 0, te = 0;

@@ -86,6 +86,27 @@ def test_topk_is_bit_exact_including_ties():
     assert sel.shape == (5, 100) and (sel == np.arange(100)[None, :]).all()
 
 
+@pytest.mark.parametrize("P", [64 * 9400, 64 * 9400 + 37])          # rows of 16-byte aligned and unaligned length
+def test_topk_over_a_long_row(P):
+    # long rows take the selection's shortcut (a lower bound on the threshold from the row's first 64K
+    # positions); rows are built so that the bound is tight, loose, or sits in a crowd of equal scores
+    cfg = latent("topk_long", P=P, R=7, Hq=2, num_shards=2)
+    dc = DsaCase(cfg, 8, 2048)
+    g = torch.Generator(device="cuda").manual_seed(77)
+    s = torch.randn(cfg.R, P, device="cuda", generator=g)
+    s[1] = torch.round(s[1] * 2.0) / 2.0                                  # few distinct values: ties everywhere
+    s[2] = 0.25                                                           # all equal: the first 2048 positions
+    s[3, :65536] -= 100.0                                                 # head far below the rest: loose bound
+    s[4, :65536] += 100.0                                                 # every selected score sits in the head
+    s[5] = torch.where(torch.rand(P, device="cuda", generator=g) < 0.5, s[5], -s[5].abs() * 1e-30)
+    s[6, 70000:70000 + 3000] = float("inf")                               # more infinities than top_k
+    sel = B.ls_dsa_topk(dc.plan, s).cpu().numpy()
+    torch.cuda.synchronize()
+    host = s.double().cpu().numpy()
+    for t in range(cfg.R):
+        assert np.array_equal(sel[t], dsa.topk_select(host[t], 2048)), t
+
+
 def run_sparse(dc):
     cfg = dc.cfg
     sel = B.ls_dsa_topk(dc.plan, dc.scores())
