@@ -1701,7 +1701,10 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   int64_t chains = (int64_t)Hkv * g * tiles_per_head;
   if (mla && ls::mla_dq_fast(h)) chains = std::max(chains, ls::mla_dq_blocks(h, R, Hq));
   const size_t ctl_bytes = ((size_t)(ls::kChainHeaderInts + chains) * sizeof(int) + 15) & ~(size_t)15;
-  float* dq_acc = reinterpret_cast<float*>(reinterpret_cast<char*>(ctl) + ctl_bytes);
+  float* kv_scratch = reinterpret_cast<float*>(reinterpret_cast<char*>(ctl) + ctl_bytes);   // 576/512 only
+  const int kv_hsplit = mla ? ls::mla_kv_hsplit(h, R, Hq) : 1;
+  float* dq_acc = kv_scratch + (kv_hsplit > 1 ? (size_t)kv_hsplit * R * Hkv * D : 0);
+  if (kv_hsplit == 1) kv_scratch = nullptr;
   const int parts = h->num_parts();
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
@@ -1717,7 +1720,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
                             ls::mla_dq_split(h, R, Hq).chain ? dq_acc : dq_acc + rows * D, ctl, dq, status_dev, cs);
     }
     ls_status_t ms =
-        ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_acc, dk_resp, dv_resp, mla_fast, status_dev, cs);
+        ls::bwd_mla(h, prm, q, k_resp, v_resp, lse, delta, d_o, dq_acc, dk_resp, dv_resp, mla_fast, kv_scratch, status_dev, cs);
     if (ms != LS_OK) return ms;
     if (mla_fast) return ls::bwd_mla_dq(h, prm, q, d_o, lse, delta, dq_acc, dq_acc + rows * D, ctl, dq, status_dev, cs);
     const int64_t n4m = rows * D / 4;

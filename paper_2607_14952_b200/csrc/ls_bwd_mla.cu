@@ -44,6 +44,11 @@ struct MlaBwdParams {
   int32_t* status;
   int R, Hq, Hkv, g, S, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;   // tiles of 64 rows
   int part_first, part_count;   // mode DQ: partials [part_first, part_first + part_count) are computed
+  // modes DK / DV: the heads of a KV group are cut into hsplit ranges, one CTA each per key tile and
+  // pass (a short response has too few key tiles to fill the GPU); with more than one the fp32 sums
+  // go to kv_part [hsplit, R, Hkv, 576 | 512] and a reduce kernel writes `out`
+  int hsplit;
+  float* kv_part;
   float scale, scale_log2;
 };
 
@@ -82,7 +87,7 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
   int idx = blockIdx.x;
   const int pass = idx % NPASS;
   idx /= NPASS;
-  int part = 0, kvh, h = 0, row0;
+  int part = 0, kvh, h = 0, row0, hs = 0, h_lo = 0;
   bool is_resp = true;
   int64_t tokens = 0;
   int page_off = 0, n_pages = 0, tail_slot = -1, n_tiles, tt_min = 0, n_tt = 0;
@@ -104,11 +109,14 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
     }
     n_tiles = (int)((tokens + 63) / 64);
   } else {
+    hs = idx % p.hsplit;
+    idx /= p.hsplit;
     kvh = idx / p.tiles_per_head;
     row0 = (idx % p.tiles_per_head) * 64;
     tt_min = row0 / 64;
     n_tt = (p.R + 63) / 64 - tt_min;
-    n_tiles = p.g * n_tt;
+    h_lo = (int)((long long)hs * p.g / p.hsplit);
+    n_tiles = ((int)((long long)(hs + 1) * p.g / p.hsplit) - h_lo) * n_tt;
   }
 
   if (threadIdx.x == 0) {
@@ -179,14 +187,14 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
         if (++slot == (uint32_t)kMlaRing) { slot = 0; phase ^= 1; }
       };
       auto load_st = [&](int i, int page) {
-        const int hh = (MODE == MLA_DQ) ? 0 : kvh * p.g + i / n_tt;
+        const int hh = (MODE == MLA_DQ) ? 0 : kvh * p.g + h_lo + i / n_tt;
         const int tq = (MODE == MLA_DQ) ? 0 : (tt_min + i % n_tt) * 64;
         for (int c = 0; c < kS1; ++c) load(0, i, c, page, hh, tq);
         if (HAS_T)
           for (int c = 0; c < kS2; ++c) load(1, i, c, page, hh, tq);
       };
       auto load_m = [&](int i, int page) {
-        const int hh = (MODE == MLA_DQ) ? 0 : kvh * p.g + i / n_tt;
+        const int hh = (MODE == MLA_DQ) ? 0 : kvh * p.g + h_lo + i / n_tt;
         const int tq = (MODE == MLA_DQ) ? 0 : (tt_min + i % n_tt) * 64;
         for (int c = 0; c < NACC; ++c) load(2, i, pass * NACC + c, page, hh, tq);
       };
@@ -296,7 +304,7 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
         float cl0 = 0.f, cl1 = 0.f, cd0 = 0.f, cd1 = 0.f;
         int tq0 = 0;
         if (MODE != MLA_DQ) {
-          const int hh = kvh * p.g + i / n_tt;
+          const int hh = kvh * p.g + h_lo + i / n_tt;
           tq0 = (tt_min + i % n_tt) * 64;
           const int ta = min(tq0 + lane, p.R - 1), tb2 = min(tq0 + lane + 32, p.R - 1);
           cl0 = __ldg(p.lse + (size_t)ta * p.Hq + hh) * kLog2eMla;
@@ -380,6 +388,13 @@ __global__ void __launch_bounds__(kMlaThreads, 1) bwd_mla_kernel(const __grid_co
                 *reinterpret_cast<float4*>(dq_dst + c + j) =
                     make_float4(__uint_as_float(o[j]), __uint_as_float(o[j + 1]), __uint_as_float(o[j + 2]),
                                 __uint_as_float(o[j + 3]));
+            } else if (p.hsplit > 1) {
+              float* dst = p.kv_part + (((size_t)hs * p.R + r_idx) * p.Hkv + kvh) * OUT_D + pass * NACC * 64 + c;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) =
+                    make_float4(__uint_as_float(o[j]) * out_scale, __uint_as_float(o[j + 1]) * out_scale,
+                                __uint_as_float(o[j + 2]) * out_scale, __uint_as_float(o[j + 3]) * out_scale);
             } else {
               __nv_bfloat16* dst = p.out + ((size_t)r_idx * p.Hkv + kvh) * OUT_D + pass * NACC * 64 + c;
 #pragma unroll
@@ -420,11 +435,34 @@ static ls_status_t launch_mla(const MlaBwdParams& prm, int64_t grid, cudaStream_
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 
+int mla_kv_hsplit(const ls_pages* h, int R, int Hq) {
+  const int Hkv = h->desc.num_kv_heads;
+  const int64_t ctas = (int64_t)Hkv * ((R + 63) / 64) * 3;       // key tiles x passes of the dK launch
+  if (ctas >= 148) return 1;
+  return (int)std::max<int64_t>(1, std::min<int64_t>(Hq / Hkv, (2 * 148 + ctas - 1) / ctas));
+}
+
+// out = bf16(sum of the head ranges' fp32 sums)
+__global__ void mla_kv_reduce_kernel(const float* __restrict__ part, int hsplit, int64_t n4, __nv_bfloat16* __restrict__ out) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < hsplit; ++s) {
+      const float4 v = *reinterpret_cast<const float4*>(part + ((int64_t)s * n4 + i) * 4);
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    uint2 pk;
+    pk.x = pack_bf16(acc.x, acc.y);
+    pk.y = pack_bf16(acc.z, acc.w);
+    *reinterpret_cast<uint2*>(out + i * 4) = pk;
+  }
+}
+
 // dq_part (fp32, unscaled; only the response block's partial, at index 0, when dq_resp_only)
 // and dk_resp / dv_resp (bf16) of the 576/512 shape.
 ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
-                    void* dk_resp, void* dv_resp, bool dq_resp_only, int32_t* status_dev, cudaStream_t cs) {
+                    void* dk_resp, void* dv_resp, bool dq_resp_only, float* kv_scratch, int32_t* status_dev,
+                    cudaStream_t cs) {
   const ls_pages_desc_t& d = h->desc;
   const int R = prm->R, Hq = prm->num_q_heads, Hkv = d.num_kv_heads;
   auto dense_map = [&](CUtensorMap* m, const void* base, int heads, int dim) {
@@ -451,6 +489,8 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   P.num_phys_pages = (int)std::min<int64_t>(d.num_phys_pages, INT32_MAX);
   P.part_first = dq_resp_only ? P.S : 0;
   P.part_count = dq_resp_only ? 1 : P.S + 1;
+  P.hsplit = kv_scratch ? mla_kv_hsplit(h, R, Hq) : 1;
+  P.kv_part = kv_scratch;
   P.scale = prm->scale;
   P.scale_log2 = prm->scale * kLog2eMla;
 
@@ -474,11 +514,21 @@ ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* 
   if (st != LS_OK) return st;
   P.b3r_map = P.b1r_map;
   P.out = static_cast<__nv_bfloat16*>(dk_resp);
-  st = launch_mla<MLA_DK>(P, (int64_t)Hkv * P.tiles_per_head * 3, cs);
+  auto reduce = [&](int dim, void* out) -> ls_status_t {
+    if (P.hsplit == 1) return LS_OK;
+    const int64_t n4 = (int64_t)R * Hkv * dim / 4;
+    mla_kv_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 8), 256, 0, cs>>>(
+        kv_scratch, P.hsplit, n4, static_cast<__nv_bfloat16*>(out));
+    return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+  };
+  st = launch_mla<MLA_DK>(P, (int64_t)Hkv * P.tiles_per_head * P.hsplit * 3, cs);
+  if (st == LS_OK) st = reduce(kD1, dk_resp);
   if (st != LS_OK) return st;
   P.b3r_map = P.b2r_map;
   P.out = static_cast<__nv_bfloat16*>(dv_resp);
-  return launch_mla<MLA_DV>(P, (int64_t)Hkv * P.tiles_per_head * 2, cs);
+  st = launch_mla<MLA_DV>(P, (int64_t)Hkv * P.tiles_per_head * P.hsplit * 2, cs);
+  if (st == LS_OK) st = reduce(kD2, dv_resp);
+  return st;
 }
 
 }  // namespace ls

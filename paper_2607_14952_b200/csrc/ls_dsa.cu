@@ -518,8 +518,11 @@ extern "C" size_t ls_dsa_workspace_bytes(const ls_dsa_plan_t* p, int which) {
   const ls_pages_desc_t& ld = p->latent->desc;
   if (which == LS_WORKSPACE_FWD)      // three partials (selected prefix rows, an empty one, the response block) with their l
     return ls::align16(3 * rows * ld.dim_v * sizeof(float)) + ls::align16(3 * rows * sizeof(float));
-  if (which == LS_WORKSPACE_BWD)      // Delta and the response block's fp32 dQ partial
-    return ls::align16(rows * sizeof(float)) + rows * ld.dim_k * sizeof(float);
+  if (which == LS_WORKSPACE_BWD) {    // Delta, the response block's fp32 dQ partial, head-range sums of its dK / dV
+    const int hsplit = ls::mla_kv_hsplit(p->response, p->desc.R, p->desc.num_q_heads);
+    return ls::align16(rows * sizeof(float)) + rows * ld.dim_k * sizeof(float) +
+           (hsplit > 1 ? (size_t)hsplit * p->desc.R * ld.dim_k * sizeof(float) : 0);
+  }
   return 0;
 }
 
@@ -641,8 +644,9 @@ extern "C" ls_status_t ls_dsa_attn_bwd(const ls_dsa_plan_t* p, float scale, cons
   pr.R = d.R;
   pr.num_q_heads = d.num_q_heads;
   pr.scale = scale;
+  float* kv_scratch = ls::mla_kv_hsplit(p->response, d.R, d.num_q_heads) > 1 ? dq_resp + rows * ld.dim_k : nullptr;
   ls_status_t st = ls::bwd_mla(p->response, &pr, q, k_resp, v_resp, lse, delta, d_o, dq_resp, dk_resp, dv_resp, true,
-                               status_dev, cs);
+                               kv_scratch, status_dev, cs);
   if (st != LS_OK) return st;
   // the selected prefix rows: every (token, head) row walks its token's gathered keys, adds the response
   // block's partial and writes dQ

@@ -1130,7 +1130,11 @@ extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_a
   const bool mla_fast = f.mla && ls::mla_dq_fast(h);
   int64_t chains = (int64_t)f.Hkv * f.g * ((f.R + 127) / 128);
   if (mla_fast) chains = std::max(chains, ls::mla_dq_blocks(h, f.R, f.Hq));     // its row blocks are 64 rows
-  const size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes(chains);
+  size_t head = ((rows * sizeof(float) + 15) & ~(size_t)15) + ls::ctl_bytes(chains);
+  if (f.mla) {         // head ranges of the response dK / dV, each with an fp32 sum
+    const int hsplit = ls::mla_kv_hsplit(h, f.R, f.Hq);
+    if (hsplit > 1) head += (size_t)hsplit * f.R * f.Hkv * d.dim_k * sizeof(float);
+  }
   if (f.mla && !mla_fast)     // 576/512 with a separate V pool: one fp32 dQ per partial
     return head + (size_t)(h->num_parts() + 1) * rows * d.dim_k * sizeof(float);
   // (short responses of the aliased 576/512 shape spread the parts over several CTA pairs per row block,

@@ -144,9 +144,14 @@ inline ls_status_t configure_smem(K kernel, int bytes, bool (&done)[64]) {
 // Backward of the shared-latent 576/512 shape (ls_bwd_mla.cu): fills dq_part (fp32, unscaled,
 // [(parts+1), R, Hq, 576]; with dq_resp_only just the response block's partial, [R, Hq, 576]) and
 // the bf16 dk_resp / dv_resp.
+// kv_scratch: mla_kv_hsplit() * R * Hkv * 576 floats when that count exceeds 1 (NULL: no head split).
 ls_status_t bwd_mla(const ls_pages* h, const ls_attn_params_t* prm, const void* q, const void* k_resp,
                     const void* v_resp, const float* lse, const float* delta, const void* d_o, float* dq_part,
-                    void* dk_resp, void* dv_resp, bool dq_resp_only, int32_t* status_dev, cudaStream_t cs);
+                    void* dk_resp, void* dv_resp, bool dq_resp_only, float* kv_scratch, int32_t* status_dev,
+                    cudaStream_t cs);
+// Head ranges per key tile of the dK / dV launches of bwd_mla (a short response has too few key tiles to fill
+// the GPU); 1 = no split.
+int mla_kv_hsplit(const ls_pages* h, int R, int Hq);
 
 // Prefix part of dQ for the 576/512 shape when V aliases K (ls_bwd_mla_dq.cu): CTA pairs walk the
 // prefix parts, add dq_resp (fp32, unscaled, [R, Hq, 576]; NULL: none) and write the final bf16 dQ.

@@ -129,18 +129,20 @@ def test_workspace_sizes():
     mla = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=True)
     # 16 row blocks of 64 are too few to fill the GPU: the 4 parts go to 4 CTA pairs per block, each with an
     # fp32 sum of its own beside the response block's
-    # (this shape's dQ kernel works on 64-row blocks: 16 hand-over counters, not 8)
+    # (this shape's dQ kernel works on 64-row blocks: 16 hand-over counters, not 8; the response dK / dV of
+    # a short response are summed over 8 head ranges, each with an fp32 [R, 576] sum)
+    kv = 8 * R * 576 * 4
     assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == \
-        rows * 4 + _ctl(16) + (1 + 4) * rows * 576 * 4
+        rows * 4 + _ctl(16) + kv + (1 + 4) * rows * 576 * 4
     # many row blocks: the parts fold into the one running dQ in order, no partials
     assert B.ls_replay_attn_workspace_bytes(mla, 4096, 64, 1 / 24, B.LS_WORKSPACE_BWD) == \
         4096 * 64 * 4 + _ctl(64 * 64) + 4096 * 64 * 576 * 4
     # forward: 6 Q tiles of 16 tokens x 8 heads, two 256-channel halves of O each
     assert B.ls_replay_attn_workspace_bytes(mla, R, Hq, 1 / 24, B.LS_WORKSPACE_FWD_MERGED) == _ctl(6 * 2) + rows * 4
     sep = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=False)
-    assert B.ls_replay_attn_workspace_bytes(sep, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + (4 + 1) * rows * 576 * 4
+    assert B.ls_replay_attn_workspace_bytes(sep, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + kv + (4 + 1) * rows * 576 * 4
     empty = B.ls_prefix_pages_build(0, 64, 1, 1, 576, 512, 1, v_aliases_k=True)
-    assert B.ls_replay_attn_workspace_bytes(empty, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + (1 + 1) * rows * 576 * 4
+    assert B.ls_replay_attn_workspace_bytes(empty, R, Hq, 1 / 24, B.LS_WORKSPACE_BWD) == head + kv + (1 + 1) * rows * 576 * 4
 
 
 def test_suffix_bookkeeping_needs_a_device_handle():

@@ -193,3 +193,32 @@ def test_config5_mla1m_shared_latent():
     finally:
         parity.sampled_rows = orig
     _free(case)
+
+
+@pytest.mark.parametrize("R", [16, 64])
+def test_short_responses_at_the_2m_prefix(R):
+    # the launch configuration of `bench.py --small-r R`: the 2M prefix in 64 shards, Q tiles that pack the
+    # rows of several heads (R = 16: one tile per KV group; R = 64: two tiles of 32 tokens x 4 heads)
+    cfg = W.scaled(CONFIGS["p2m"], name="p2m-R%d" % R, R=R, num_shards=64, needles=0)
+    case = parity.Case(cfg)
+    fw = parity.check_forward(case, kv_groups=[2], full=False, per_shard=False, strict_abs=True)
+    parity.check_backward(case, fw, kv_groups=[2], full=False, tail=4, strict_abs=True)
+    _free(case)
+
+
+def test_short_response_over_the_1m_shared_latent():
+    # `bench.py --workload mla1m --small-r 4`: four row blocks of 64 heads, the parts spread over CTA pairs
+    cfg = W.scaled(CONFIGS["mla1m"], name="mla1m-R4", R=4, num_shards=64, needles=0)
+    case = parity.Case(cfg)
+    orig = parity.sampled_rows
+    try:
+        def few(c, kv, tail=4, n_random=8, seed=0, extra=()):
+            t, h = orig(c, kv, tail=tail, n_random=n_random, seed=seed, extra=extra)
+            keep = (h % 9 == 0) | (t >= c.R - 1)          # every head at the last row (dK / dV of the last key)
+            return t[keep], h[keep]
+        parity.sampled_rows = few
+        fw = parity.check_forward(case, kv_groups=[0], full=False, per_shard=False, strict_abs=True)
+        parity.check_backward(case, fw, kv_groups=[0], full=False, tail=1, strict_abs=True)
+    finally:
+        parity.sampled_rows = orig
+    _free(case)

@@ -188,3 +188,26 @@ def test_sparse_replay_at_a_64k_prefix():
     t_rows = np.repeat(t_s, cfg.Hq)
     heads = np.tile(np.arange(cfg.Hq), len(t_s))
     check_sparse(dc, got, t_rows, heads, check_kv=False)
+
+
+def test_sparse_replay_at_the_1m_workload():
+    # the launch configuration of `bench.py --mode dsa`: 1,048,576 latent positions, 1,024 response tokens,
+    # 64 heads, 32 index heads of 128, top-2,048
+    cfg = W.CONFIGS["mla1m"]
+    dc = DsaCase(cfg, 32, 2048, extra_phys_pages=0)
+    got = run_sparse(dc)
+    sel = got[0]
+    assert sel.shape == (cfg.R, 2048) and (np.diff(sel, axis=1) > 0).all() and sel.max() < cfg.P
+    rows = np.array([0, 511, cfg.R - 1])
+    want = dc.oracle_scores(rows)
+    gpu = dc.scores()[torch.as_tensor(rows, device="cuda")].double().cpu().numpy()
+    assert np.abs(gpu - want).max() <= 1e-4 * (1.0 + np.abs(want).max())
+    for i, t in enumerate(rows):
+        assert np.array_equal(sel[t], dsa.topk_select(gpu[i], 2048))         # bit-exact on the GPU's scores
+        kth = np.sort(want[i])[-2048]
+        assert (want[i][sel[t]] >= kth - 1e-3).all()                         # and the right set up to fp32 near-ties
+    t_s = np.array([0, 1, 700, cfg.R - 1])
+    heads_s = np.array([0, 5, 31, 63])
+    t_rows = np.repeat(t_s, len(heads_s))
+    heads = np.tile(heads_s, len(t_s))
+    check_sparse(dc, got, t_rows, heads, check_kv=False)
