@@ -198,7 +198,7 @@ def test_config5_mla1m_shared_latent():
 @pytest.mark.parametrize("R", [16, 64])
 def test_short_responses_at_the_2m_prefix(R):
     # the launch configuration of `bench.py --small-r R`: the 2M prefix in 64 shards, Q tiles that pack the
-    # rows of several heads (R = 16: one tile per KV group; R = 64: two tiles of 32 tokens x 4 heads)
+    # rows of several heads (R = 16: one tile per KV group; R = 64: four tiles of 21 tokens x 6 heads)
     cfg = W.scaled(CONFIGS["p2m"], name="p2m-R%d" % R, R=R, num_shards=64, needles=0)
     case = parity.Case(cfg)
     fw = parity.check_forward(case, kv_groups=[2], full=False, per_shard=False, strict_abs=True)
