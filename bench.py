@@ -41,21 +41,25 @@ DQ_KERNEL_NAME = {(256, 256): "bwd_dq3_kernel", (128, 128): "bwd_dq2_kernel", (5
 
 
 def packed_tiles(cfg, tile_rows=128):
-    """True when the library packs rows of several heads of a KV group into one Q tile (a response
-    shorter than a tile, and fewer tiles that way): which kernels run depends on it."""
+    """Number of Q tiles per KV group when the library packs rows of several heads into one Q tile (a
+    response shorter than a tile, and fewer tiles that way), else 0: which kernels run depends on it."""
     g = cfg.Hq // cfg.Hkv
     if g <= 1 or cfg.R >= tile_rows:
-        return False
+        return 0
     bh = min(g, tile_rows)
     bt = min(cfg.R, tile_rows // bh)
-    return -(-cfg.R // bt) * -(-g // bh) < g
+    tiles = -(-cfg.R // bt) * -(-g // bh)
+    return tiles if tiles < g else 0
 
 
 def kernel_names(cfg):
-    """(forward kernel, query-gradient kernel) the library launches for this workload."""
-    packed = packed_tiles(cfg)
-    fwd = "fwd2_kernel" if (cfg.Dk in (256, 576) and not packed) else "fwd_kernel"
-    dq = "bwd_dq1_kernel" if (packed and cfg.Dk != 576) else DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv))
+    """(forward kernel, query-gradient kernel) the library launches for this workload: the single-CTA
+    kernels when a KV group is one packed tile, the pair kernels otherwise (head dim 128: single CTAs)."""
+    tiles = packed_tiles(cfg)
+    fwd = "fwd2_kernel" if (cfg.Dk in (256, 576) and tiles != 1) else "fwd_kernel"
+    dq = DQ_KERNEL_NAME.get((cfg.Dk, cfg.Dv))
+    if cfg.Dk != 576 and tiles and (tiles == 1 or cfg.Dk != 256):
+        dq = "bwd_dq1_kernel"
     return fwd, dq
 
 

@@ -1343,11 +1343,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   const bool is_resp = it.is_resp;
   auto tile_of = [&](int qt, int& hh, int& r0) {
     if (qt < p.nq_tiles) {
-      hh = kvh * p.g + qt / p.tiles_per_head;
-      r0 = (qt % p.tiles_per_head) * 128;
-    } else {
+      hh = kvh * p.g + (qt / p.tiles_tok) * p.bh;     // tile of bt tokens x bh heads (RowTiling)
+      r0 = (qt % p.tiles_tok) * p.bt;
+    } else {                                           // odd tile count: the pair's second CTA works on zero rows
       hh = kvh * p.g + p.g - 1;
-      r0 = p.tiles_per_head * 128;
+      r0 = p.tiles_tok * p.bt;
     }
   };
   const int qtile = 2 * pairi + (int)rank;
@@ -1357,7 +1357,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = p.no_resp ? 0 : min(p.R, max(row0, row0_o) + 128);
+    tokens = p.no_resp ? 0 : min(p.R, max(row0, row0_o) + p.bt);
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -1369,7 +1369,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   if (warp == 0) {
     // =========================================================== producer (one thread per CTA)
     if (lane == 0 && n_tiles > 0) {
-      const int a_rows = 128;
+      const int a_rows = p.bt * p.bh;
       if (leader) mbar_arrive_expect_tx(a_full, 2 * 2 * C::SLABS * a_rows * 128);
       for (int c = 0; c < C::SLABS; ++c) {
         tma_load_5d_pair(a1_smem + c * 16384, &p.a1_map, a_full, 0, row0, c, h, 0);
@@ -1519,11 +1519,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
     const int quad = warp & 3;
     const int sub = (warp - 2) >> 2;                // which 32 of every 64-column quarter this thread owns (2 threads per row)
     const int row = quad * 32 + lane;
-    const int r_idx = row0 + row;
-    const int hr = h;
+    const int hj = row / p.bt;                      // head and token of this row of the tile
+    const int r_idx = row0 + row - hj * p.bt;
+    const int hr = min(h + hj, p.Hq - 1);
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const bool tile_ok = qtile < p.nq_tiles;
-    const bool row_ok = tile_ok && r_idx < p.R;
+    const bool row_ok = tile_ok && hj < p.bh && r_idx < p.R && h + hj < (kvh + 1) * p.g;
     const size_t ri = (size_t)min(r_idx, p.R - 1) * p.Hq + hr;
     bool ok = true;
     if (n_tiles > 0) {
@@ -1767,14 +1768,12 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   P.bt = rt.bt;
   P.bh = rt.bh;
   P.tiles_tok = rt.tiles_tok;
-  if (rt.packed) {                       // short response: rows of several heads share a Q tile
-    P.nq_tiles = rt.nq_tiles;
-    st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, rt.bt, rt.bh);
-    if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, rt.bt, rt.bh);
-  } else {
-    st = dense_map(&P.a1_map, q, Hq, 128, 1);
-    if (st == LS_OK) st = dense_map(&P.a2_map, d_o, Hq, 128, 1);
-  }
+  // short response: rows of several heads share a Q tile; a KV group of one tile runs on the single-CTA
+  // kernel, several tiles (head dim 256) on the pair kernel, two tiles sharing every key tile
+  const bool single = rt.packed && (rt.nq_tiles == 1 || D != 256);
+  P.nq_tiles = rt.nq_tiles;
+  st = ls::encode_map_rows(&P.a1_map, q, D, R, Hq, rt.bt, rt.bh);
+  if (st == LS_OK) st = ls::encode_map_rows(&P.a2_map, d_o, D, R, Hq, rt.bt, rt.bh);
   if (st == LS_OK) st = dense_map(&P.rk_s, k_resp, Hkv, 64, 2);
   if (st == LS_OK) st = dense_map(&P.rv_s, v_resp, Hkv, 64, 2);
   if (st == LS_OK) st = dense_map(&P.rk_m, k_resp, Hkv, 128, 1);
@@ -1789,7 +1788,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   if (st == LS_OK) st = ls::pool_map(&P.pv_m_tail, h, 1, mbox, 1, true);
   if (st != LS_OK) return st;
   if (cudaMemsetAsync(ctl, 0, ctl_bytes, cs) != cudaSuccess) return LS_ERR_CUDA;
-  if (rt.packed) {
+  if (single) {
     // short response: one single-CTA work item per (KV head, part, Q tile); K/V pages come from DRAM once
     const int pbox = small_pages ? 64 : 128, pgroups = small_pages ? 1 : 2;
     st = dense_map(&P.b1r_map, k_resp, Hkv, 128, 2);

@@ -671,11 +671,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   const bool is_resp = it.is_resp;
   auto tile_of = [&](int qt, int& hh, int& r0) {
     if (qt < p.nq_tiles) {
-      hh = kvh * p.g + qt / p.tiles_tok;     // (this kernel serves tiles of 128 tokens of one head only)
-      r0 = (qt % p.tiles_tok) * 128;
+      hh = kvh * p.g + (qt / p.tiles_tok) * p.bh;     // tile of bt tokens x bh heads (RowTiling)
+      r0 = (qt % p.tiles_tok) * p.bt;
     } else {                                 // odd tile count: the pair's second CTA works on zero rows
       hh = kvh * p.g + p.g - 1;
-      r0 = p.tiles_tok * 128;                // token coordinate past R: TMA delivers zeros
+      r0 = p.tiles_tok * p.bt;               // token coordinate past R: TMA delivers zeros
     }
   };
   const int qtile = 2 * pairi + (int)rank;
@@ -685,7 +685,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
   int64_t tokens;
   int page_off = 0, n_pages = 0, tail_slot = -1;
   if (is_resp) {
-    tokens = p.no_resp ? 0 : min(p.R, max(t0, t0_o) + 128);   // both CTAs walk the longer causal range
+    tokens = p.no_resp ? 0 : min(p.R, max(t0, t0_o) + p.bt);  // both CTAs walk the longer causal range
   } else {
     tokens = p.part_tokens[part];
     page_off = p.part_page_offset[part];
@@ -831,10 +831,11 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFwdThreads, 1)
     // =========================================================== softmax + epilogue (both CTAs)
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    const int t = t0 + row;
-    const int hr = h;
+    const int hj = row / p.bt;               // this thread's (token, head) inside the tile of bt tokens x bh heads
+    const int t = t0 + row - hj * p.bt;
+    const int hr = min(h + hj, p.Hq - 1);
     const bool tile_ok = qtile < p.nq_tiles;
-    const bool row_ok = tile_ok && t < p.R;
+    const bool row_ok = tile_ok && hj < p.bh && t < p.R && h + hj < (kvh + 1) * p.g;
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     const size_t out_row = ((size_t)fwd_out_part(p, it) * p.R + (size_t)min(t, p.R - 1)) * p.Hq + hr;
     const bool to_resp = is_resp && p.chain_mode != 2;
@@ -1015,7 +1016,9 @@ static ls_status_t run_forward(const ls_pages* h, const ls_attn_params_t* prm, i
   const int dvt = f.mla ? 256 : d.dim_v;                    // O channels per CTA
   const int vkeys = (d.dim_k == 256 ? 32768 : 16384) / (dvt * 2);
   const bool small_pages = d.page_size == 64;
-  const bool pair = (d.dim_k == 256 || f.mla) && !f.packed;  // CTA pairs share every key tile between two Q tiles
+  // CTA pairs share every key tile between two Q tiles; a short response whose KV group is ONE packed tile
+  // streams K/V once on the single-CTA kernel
+  const bool pair = (d.dim_k == 256 || f.mla) && !(f.packed && f.nq_tiles == 1);
   if (prm->flags & LS_FLAG_NO_RESPONSE_BLOCK) k_resp = v_resp = q;   // the response maps are encoded but never used
   ls_status_t st = encode_map_rows(&P.q_map, q, d.dim_k, R, Hq, f.rt.bt, f.rt.bh);
   if (pair) {
