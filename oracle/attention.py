@@ -198,3 +198,39 @@ def merge(o_parts, lse_parts):
         o = np.where(a[..., None] > 0, n / a[..., None], 0.0)
         l = m_safe + np.log(a)
     return o, l
+
+
+def round_bf16(x):
+    """Nearest bf16 value (8 significant bits, ties to even) of every element, as float64.
+    Written out on the number itself: quantum 2^(e-7) for 2^e <= |x| < 2^(e+1) (normal range)."""
+    x = np.asarray(x, dtype=np.float64)
+    out = np.zeros_like(x)
+    nz = (x != 0) & np.isfinite(x)
+    e = np.floor(np.log2(np.abs(x[nz])))
+    q = np.exp2(np.maximum(e, -126.0) - 7.0)
+    out[nz] = np.rint(x[nz] / q) * q          # rint rounds halves to even
+    out[~np.isfinite(x)] = x[~np.isfinite(x)]
+    return out
+
+
+def merge_bf16_numerator(o_parts, lse_parts):
+    """The merge as the paper's production run carries it out (Sec. "Global Full-Attention Forward
+    Composition", last paragraph): the numerator n = sum_r e^{l_r - m} o_r is exchanged and summed in
+    bf16, the maximum, the denominator and the global LSE stay in full precision.  Reading: every
+    shard's term e^{l_r - m} o_r is rounded to bf16, the terms are added in shard order and every
+    running sum is rounded to bf16 again (the order of a collective's additions is not stated);
+    o = n / a is then formed from the bf16 n."""
+    o_parts = np.asarray(o_parts, dtype=np.float64)
+    lse_parts = np.asarray(lse_parts, dtype=np.float64)
+    m = lse_parts.max(axis=0)
+    m_safe = np.where(np.isfinite(m), m, 0.0)
+    w = np.exp(lse_parts - m_safe)
+    a = w.sum(axis=0)
+    n = np.zeros(o_parts.shape[1:])
+    for r in range(o_parts.shape[0]):
+        n = round_bf16(n + round_bf16(w[r][..., None] * o_parts[r]))
+    with np.errstate(divide="ignore", invalid="ignore"):
+        o = np.where(a[..., None] > 0, n / a[..., None], 0.0)
+        l = m_safe + np.log(a)
+    return o, l
+

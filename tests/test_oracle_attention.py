@@ -310,3 +310,44 @@ def test_local_attention_value_slice_of_the_key_page():
     # without dv the whole page would be the value: the slice is what makes the shapes differ
     o_full, _ = oa.local_attention(q, 0, pool, pool, table, pg, positions, scale)
     assert o_full.shape == (3, dk) and np.allclose(o_full[:, :dv], o)
+
+
+def test_round_bf16_against_bit_patterns_and_ties():
+    # every bf16 value is a float32 whose low 16 bits are zero: rounding must land on such a value, be the
+    # nearest one, and send exact halves to the even neighbour
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.standard_normal(2000) * 10.0 ** rng.integers(-6, 6, 2000), [0.0, 1.0, -3.5, 2.0 ** -20]])
+    r = oa.round_bf16(x)
+    bits = r.astype(np.float32).view(np.uint32)
+    assert (r.astype(np.float32).astype(np.float64) == r).all() and (bits & 0xFFFF == 0).all()
+    ulp = np.exp2(np.floor(np.log2(np.abs(np.where(x == 0, 1.0, x)))) - 7)
+    assert (np.abs(r - x) <= ulp / 2 + 1e-300).all()
+    # 1 + 2^-8 is halfway between 1 and 1 + 2^-7: even neighbour 1; 1 + 3 * 2^-8 is halfway: even neighbour 1 + 2^-6
+    assert oa.round_bf16(np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, 1 + 2.0 ** -8 + 2.0 ** -20])).tolist() == \
+        [1.0, 1 + 2.0 ** -6, 1 + 2.0 ** -7]
+
+
+def test_merge_bf16_numerator_hand_example_and_bounds():
+    # two shards of equal weight, o = 1 and 2^-9: the fp32 numerator 1 + 2^-9 is below half a bf16 step
+    # above 1, so the bf16 numerator is 1 and o = 1/2, where the full-precision merge gives (1 + 2^-9)/2
+    o = np.array([[[1.0]], [[2.0 ** -9]]])
+    l = np.array([[0.3], [0.3]])
+    got, lse = oa.merge_bf16_numerator(o, l)
+    assert got[0, 0] == 0.5 and abs(lse[0] - (0.3 + np.log(2.0))) < 1e-15
+    assert oa.merge(o, l)[0][0, 0] == (1 + 2.0 ** -9) / 2
+    # one shard: the output is that shard's o rounded to bf16; LSE untouched
+    rng = np.random.default_rng(8)
+    o1 = rng.standard_normal((1, 7, 5))
+    g1, l1 = oa.merge_bf16_numerator(o1, rng.standard_normal((1, 7)))
+    assert (g1 == oa.round_bf16(o1[0])).all()
+    # S shards: within S + 1 roundings of the exact merge (each 2^-9 relative to the running magnitude), same LSE
+    S = 9
+    o = rng.standard_normal((S, 50, 16))
+    l = rng.standard_normal((S, 50)) * 3.0
+    l[2, ::5] = -np.inf
+    got, lse = oa.merge_bf16_numerator(o, l)
+    ref, lref = oa.merge(o, l)
+    w = np.exp(l - l.max(axis=0))
+    bound = (S + 1) * 2.0 ** -9 * (w[..., None] * np.abs(o)).sum(axis=0) / w.sum(axis=0)[..., None]
+    assert (np.abs(got - ref) <= bound).all() and np.array_equal(lse, lref)
+    assert np.abs(got - ref).max() > 0          # the rounding is really there
