@@ -193,6 +193,18 @@ ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim_v,
                          void* o_bf16, float* o_f32, float* lse, int32_t* status_dev, void* stream);
 
 /*
+ * The same merge with the numerator carried the way the paper's production run exchanges it
+ * (Sec. "Global Full-Attention Forward Composition", last paragraph: n_t is reduced in BF16,
+ * the maximum, the denominator and the global LSE stay FP32): every shard's term
+ * e^{l_r-m} o_r is rounded to bf16 and the terms are added in shard order with a bf16
+ * running sum; o = n/a from that n.  Same arguments, layouts and status rules as
+ * ls_lse_merge; lse is identical to ls_lse_merge's.
+ */
+ls_status_t ls_lse_merge_bf16_numerator(int32_t num_parts, int64_t rows, int32_t dim_v,
+                         const float* o_part, const float* lse_part,
+                         void* o_bf16, float* o_f32, float* lse, int32_t* status_dev, void* stream);
+
+/*
  * Replay forward with the merge folded in: the composed output of Eq. qwen-global-attn and
  * its log-normaliser, without the per-shard partials ever reaching memory.  This is the
  * form of the score-only passes of a group member (old and reference scoring keep no

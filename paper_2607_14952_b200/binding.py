@@ -69,6 +69,7 @@ def lib():
         L.ls_replay_attn_workspace_bytes.restype = C.c_size_t
         L.ls_replay_attn_fwd.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
         L.ls_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.ls_lse_merge_bf16_numerator.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp, vp, vp]
         L.ls_replay_attn_fwd_merged.argtypes = [vp, C.POINTER(ls_attn_params_t), vp, vp, vp, vp, vp, vp, vp, C.c_size_t,
                                                 vp, vp]
         L.ls_suffix_pages_reserve.argtypes = [vp, i32, i32, vp, vp]
@@ -107,7 +108,8 @@ def lib():
         L.ls_status_string.argtypes = [C.c_int]
         L.ls_status_string.restype = C.c_char_p
         for f in ("ls_prefix_pages_build", "ls_prefix_pages_export", "ls_prefix_pages_checksum",
-                  "ls_prefix_pages_destroy", "ls_replay_attn_fwd", "ls_lse_merge", "ls_replay_attn_bwd",
+                  "ls_prefix_pages_destroy", "ls_replay_attn_fwd", "ls_lse_merge", "ls_lse_merge_bf16_numerator",
+                  "ls_replay_attn_bwd",
                   "ls_replay_attn_fwd_merged", "ls_suffix_pages_reserve", "ls_suffix_pages_append",
                   "ls_suffix_pages_pop"):
             getattr(L, f).restype = C.c_int
@@ -226,8 +228,10 @@ def ls_replay_attn_fwd(pages, q, k_resp, v_resp, scale, o_part=None, lse_part=No
     return o_part, lse_part
 
 
-def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=True, want_f32=True, status=None):
-    """o_part [parts, ..., Dv] fp32, lse_part [parts, ...] fp32 -> (o_bf16, o_f32, lse)."""
+def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=True, want_f32=True, status=None,
+                 bf16_numerator=False):
+    """o_part [parts, ..., Dv] fp32, lse_part [parts, ...] fp32 -> (o_bf16, o_f32, lse).
+    bf16_numerator: ls_lse_merge_bf16_numerator (the numerator summed in bf16)."""
     parts, dv = o_part.shape[0], o_part.shape[-1]
     rows = lse_part[0].numel()
     shape = tuple(o_part.shape[1:])
@@ -237,8 +241,8 @@ def ls_lse_merge(o_part, lse_part, o_bf16=None, o_f32=None, lse=None, want_bf16=
         o_f32 = torch.empty(shape, dtype=torch.float32, device=o_part.device)
     if lse is None:
         lse = torch.empty(shape[:-1], dtype=torch.float32, device=o_part.device)
-    st = lib().ls_lse_merge(parts, rows, dv, _ptr(o_part), _ptr(lse_part), _ptr(o_bf16), _ptr(o_f32), _ptr(lse),
-                            _ptr(status), _stream())
+    fn = lib().ls_lse_merge_bf16_numerator if bf16_numerator else lib().ls_lse_merge
+    st = fn(parts, rows, dv, _ptr(o_part), _ptr(lse_part), _ptr(o_bf16), _ptr(o_f32), _ptr(lse), _ptr(status), _stream())
     _check(st, "ls_lse_merge")
     return o_bf16, o_f32, lse
 

@@ -1,6 +1,9 @@
 // Stable LSE/output merge of per-shard partials (Eq. qwen-lse-parts, Eq. qwen-global-attn):
 //   m = max_r l_r;  a = sum_r e^{l_r - m};  n = sum_r e^{l_r - m} o_r;  o = n / a;  l = m + log a.
-// HBM-bound: one warp per row, 16-byte vector loads, fp32 throughout.
+// HBM-bound: one warp per row, 16-byte vector loads, fp32 throughout -- or, BF16N, with the numerator
+// carried the way the paper's production run exchanges it (Sec. "Global Full-Attention Forward
+// Composition", last paragraph): every shard's term e^{l_r - m} o_r rounded to bf16 and the terms added in
+// shard order with a bf16 running sum; maximum, denominator and l stay fp32.
 #include <cuda_bf16.h>
 
 #include "ls_internal.h"
@@ -9,6 +12,9 @@ namespace ls {
 
 constexpr int kMergeWarps = 8;
 
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+template <bool BF16N>
 __global__ void __launch_bounds__(kMergeWarps * 32) merge_kernel(int num_parts, int64_t rows, int dv,
                                                                  const float* __restrict__ o_part,
                                                                  const float* __restrict__ lse_part,
@@ -33,10 +39,17 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_kernel(int num_parts, 
       const float w = expf(lse_part[(int64_t)r * rows + row] - m_safe);
       if (w == 0.f) continue;     // an empty partial weighs exactly nothing
       const float4 v = *reinterpret_cast<const float4*>(o_part + ((int64_t)r * rows + row) * dv + c);
-      acc.x = fmaf(w, v.x, acc.x);
-      acc.y = fmaf(w, v.y, acc.y);
-      acc.z = fmaf(w, v.z, acc.z);
-      acc.w = fmaf(w, v.w, acc.w);
+      if (BF16N) {
+        acc.x = bf16_round(acc.x + bf16_round(w * v.x));
+        acc.y = bf16_round(acc.y + bf16_round(w * v.y));
+        acc.z = bf16_round(acc.z + bf16_round(w * v.z));
+        acc.w = bf16_round(acc.w + bf16_round(w * v.w));
+      } else {
+        acc.x = fmaf(w, v.x, acc.x);
+        acc.y = fmaf(w, v.y, acc.y);
+        acc.z = fmaf(w, v.z, acc.z);
+        acc.w = fmaf(w, v.w, acc.w);
+      }
     }
     acc.x *= inv_a;
     acc.y *= inv_a;
@@ -61,9 +74,9 @@ __global__ void __launch_bounds__(kMergeWarps * 32) merge_kernel(int num_parts, 
 
 }  // namespace ls
 
-extern "C" ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim_v, const float* o_part,
-                                    const float* lse_part, void* o_bf16, float* o_f32, float* lse,
-                                    int32_t* status_dev, void* stream) {
+static ls_status_t launch_merge(bool bf16n, int32_t num_parts, int64_t rows, int32_t dim_v, const float* o_part,
+                                const float* lse_part, void* o_bf16, float* o_f32, float* lse, int32_t* status_dev,
+                                void* stream) {
   if (num_parts < 1 || rows < 0 || dim_v < 4 || dim_v % 4 != 0) return LS_ERR_INVALID_ARG;
   if (!o_part || !lse_part || !lse) return LS_ERR_INVALID_ARG;
   if (!ls::aligned16(o_part) || (o_f32 && !ls::aligned16(o_f32)) || (o_bf16 && !ls::aligned16(o_bf16)))
@@ -71,7 +84,24 @@ extern "C" ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim
   if (rows == 0) return LS_OK;
   const int64_t blocks = (rows + ls::kMergeWarps - 1) / ls::kMergeWarps;
   if (blocks > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  ls::merge_kernel<<<(int)blocks, ls::kMergeWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(
-      num_parts, rows, dim_v, o_part, lse_part, static_cast<__nv_bfloat16*>(o_bf16), o_f32, lse, status_dev);
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (bf16n)
+    ls::merge_kernel<true><<<(int)blocks, ls::kMergeWarps * 32, 0, cs>>>(
+        num_parts, rows, dim_v, o_part, lse_part, static_cast<__nv_bfloat16*>(o_bf16), o_f32, lse, status_dev);
+  else
+    ls::merge_kernel<false><<<(int)blocks, ls::kMergeWarps * 32, 0, cs>>>(
+        num_parts, rows, dim_v, o_part, lse_part, static_cast<__nv_bfloat16*>(o_bf16), o_f32, lse, status_dev);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+
+extern "C" ls_status_t ls_lse_merge(int32_t num_parts, int64_t rows, int32_t dim_v, const float* o_part,
+                                    const float* lse_part, void* o_bf16, float* o_f32, float* lse,
+                                    int32_t* status_dev, void* stream) {
+  return launch_merge(false, num_parts, rows, dim_v, o_part, lse_part, o_bf16, o_f32, lse, status_dev, stream);
+}
+
+extern "C" ls_status_t ls_lse_merge_bf16_numerator(int32_t num_parts, int64_t rows, int32_t dim_v, const float* o_part,
+                                                   const float* lse_part, void* o_bf16, float* o_f32, float* lse,
+                                                   int32_t* status_dev, void* stream) {
+  return launch_merge(true, num_parts, rows, dim_v, o_part, lse_part, o_bf16, o_f32, lse, status_dev, stream);
 }

@@ -54,3 +54,32 @@ def test_bounded_wait_gives_up_and_reports_timeout():
     assert int(status.item()) == B.LS_ERR_TIMEOUT
     x = torch.ones(4, device="cuda") * 2                      # the context still works
     assert float(x.sum()) == 8.0
+
+
+@pytest.mark.parametrize("parts,dv", [(1, 128), (9, 256), (33, 512)])
+def test_merge_with_the_numerator_summed_in_bf16(parts, dv):
+    # ls_lse_merge_bf16_numerator against the oracle's emulation of the same roundings; the two form the
+    # products w * o in fp32 and fp64, so a term may now and then fall on the other side of a bf16 rounding
+    # boundary: one bf16 step of the running magnitude per element is allowed, the typical error must be far less
+    g = torch.Generator(device="cuda").manual_seed(parts * 77 + dv)
+    rows = 300 + parts
+    o = torch.randn(parts, rows, dv, generator=g, device="cuda")
+    l = torch.randn(parts, rows, generator=g, device="cuda") * 4.0
+    if parts > 1:
+        l[1, ::4] = -float("inf")
+        o[1, ::4] = 0.0
+    o_bf16, o_f32, lse = B.ls_lse_merge(o, l, bf16_numerator=True)
+    _, o_plain, lse_plain = B.ls_lse_merge(o, l)
+    torch.cuda.synchronize()
+    od, ld = o.double().cpu().numpy(), l.double().cpu().numpy()
+    ro, rl = oa.merge_bf16_numerator(od, ld)
+    assert torch.equal(lse, lse_plain) and np.abs(lse.double().cpu().numpy() - rl).max() < 1e-4
+    got = o_f32.double().cpu().numpy()
+    w = np.exp(ld - ld.max(axis=0))
+    step = 2.0 ** -7 * (w[..., None] * np.abs(od)).sum(axis=0) / w.sum(axis=0)[..., None]
+    err = np.abs(got - ro)
+    assert (err <= step + 1e-6).all()
+    assert (err <= 1e-6).mean() > 0.98                     # almost every element takes identical roundings
+    assert torch.equal(o_f32.to(torch.bfloat16), o_bf16)
+    if parts > 1:                                          # and it is not the fp32 merge
+        assert (o_f32 != o_plain).any()
