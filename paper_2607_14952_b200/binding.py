@@ -20,6 +20,7 @@ LS_ERR_WORKSPACE, LS_ERR_STALE, LS_ERR_CUDA, LS_ERR_TIMEOUT, LS_ERR_NONFINITE = 
 LS_SHARD_CONTIGUOUS, LS_SHARD_CYCLIC, LS_SHARD_ZIGZAG = 0, 1, 2
 LS_WORKSPACE_FWD, LS_WORKSPACE_BWD, LS_WORKSPACE_FWD_MERGED = 0, 1, 2
 LS_FLAG_ADD_SUFFIX_GRAD = 1
+LS_FLAG_NO_RESPONSE_BLOCK = 2
 LS_KERNEL_FWD, LS_KERNEL_BWD_DQ, LS_KERNEL_BWD_DK, LS_KERNEL_BWD_DV = 0, 1, 2, 3
 
 
@@ -304,9 +305,9 @@ def ls_replay_attn_bwd(pages, q, k_resp, v_resp, o_f32, lse, d_o, scale, workspa
         workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
     if dq is None:
         dq = torch.empty_like(q)
-    if dk_resp is None:
+    if dk_resp is None and k_resp is not None:       # (no response block: nothing to return for its keys)
         dk_resp = torch.empty_like(k_resp)
-    if dv_resp is None:
+    if dv_resp is None and v_resp is not None:
         dv_resp = torch.empty_like(v_resp)
     prm = _params(R, Hq, scale, flags, generation)
     st = lib().ls_replay_attn_bwd(pages.handle, C.byref(prm), _ptr(q), _ptr(k_resp), _ptr(v_resp), _ptr(o_f32),

@@ -547,12 +547,14 @@ MlaDqSplit mla_dq_split(const ls_pages* h, int R, int Hq) {
   const int parts = h->prefix_parts();
   MlaDqSplit sp;
   if (blocks >= 74) {
-    // a row block for every CTA pair of the GPU and more: ranges of about 48 MB of keys (whole parts), the
-    // pairs of a range run together, so that its keys stay in L2 while every row block passes over them.
-    // (Measured at the 1M workload, dQ pass: 19 MB ranges 325 ms, 38 MB 314 ms, 75 MB 316 ms: shorter
-    // ranges pay the pair's prologue and hand-over more often, longer ones start to fall out of L2.)
+    // a row block for every CTA pair of the GPU and more: ranges of whole parts holding up to 1.5 stream
+    // budgets of keys (48 MB by default), the pairs of a range run together, so that its keys stay in L2
+    // while every row block passes over them.  (Measured at the 1M workload, dQ pass: 19 MB ranges 325 ms,
+    // 38 MB 314 ms, 75 MB 316 ms: shorter ranges pay the pair's prologue and hand-over more often, longer
+    // ones start to fall out of L2.)
+    const int64_t budget = ((h->desc.stream_budget_kib > 0 ? (int64_t)h->desc.stream_budget_kib : 32768ll) << 10) * 3 / 2;
     const int64_t part_bytes = std::max<int64_t>(1, h->desc.prefix_len * 576 * 2 / std::max(parts, 1));
-    const int per_range = (int)std::max<int64_t>(1, std::min<int64_t>(parts, (48ll << 20) / part_bytes));
+    const int per_range = (int)std::max<int64_t>(1, std::min<int64_t>(parts, budget / part_bytes));
     sp.count = (parts + per_range - 1) / per_range;
     sp.chain = sp.count > 1;
   } else {

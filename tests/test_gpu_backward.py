@@ -143,6 +143,28 @@ def test_shared_latent_dq_paths(aliased):
         parity.check_backward(case, fw)
 
 
+def test_shared_latent_dq_chained_ranges():
+    # many row blocks (64 heads x 2 blocks of the 96 rows) and a tiny stream budget: the transposed dQ kernel
+    # hands the pairs of one range of parts out together and folds the 32 ranges of every row block into one
+    # running dQ, in order, on top of the response block's partial
+    cfg = small("mla_chain", Dk=576, Dv=512, v_aliases_k=True, Hq=64, Hkv=1, P=64 * 40, page_size=64, num_shards=4, R=96,
+                seed=431)
+    case = parity.Case(cfg, stream_budget_kib=96)
+    fw = parity.check_forward(case, per_shard=False)
+    parity.check_backward(case, fw)
+    # without a response block the running dQ starts empty: same result as the one-range walk of a handle
+    # with the default budget, up to the fp32 summation order and the bf16 output rounding
+    q, k, v, d_o = case.member(0)
+    _, _, _, o_f32, lse = case.forward(q, k, v)
+    a = case.backward(q, None, None, o_f32, lse, d_o, flags=B.LS_FLAG_NO_RESPONSE_BLOCK)[0].float()
+    one = parity.Case(cfg)
+    b = one.backward(q, None, None, o_f32, lse, d_o, flags=B.LS_FLAG_NO_RESPONSE_BLOCK)[0].float()
+    torch.cuda.synchronize()
+    assert torch.isfinite(a).all() and (a - b).abs().max() <= 2.0 ** -7 * b.abs().max() + 1e-6
+    again = case.backward(q, None, None, o_f32, lse, d_o, flags=B.LS_FLAG_NO_RESPONSE_BLOCK)[0].float()
+    assert torch.equal(a, again)                       # fixed fold order: bit-reproducible
+
+
 def test_shared_latent_dq_ignores_unmapped_pages():
     # 64-token pages, an odd page count per shard (the last 128-key tile of a shard is half
     # empty), a pool larger than the prefix whose unmapped pages -- physical page 0 among them --
