@@ -248,7 +248,16 @@ def run_cuda(args):
                                      status=status, flags=B.LS_FLAG_ADD_SUFFIX_GRAD)
 
     # kernels of this library launched per step (memsets and copies are not kernels)
-    bwd_launches = 5 if mla else 4                       # Delta, dQ (+ the response block's dQ for 576/512), dK, dV
+    bwd_launches = 4                                     # Delta, dQ, dK, dV
+    if mla:
+        # + the response block's dQ partial; + a reduce per dK / dV when their key tiles alone cannot fill the GPU
+        # (head ranges); + a reduce of the part ranges when a short response spreads them over CTA pairs
+        bwd_launches = 5
+        if cfg.Hkv * -(-cfg.R // 64) * 3 < 148:
+            bwd_launches += 2
+        blocks64 = cfg.Hkv * (packed_tiles(cfg, 64) or (cfg.Hq // cfg.Hkv) * -(-cfg.R // 64))
+        if blocks64 < 74 and S > 1:
+            bwd_launches += 1
     launches = {"replay": 2 + bwd_launches, "fused": 1 + bwd_launches, "score": 1,
                 "blocks": 0 if not nblocks else sum(1 + 2 + 1 + bwd_launches + 2 * b for b in range(nblocks))}[mode]
 
@@ -271,14 +280,33 @@ def run_cuda(args):
     if rank == 0:
         sampler.start()
     barrier()
+    graph = None
+    if args.graph and mode != "blocks":
+        # the step's launches captured once and replayed: no host work per step (the per-call tensor maps and
+        # kernel arguments are baked in, so the replays all take member 0's buffers)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step(*members[0])
+        graph.replay()
+        barrier()
     for i in range(args.steps):
-        if mode != "blocks":
+        if mode != "blocks" and graph is None:
             for k in kev:
                 B.ls_profile_arm_events(k, kev[k][i][0], kev[k][i][1])
         ev[i][0].record()
-        step(*members[i % n_members])
+        if graph is not None:
+            graph.replay()
+        else:
+            step(*members[i % n_members])
         ev[i][1].record()
     barrier()
+    if graph is not None:              # the dominant kernels' own times: one eager step with armed events
+        for k in kev:
+            B.ls_profile_arm_events(k, kev[k][0][0], kev[k][0][1])
+        step(*members[0])
+        barrier()
+        for k in kev:
+            kev[k] = [kev[k][0]] * args.steps
     clocks = sampler.stop() if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
     ms = sum(step_ms)
@@ -331,6 +359,7 @@ def run_cuda(args):
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "%s: P=%d R=%d Hq=%d Hkv=%d Dk=%d Dv=%d page=%d shards=%d, one member per step" % (
             cfg.name, cfg.P, cfg.R, cfg.Hq, cfg.Hkv, cfg.Dk, cfg.Dv, cfg.page_size, cfg.num_shards),
+            "launch": "cuda graph replay" if graph is not None else "eager",
             "mode": mode if not nblocks else "blocks x%d of %d tokens (suffix pass + reverse policy pass)" % (nblocks, rb),
             "l2": "inputs larger than L2 (%.2f GiB of K/V streamed per pass)" % (pool_bytes / 2**30),
             "parallelism": "replicas x%d" % world, "flops_per_step": step_flops,
@@ -546,6 +575,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-rows", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="replay the step as one CUDA graph (launch-bound workloads)")
     ap.add_argument("--small-r", type=int, default=0, help="short-response regime: R rows per head")
     ap.add_argument("--shards", type=int, default=0, help="key shards for --small-r (default 64)")
     ap.add_argument("--prefix", type=int, default=0, help="override the workload's prefix length (profiling on a small case)")
