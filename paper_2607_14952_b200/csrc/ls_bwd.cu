@@ -62,6 +62,10 @@ struct BwdParams {
   int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   // dQ pass of a short response (single-CTA kernel): Q tiles of bt tokens x bh heads (RowTiling)
   int bt, bh, tiles_tok;
+  // single-CTA dQ kernel, one tile per KV group: every part writes its fp32 sum to dq_split
+  // [parts + 1, R, Hq, D] and a reduce kernel adds them (a chain of parts + 1 links per KV group would
+  // run its folds one after the other at the end of a launch in which all parts finish together)
+  float* dq_split;
   int no_resp;   // dQ pass: the response block is left out
   // dK / dV pass: keys of a suffix block (1) read through pages [key_page_off, ..) of part_pages,
   // key_tokens of them, first gradient slot grad_slot0; or the response block (0)
@@ -1180,15 +1184,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
       if (ok) ok = bwd_wait_warp(acc_final, 0, abort_flag);
       if (ok) tc_fence_after();
     }
-    // ---- epilogue: add this part's sum to the running dQ of the KV group's rows, in link order
-    const bool fold = it.link > 0, last = it.link == p.parts;
-    int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + qtile;
-    if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
-    if (ok)
-      dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, fold, last, p.scale,
-                          p.dq_acc + ri * D + half * (D / 2), p.dq + ri * D + half * (D / 2), row_ok);
-    const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
-    if (row == 0 && half == 0 && all_ok) chain_publish(counter, it.link + 1);
+    // ---- epilogue: this part's sum goes to its own partial (one tile per KV group), or is added to the
+    // running dQ of the tile's rows, in link order
+    if (p.dq_split) {
+      if (ok)
+        dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, false, false, p.scale,
+                            p.dq_split + ((size_t)it.link * p.R * p.Hq + ri) * D + half * (D / 2), nullptr, row_ok);
+    } else {
+      const bool fold = it.link > 0, last = it.link == p.parts;
+      int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + qtile;
+      if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
+      if (ok)
+        dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, fold, last, p.scale,
+                            p.dq_acc + ri * D + half * (D / 2), p.dq + ri * D + half * (D / 2), row_ok);
+      const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
+      if (row == 0 && half == 0 && all_ok) chain_publish(counter, it.link + 1);
+    }
   }
 
   tc_fence_before();
@@ -1743,6 +1754,7 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
   P.lse = lse;
   P.delta = delta;
   P.dq_acc = dq_acc;
+  P.dq_split = nullptr;
   P.dq = static_cast<__nv_bfloat16*>(dq);
   P.ctl = ctl;
   P.out = nullptr;
@@ -1799,7 +1811,14 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     if (st == LS_OK) st = ls::pool_map(&P.bv_tail, h, 1, pbox, pgroups, true);
     if (st != LS_OK) return st;
     const int64_t grid1 = (int64_t)Hkv * (parts + 1) * rt.nq_tiles;
+    if (rt.nq_tiles == 1) P.dq_split = dq_acc + rows * D;      // (see ls_replay_attn_workspace_bytes)
     st = (D == 128) ? ls::launch_dq1<128>(P, grid1, cs) : ls::launch_dq1<256>(P, grid1, cs);
+    if (st == LS_OK && P.dq_split) {
+      const int64_t n4 = rows * D / 4;
+      ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 16), 256, 0, cs>>>(
+          P.dq_split, parts + 1, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
+      if (cudaGetLastError() != cudaSuccess) st = LS_ERR_CUDA;
+    }
   } else {
     const int64_t grid2 = (int64_t)Hkv * (parts + 1) * ((P.nq_tiles + 1) / 2) * 2;
     st = (D == 128) ? ls::launch_dq2<128>(P, grid2, cs) : ls::launch_dq3(P, grid2, cs);
