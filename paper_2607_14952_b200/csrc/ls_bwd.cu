@@ -1280,7 +1280,9 @@ static ls_status_t launch_kv(const BwdParams& prm, int grid, cudaStream_t st, bo
 // Chunks of 16 KB per CTA: K or V as (this CTA's 128 keys x 64 channels) for S / T, and K as
 // (64 keys x this CTA's 128 channels) for the accumulate.
 // ---------------------------------------------------------------------------------
-constexpr int kDq3Threads = 320;        // producer warp, MMA warp, 8 elementwise warps (2 threads per row)
+constexpr int kDq3Tpr = 4;                              // threads per row of the elementwise warps
+constexpr int kDq3Threads = 64 + 128 * kDq3Tpr;         // producer warp, MMA warp, 4 * kDq3Tpr elementwise warps
+constexpr int kDq3Cw = 64 / kDq3Tpr;                    // columns of every 64-key quarter one thread owns
 
 struct Dq3Cfg {
   static constexpr int D = 256;
@@ -1304,9 +1306,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   uint64_t* full = bars + 1;             // (even CTA) both halves of a chunk landed
   uint64_t* empty = full + C::RING;      // (each CTA) chunk consumed
   uint64_t* s_full = empty + C::RING;    // (each CTA) S in TMEM
-  uint64_t* s_read = s_full + 1;         // (even CTA) every row thread of both CTAs has pulled S: 16 warp arrivals
+  uint64_t* s_read = s_full + 1;         // (even CTA) every row thread of both CTAs has pulled S: one arrival per warp
   uint64_t* t_full = s_read + 1;         // (each CTA) T in TMEM
-  uint64_t* e_full = t_full + 1;         // [4] (even CTA) quarter of E in both CTAs' TMEM: 16 warp arrivals
+  uint64_t* e_full = t_full + 1;         // [4] (even CTA) quarter of E in both CTAs' TMEM: one arrival per warp
   uint64_t* acc_final = e_full + 4;      // (each CTA)
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
@@ -1327,9 +1329,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
       mbar_init(&empty[i], 1);
     }
     mbar_init(s_full, 1);
-    mbar_init(s_read, 16);
+    mbar_init(s_read, 8 * kDq3Tpr);
     mbar_init(t_full, 1);
-    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 16);
+    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 8 * kDq3Tpr);
     mbar_init(acc_final, 1);
     *abort_flag = 0;
     // work items are handed out in launch order of the pairs that ask (see chain_wait)
@@ -1528,7 +1530,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   } else {
     // =========================================================== elementwise + epilogue (both CTAs)
     const int quad = warp & 3;
-    const int sub = (warp - 2) >> 2;                // which 32 of every 64-column quarter this thread owns (2 threads per row)
+    const int sub = (warp - 2) >> 2;                // which kDq3Cw columns of every 64-key quarter this thread owns
+    constexpr int CW = kDq3Cw;
+    constexpr int NT = 128 * kDq3Tpr;               // elementwise threads of the CTA
     const int row = quad * 32 + lane;
     const int hj = row / p.bt;                      // head and token of this row of the tile
     const int r_idx = row0 + row - hj * p.bt;
@@ -1550,26 +1554,26 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
         const int key0 = i * 256;
         const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 255 > lim);
         // No thread leaves this loop on its own: a wait that gave up is remembered in `ok` and put
-        // to the vote at the first named barrier of the tile, where all 256 leave together.
+        // to the vote at the first named barrier of the tile, where all leave together.
         ok = ok && LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
         tc_fence_after();
-        // p = exp(s - LSE) for this thread's 4 x 32 columns: all four TMEM loads in flight at once,
-        // p kept as packed bf16 pairs (64 registers) until T is ready
-        uint32_t sr[128];
+        // p = exp(s - LSE) for this thread's 4 x CW columns: all four TMEM loads in flight at once,
+        // p kept as packed bf16 pairs until T is ready
+        uint32_t sr[4 * CW];
 #pragma unroll
-        for (int qd = 0; qd < 4; ++qd) tmem_ld32(tmem_st + lane_sel + 64 * qd + 32 * sub, sr + 32 * qd);
+        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_st + lane_sel + 64 * qd + CW * sub, sr + CW * qd);
 #pragma unroll
-        for (int qd = 0; qd < 4; ++qd) tc_wait_ld32(sr + 32 * qd);
+        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(sr + CW * qd);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(s_read_remote);    // this warp no longer needs S: T may overwrite it
-        uint32_t pp[64];
+        uint32_t pp[2 * CW];
 #pragma unroll
-        for (int j = 0; j < 128; j += 2) {
+        for (int j = 0; j < 4 * CW; j += 2) {
           float e0 = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
           float e1 = ex2(fmaf(__uint_as_float(sr[j + 1]), p.scale_log2, -lse2_row));
           if (edge) {
-            const int64_t col = (int64_t)key0 + 64 * (j >> 5) + 32 * sub + (j & 31);
+            const int64_t col = (int64_t)key0 + 64 * (j / CW) + CW * sub + (j % CW);
             if (col > lim) e0 = 0.f;
             if (col + 1 > lim) e1 = 0.f;
           }
@@ -1577,28 +1581,28 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
         }
         ok = ok && LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
         tc_fence_after();
-        uint32_t tr[2][32];
-        tmem_ld32(tmem_st + lane_sel + 32 * sub, tr[0]);
+        uint32_t tr[2][CW];
+        tmem_ld16(tmem_st + lane_sel + CW * sub, tr[0]);
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-          tc_wait_ld32(tr[qd & 1]);
-          if (qd < 3) tmem_ld32(tmem_st + lane_sel + 64 * (qd + 1) + 32 * sub, tr[(qd + 1) & 1]);   // in flight meanwhile
-          uint32_t pk[16];
+          tc_wait_ld16(tr[qd & 1]);
+          if (qd < 3) tmem_ld16(tmem_st + lane_sel + 64 * (qd + 1) + CW * sub, tr[(qd + 1) & 1]);   // in flight meanwhile
+          uint32_t pk[CW / 2];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const uint32_t pw = pp[16 * qd + (j >> 1)];
+          for (int j = 0; j < CW; j += 2) {
+            const uint32_t pw = pp[(CW / 2) * qd + (j >> 1)];
             pk[j >> 1] = pack_bf16(__uint_as_float(pw << 16) * (__uint_as_float(tr[qd & 1][j]) - delta_row),
                                    __uint_as_float(pw & 0xffff0000u) * (__uint_as_float(tr[qd & 1][j + 1]) - delta_row));
           }
           // E (bf16 pairs) of quarter q goes to columns [32 q, 32 q + 32) of the buffer: T columns that
-          // this quarter or an earlier one has read -- by either thread of the row, hence the barrier
+          // this quarter or an earlier one has read -- by any thread of the row, hence the barrier
           if (qd == 0) {
-            ok = bar_and(1, 256, ok);
+            ok = bar_and(1, NT, ok);
             if (!ok) break;
           } else {
-            bar_sync(1, 256);
+            bar_sync(1, NT);
           }
-          tmem_st16(tmem_st + lane_sel + 32 * qd + 16 * sub, pk);
+          tmem_st8(tmem_st + lane_sel + 32 * qd + (CW / 2) * sub, pk);
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
@@ -1620,9 +1624,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
     if (tile_ok) {
       if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
       if (ok)
-        dq_store_row<D / 2>(tmem_acc + lane_sel + sub * (D / 2), n_tiles > 0, fold, last, p.scale,
-                            p.dq_acc + ri * D + sub * (D / 2), p.dq + ri * D + sub * (D / 2), row_ok);
-      const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
+        dq_store_row<D / kDq3Tpr>(tmem_acc + lane_sel + sub * (D / kDq3Tpr), n_tiles > 0, fold, last, p.scale,
+                                  p.dq_acc + ri * D + sub * (D / kDq3Tpr), p.dq + ri * D + sub * (D / kDq3Tpr), row_ok);
+      const bool all_ok = bar_and(2, 128 * kDq3Tpr, ok);     // every row of the tile is written
       if (row == 0 && sub == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
