@@ -86,7 +86,10 @@ struct MlaDqParams {
 #define LS_TQABLATE(bit) false
 #endif
 
-constexpr int kTqThreads = 256;   // K-major producer, [S^T|T^T] issuer, 4 warps of key threads, dQ^T issuer, MN-major producer
+constexpr int kTqKt = 2;                        // threads per key: each forms E^T for 64 / kTqKt of the rows
+// warps: 0 K-major producer, 1 [S^T|T^T] issuer, 2 dQ^T issuer, 3 MN-major producer, then 4 * kTqKt warps of key threads
+constexpr int kTqThreads = 128 + 128 * kTqKt;
+static_assert(kTqKt == 2, "a key thread's rows are one CTA's half of E^T");
 constexpr int kTqSlab = 16384;                 // 128 keys x 128 B
 constexpr int kTqStSlots = 3;                  // ring slots of 16 KB: [S^T | T^T] slabs
 constexpr int kTqAccSlots = 4;                 //                      dQ^T slots
@@ -163,10 +166,10 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&st_full[i], 1);
-      mbar_init(&s_read[i], 8);
+      mbar_init(&s_read[i], 8 * kTqKt);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&e_full[i], 8);
+      mbar_init(&e_full[i], 8 * kTqKt);
       mbar_init(&e_free[i], 1);
     }
     mbar_init(acc_final, 1);
@@ -190,13 +193,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
   const uint32_t tmem_st = tmem_base;           // two buffers of S^T [0,64) | T^T [64,128) of this CTA's 128 keys
   const uint32_t tmem_acc = tmem_base + 256;    // 3 x 64 columns: this CTA's 128 channels of each block
 
-  if (warp == 0 || warp == 7) {
+  if (warp == 0 || warp == 3) {
     // =========================================================== producers (two threads per CTA)
     // Two rings, one producer thread each (a single thread issues a TMA instruction every ~200
     // cycles, too slow for both): slots [0, kTqStSlots) carry K-major slabs (this CTA's 128 keys x
     // one channel group, two 64-token boxes) for [S^T | T^T], filled by warp 0; the rest carry
     // MN-major slots (64 keys of either CTA's tile x two of THIS CTA's channel groups, one box) for
-    // dQ^T, filled by warp 7.  Every load credits the even CTA's barrier of the slot.
+    // dQ^T, filled by warp 3.  Every load credits the even CTA's barrier of the slot.
     if (lane == 0 && total_steps > 0) {
       const bool st_role = warp == 0;
       if (st_role) {
@@ -345,7 +348,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
       LS_TQDUMP(10, tw2);
       LS_TQDUMP(12, clock64() - t_begin);
     }
-  } else if (warp == 6) {
+  } else if (warp == 2) {
     // =========================================================== dQ^T issuer (one thread of the even CTA)
     if (leader && lane == 0 && total_steps > 0) {
       constexpr uint32_t idesc_acc = make_idesc(256, 64, 1, 1);
@@ -384,14 +387,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
       LS_TQDUMP(13, clock64() - t_begin);
     }
   } else {
-    // =========================================================== one thread per key: E^T, epilogue
+    // =========================================================== two threads per key: E^T, epilogue
+    // (thread `sub` of a key owns rows 32 sub .. 32 sub + 31, i.e. the half of E^T that lives in CTA `sub`;
+    // with one thread per key -- one warp per scheduler -- these warps were busy 83 % of a step on TMEM-load,
+    // MUFU and store latency that nothing overlapped)
     const int quad = warp & 3;
+    const int sub = (warp - 4) >> 2;
     const int key = quad * 32 + lane;                      // TMEM lane = key of this CTA's tile
     const uint32_t lane_sel = (uint32_t)(quad * 32) << 16;
     // E^T of this CTA's keys, MN-major [key][row] in 64-byte lines (64-byte swizzle): rows 0-31 go
     // to the even CTA's copy, rows 32-63 to the odd CTA's, each at offset rank * 8 KB of the E^T area
     const uint32_t e_mine = smem_u32(e_smem) + rank * 8192 + (key >> 3) * 512 + (key & 7) * 64;
-    const uint32_t e_dst[2] = {mapa_u32(e_mine, 0), mapa_u32(e_mine, 1)};
+    const uint32_t e_dst = mapa_u32(e_mine, (uint32_t)sub);
     const uint32_t sw = (uint32_t)(key & 7) >> 1;
     const uint32_t s_read_remote[2] = {mapa_u32(smem_u32(&s_read[0]), 0), mapa_u32(smem_u32(&s_read[1]), 0)};
     const uint32_t e_full_remote[2] = {mapa_u32(smem_u32(&e_full[0]), 0), mapa_u32(smem_u32(&e_full[1]), 0)};
@@ -411,31 +418,27 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
         if (!ok) break;
         tc_fence_after();
         const uint32_t tst = tmem_st + (i & 1) * 128 + lane_sel;
-        uint32_t pk[32];
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
+        uint32_t pk[16];
+        {
           uint32_t sr[32], tr[32];
-          tmem_ld32(tst + half * 32, sr);
-          tmem_ld32(tst + 64 + half * 32, tr);
+          tmem_ld32(tst + sub * 32, sr);
+          tmem_ld32(tst + 64 + sub * 32, tr);
           tc_wait_ld32(sr);
           tc_wait_ld32(tr);
-          if (half == 1) {          // the whole buffer is in registers: the next step may overwrite it
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(s_read_remote[i & 1]);
-          }
+          tc_fence_before();        // this warp's share of the buffer is in registers: the next step may overwrite it
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(s_read_remote[i & 1]);
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
-            const float4 rp = *reinterpret_cast<const float4*>(rowp + half * 32 + j);   // two rows
+            const float4 rp = *reinterpret_cast<const float4*>(rowp + sub * 32 + j);   // two rows
             const float p0 = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -rp.x));
             const float p1 = ex2(fmaf(__uint_as_float(sr[j + 1]), p.scale_log2, -rp.z));
-            pk[half * 16 + (j >> 1)] =
-                pack_bf16(p0 * (__uint_as_float(tr[j]) - rp.y), p1 * (__uint_as_float(tr[j + 1]) - rp.w));
+            pk[j >> 1] = pack_bf16(p0 * (__uint_as_float(tr[j]) - rp.y), p1 * (__uint_as_float(tr[j + 1]) - rp.w));
           }
         }
         if (!valid) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) pk[j] = 0u;
+          for (int j = 0; j < 16; ++j) pk[j] = 0u;
         }
         if (i > 1) {      // the dQ^T instructions of step i - 2 have read this E^T buffer
           ok = LS_TQWAIT(tw1, mbar_wait(&e_free[i & 1], ((i >> 1) - 1) & 1, abort_flag));
@@ -443,16 +446,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
           if (!ok) break;
         }
 #pragma unroll
-        for (int c = 0; c < 2; ++c)          // destination CTA = half of the rows
-#pragma unroll
-          for (int q = 0; q < 4; ++q)        // 16-byte chunk: rows 32 c + 8 q .. + 7
-            st_shared_cluster_v4(e_dst[c] + (i & 1) * kTqE + (((uint32_t)q ^ sw) << 4), pk[16 * c + 4 * q], pk[16 * c + 4 * q + 1],
-                                 pk[16 * c + 4 * q + 2], pk[16 * c + 4 * q + 3]);
+        for (int q = 0; q < 4; ++q)          // 16-byte chunk: rows 32 sub + 8 q .. + 7, in CTA `sub`
+          st_shared_cluster_v4(e_dst + (i & 1) * kTqE + (((uint32_t)q ^ sw) << 4), pk[4 * q], pk[4 * q + 1], pk[4 * q + 2],
+                               pk[4 * q + 3]);
         fence_proxy_async_all();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster_release(e_full_remote[i & 1]);
       }
-      if (threadIdx.x == 64) {
+      if (threadIdx.x == 128) {
         LS_TQDUMP(16, tw0);
         LS_TQDUMP(17, tw1);
         LS_TQDUMP(18, clock64() - t_begin);
@@ -477,8 +478,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
       for (int m = 0; m < 3; ++m) {
         if (m == 2 && (!leader || quad >= 2)) break;      // block 2 is the 64 rope channels, in the even CTA
         const int ch = m * 256 + (int)rank * 128 + key;
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
+        {
+          const int half = sub;             // this thread's 32 of the 64 rows
           uint32_t o[32];
           if (have_acc) {
             tmem_ld32(tmem_acc + lane_sel + m * 64 + half * 32, o);
@@ -513,8 +514,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kTqThreads, 1)
       }
     }
     if (p.chain) {
-      const bool all_ok = bar_and(1, 128, key_ok);      // every row of this CTA's channels is written
-      if (key == 0 && all_ok) chain_publish_add(counter);
+      const bool all_ok = bar_and(1, 128 * kTqKt, key_ok);      // every row of this CTA's channels is written
+      if (key == 0 && sub == 0 && all_ok) chain_publish_add(counter);
     }
   }
 
