@@ -82,6 +82,7 @@ struct BwdParams {
 #endif
 
 constexpr int kBwdThreads = 320;        // producer warp, MMA warp, 8 elementwise warps (2 threads per row)
+constexpr int kDq1Threads = 576;        // single-CTA dQ kernel: 16 elementwise warps (4 threads per row)
 constexpr int kBwdChunk = 32768;        // 128 columns x 128 channels
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -904,7 +905,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
 // TMEM: ACC [0, D), S [D, D+128), T [D+128, D+256).  Chunks of 32 KB: 128 keys x 128 channels.
 // ---------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_constant__ BwdParams p) {
+__global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_constant__ BwdParams p) {
   using C = BwdCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -933,9 +934,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
       mbar_init(&empty[i], 1);
     }
     mbar_init(s_full, 1);
-    mbar_init(s_read, 256);
+    mbar_init(s_read, 512);
     mbar_init(t_full, 1);
-    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 256);
+    for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 128);
     mbar_init(acc_final, 1);
     *abort_flag = 0;
     *work_idx = atomicAdd(p.ctl, 1);      // work items in launch order of the CTAs that ask (see chain_wait)
@@ -1121,7 +1122,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
   } else {
     // =========================================================== elementwise + epilogue
     const int quad = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int sub = (warp - 2) >> 2;                       // four threads per row: thread `sub` owns the 32-key quarter `sub`
     const int row = quad * 32 + lane;
     const int hj = row / p.bt;                            // head and token of this row of the tile
     const int r_tok = t0 + row - hj * p.bt;
@@ -1139,46 +1140,39 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
         const int key0 = i * 128;
         const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim);
         // No thread leaves this loop on its own: a wait that gave up is remembered in `ok` and put
-        // to the vote at the tile's named barrier, where all 256 leave together.
+        // to the vote at the tile's named barrier, where all 512 leave together.
         ok = ok && mbar_wait(s_full, i & 1, abort_flag);
         tc_fence_after();
-        uint32_t sr[64];
-#pragma unroll
-        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_s + lane_sel + 32 * qd + 16 * half, sr + 16 * qd);
-#pragma unroll
-        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(sr + 16 * qd);
+        uint32_t sr[32];
+        tmem_ld32(tmem_s + lane_sel + 32 * sub, sr);
+        tc_wait_ld32(sr);
         tc_fence_before();
         mbar_arrive(s_read);                 // S is in registers: the next tile's S may overwrite the buffer
-        float pr[64];
+        float pr[32];
 #pragma unroll
-        for (int j = 0; j < 64; ++j) {
+        for (int j = 0; j < 32; ++j) {
           float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
-          if (edge && (int64_t)key0 + 32 * (j >> 4) + 16 * half + (j & 15) > lim) e = 0.f;
+          if (edge && (int64_t)key0 + 32 * sub + j > lim) e = 0.f;
           pr[j] = e;
         }
         ok = ok && mbar_wait(t_full, i & 1, abort_flag);
         tc_fence_after();
-        uint32_t tr[64];
-#pragma unroll
-        for (int qd = 0; qd < 4; ++qd) tmem_ld16(tmem_t + lane_sel + 32 * qd + 16 * half, tr + 16 * qd);
-#pragma unroll
-        for (int qd = 0; qd < 4; ++qd) tc_wait_ld16(tr + 16 * qd);
-        // E (bf16) goes over T's columns, which the row's other thread reads too: every T read of the
+        uint32_t tr[32];
+        tmem_ld32(tmem_t + lane_sel + 32 * sub, tr);
+        tc_wait_ld32(tr);
+        // E (bf16) goes over T's columns, which the row's other threads read too: every T read of the
         // CTA comes before any E write (named barrier 1, which also carries the vote)
-        ok = bar_and(1, 256, ok);
+        ok = bar_and(1, 512, ok);
         if (!ok) break;
+        uint32_t pk[16];
 #pragma unroll
-        for (int qd = 0; qd < 4; ++qd) {
-          uint32_t pk[8];
-#pragma unroll
-          for (int j = 0; j < 16; j += 2)
-            pk[j >> 1] = pack_bf16(pr[16 * qd + j] * (__uint_as_float(tr[16 * qd + j]) - delta_row),
-                                   pr[16 * qd + j + 1] * (__uint_as_float(tr[16 * qd + j + 1]) - delta_row));
-          tmem_st8(tmem_t + lane_sel + 16 * qd + 8 * half, pk);
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(&e_full[qd]);
-        }
+        for (int j = 0; j < 32; j += 2)
+          pk[j >> 1] = pack_bf16(pr[j] * (__uint_as_float(tr[j]) - delta_row),
+                                 pr[j + 1] * (__uint_as_float(tr[j + 1]) - delta_row));
+        tmem_st16(tmem_t + lane_sel + 16 * sub, pk);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(&e_full[sub]);
       }
       ok = __all_sync(0xffffffffu, ok);
       if (ok) ok = bwd_wait_warp(acc_final, 0, abort_flag);
@@ -1188,17 +1182,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_dq1_kernel(const __grid_co
     // running dQ of the tile's rows, in link order
     if (p.dq_split) {
       if (ok)
-        dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, false, false, p.scale,
-                            p.dq_split + ((size_t)it.link * p.R * p.Hq + ri) * D + half * (D / 2), nullptr, row_ok);
+        dq_store_row<D / 4>(tmem_acc + lane_sel + sub * (D / 4), n_tiles > 0, false, false, p.scale,
+                            p.dq_split + ((size_t)it.link * p.R * p.Hq + ri) * D + sub * (D / 4), nullptr, row_ok);
     } else {
       const bool fold = it.link > 0, last = it.link == p.parts;
       int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + qtile;
       if (ok && fold) ok = __all_sync(0xffffffffu, chain_wait(counter, it.link, p.ctl, abort_flag));
       if (ok)
-        dq_store_row<D / 2>(tmem_acc + lane_sel + half * (D / 2), n_tiles > 0, fold, last, p.scale,
-                            p.dq_acc + ri * D + half * (D / 2), p.dq + ri * D + half * (D / 2), row_ok);
-      const bool all_ok = bar_and(2, 256, ok);     // every row of the tile is written
-      if (row == 0 && half == 0 && all_ok) chain_publish(counter, it.link + 1);
+        dq_store_row<D / 4>(tmem_acc + lane_sel + sub * (D / 4), n_tiles > 0, fold, last, p.scale,
+                            p.dq_acc + ri * D + sub * (D / 4), p.dq + ri * D + sub * (D / 4), row_ok);
+      const bool all_ok = bar_and(2, 512, ok);     // every row of the tile is written
+      if (row == 0 && sub == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
 
@@ -1652,7 +1646,7 @@ static ls_status_t launch_dq1(const BwdParams& prm, int64_t grid, cudaStream_t s
   const ls_status_t cs = configure_smem(bwd_dq1_kernel<D>, C::SMEM_BYTES, configured);
   if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_BWD_DQ, st);
-  bwd_dq1_kernel<D><<<(int)grid, kBwdThreads, C::SMEM_BYTES, st>>>(prm);
+  bwd_dq1_kernel<D><<<(int)grid, kDq1Threads, C::SMEM_BYTES, st>>>(prm);
   profile_end(LS_KERNEL_BWD_DQ, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
