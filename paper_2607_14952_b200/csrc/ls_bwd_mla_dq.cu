@@ -11,8 +11,8 @@
 //        TMEM, each for its own keys;
 //   S^T += K_8 x Q_8^T  (rope channels, N = 64: each CTA contributes 32 rows of Q_8, of which both
 //        hold a copy);
-//   E^T  = p (T^T - Delta) : one thread per key.  dQ^T is split along the channels (M) between the
-//        CTAs, and its B operand E^T along the rows (N): a thread writes rows 0-31 of its key into
+//   E^T  = p (T^T - Delta) : two threads per key, 32 rows each.  dQ^T is split along the channels
+//        (M) between the CTAs, and its B operand E^T along the rows (N): rows 0-31 of a key go into
 //        the even CTA's shared memory and rows 32-63 into the odd CTA's (st.shared::cluster), as
 //        bf16 in MN-major 64-byte lines;
 //   dQ^T (this CTA's 128 of 256 channels x 64 rows) += K^T (MN-major, 16 keys) x E^T, for the keys
