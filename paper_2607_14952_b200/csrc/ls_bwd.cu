@@ -62,10 +62,14 @@ struct BwdParams {
   int R, Hq, Hkv, g, parts, pg_shift, tiles_per_head, nq_tiles, num_phys_pages;
   // dQ pass of a short response (single-CTA kernel): Q tiles of bt tokens x bh heads (RowTiling)
   int bt, bh, tiles_tok;
-  // single-CTA dQ kernel, one tile per KV group: every part writes its fp32 sum to dq_split
-  // [parts + 1, R, Hq, D] and a reduce kernel adds them (a chain of parts + 1 links per KV group would
-  // run its folds one after the other at the end of a launch in which all parts finish together)
+  // single-CTA dQ kernel, one tile per KV group: the key tiles of a KV head are cut into dq1_ranges equal
+  // ranges, one CTA each; every CTA writes its fp32 sum to dq_split [dq1_ranges, R, Hq, D] and a reduce
+  // kernel adds them (a chain of links per KV group would run its folds one after the other at the end
+  // of a launch in which all CTAs finish together)
   float* dq_split;
+  int a_slab_bytes;   // single-CTA dQ kernel: bytes of one 64-channel group of the tile's Q (dO) rows
+  int dq1_ring;       // ... and the number of 32 KB ring slots that fit beside them
+  int dq1_ranges;     // ... with dq_split: CTAs (= partials) per KV head
   int no_resp;   // dQ pass: the response block is left out
   // dK / dV pass: keys of a suffix block (1) read through pages [key_page_off, ..) of part_pages,
   // key_tokens of them, first gradient slot grad_slot0; or the response block (0)
@@ -897,39 +901,81 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kBwdThreads, 1)
 
 
 // ---------------------------------------------------------------------------------
-// dQ pass for short responses (g * R <= 128): every (head, token) row of a KV group sits in ONE
-// Q tile, so a (KV head, part) is one work item and its K/V pages are read once: the pass is
-// bound by HBM, not by the tensor pipe.  A single CTA per item (a pair would spend half of every
-// 256-row MMA on rows that do not exist), 128-key tiles, E written over T so that the tensor pipe
-// runs S(i+1) while the row threads form E(i):   S(0) T(0) | S(i+1)  ACC(i)  T(i+1) | ...
+// dQ pass for short responses: the rows of a Q tile (bt tokens x bh heads of one KV group) stay in
+// shared memory and the keys stream past once, so the pass is bound by HBM, not by the tensor pipe.
+// A single CTA per work item (a pair would spend half of every 256-row MMA on rows that do not
+// exist), 128-key tiles, E written over T so that the tensor pipe runs S(i+1) while the row threads
+// form E(i):   S(0) T(0) | S(i+1)  ACC(i)  T(i+1) | ...
 // TMEM: ACC [0, D), S [D, D+128), T [D+128, D+256).  Chunks of 32 KB: 128 keys x 128 channels.
+//
+// Work.  A KV group of several tiles: one item per (KV head, link, tile), the links of a tile summed
+// through the running dQ in link order.  A KV group of ONE tile (p.dq_split): the key tiles of all
+// links of a KV head, laid end to end, are cut into p.dq1_ranges equal ranges, one CTA each (a range
+// may cross link boundaries); every CTA writes one fp32 partial and a reduce kernel adds them.  With
+// one item per (KV head, part) the 4 x 65 items of the 2M prefix ran as two waves on 148 SMs.
 // ---------------------------------------------------------------------------------
+struct Dq1Cursor {      // a position in the CTA's list of key tiles
+  int link, i, n;       // link (0 = response block, 1.. = parts), tile of the link, tiles of the link
+  int left;             // tiles of the list from here on, this one included
+  bool is_resp;
+  int64_t tokens;
+  int page_off, n_pages, tail_slot;
+};
+__device__ __forceinline__ void dq1_link(const BwdParams& p, int resp_tokens, Dq1Cursor& c) {
+  c.is_resp = c.link == 0;
+  if (c.is_resp) {
+    c.tokens = resp_tokens;
+    c.page_off = c.n_pages = 0;
+    c.tail_slot = -1;
+  } else {
+    const int part = c.link - 1;
+    c.tokens = p.part_tokens[part];
+    c.page_off = p.part_page_offset[part];
+    c.n_pages = p.part_page_offset[part + 1] - c.page_off;
+    c.tail_slot = p.part_tail_slot[part];
+  }
+  c.n = (int)((c.tokens + 127) / 128);
+}
+__device__ __forceinline__ void dq1_next(const BwdParams& p, int resp_tokens, Dq1Cursor& c) {
+  if (--c.left <= 0) return;
+  ++c.i;
+  while (c.i >= c.n && c.link < p.parts) {     // left > 0: a later link holds the tile
+    ++c.link;
+    dq1_link(p, resp_tokens, c);
+    c.i = 0;
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_constant__ BwdParams p) {
   using C = BwdCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // Q and dO keep only the rows of the tile (padded to 8): the 128-row MMAs read on into whatever
+  // follows, which yields rows nobody stores; the ring gets the shared memory this frees
+  const uint32_t slab = (uint32_t)p.a_slab_bytes;     // one 64-channel group of the resident rows
+  const uint32_t nring = (uint32_t)p.dq1_ring;
   uint8_t* a1_smem = smem;
-  uint8_t* a2_smem = smem + C::SLABS * 16384;
-  uint8_t* ring = smem + C::A_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + C::RING * kBwdChunk);
+  uint8_t* a2_smem = smem + C::SLABS * slab;
+  uint8_t* ring = smem + 2 * C::SLABS * slab;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ring + nring * kBwdChunk);
   uint64_t* a_full = bars;
   uint64_t* full = bars + 1;
-  uint64_t* empty = full + C::RING;
-  uint64_t* s_full = empty + C::RING;    // S of a tile is in TMEM
+  uint64_t* empty = full + nring;
+  uint64_t* s_full = empty + nring;      // S of a tile is in TMEM
   uint64_t* s_read = s_full + 1;         // every row thread has pulled S
   uint64_t* t_full = s_read + 1;         // T of a tile is in TMEM
   uint64_t* e_full = t_full + 1;         // [4] quarter q of E is in TMEM
   uint64_t* acc_final = e_full + 4;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(acc_final + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
-  int* work_idx = const_cast<int*>(abort_flag) + 1;
+  int* work = const_cast<int*>(abort_flag) + 1;      // [4] ticket, first link, first tile, tiles of the list
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     mbar_init(a_full, 1);
-    for (int i = 0; i < C::RING; ++i) {
+    for (uint32_t i = 0; i < nring; ++i) {
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], 1);
     }
@@ -939,7 +985,29 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
     for (int i = 0; i < 4; ++i) mbar_init(&e_full[i], 128);
     mbar_init(acc_final, 1);
     *abort_flag = 0;
-    *work_idx = atomicAdd(p.ctl, 1);      // work items in launch order of the CTAs that ask (see chain_wait)
+    const int widx = atomicAdd(p.ctl, 1);      // work items in launch order of the CTAs that ask (see chain_wait)
+    work[0] = widx;
+    if (p.dq_split) {
+      // range widx % dq1_ranges of the KV head's key tiles, all links end to end
+      const int resp_tokens = p.no_resp ? 0 : min(p.R, p.bt);
+      auto tiles_of = [&](int link) -> int64_t {
+        return ((link == 0 ? (int64_t)resp_tokens : p.part_tokens[link - 1]) + 127) / 128;
+      };
+      int64_t total = 0;
+      for (int link = 0; link <= p.parts; ++link) total += tiles_of(link);
+      const int c = widx % p.dq1_ranges;
+      const int64_t v0 = total * c / p.dq1_ranges, v1 = total * (c + 1) / p.dq1_ranges;
+      int link = 0;
+      int64_t v = 0;
+      for (; link < p.parts; ++link) {
+        const int64_t n = tiles_of(link);
+        if (v0 < v + n) break;
+        v += n;
+      }
+      work[1] = link;
+      work[2] = (int)(v0 - v);
+      work[3] = (int)(v1 - v0);
+    }
     fence_barrier_init();
   }
   if (warp == 1) {
@@ -954,59 +1022,80 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
   const uint32_t tmem_s = tmem_base + D;
   const uint32_t tmem_t = tmem_base + D + 128;
 
-  // ---- work item: (KV head, link, Q tile of bt tokens x bh heads of the KV group)
-  const DqItem it = dq_item(p, *work_idx, p.nq_tiles);
-  const int part = it.part, kvh = it.kvh, qtile = it.pairi;
-  const bool is_resp = it.is_resp;
+  // ---- the CTA's rows (KV head, Q tile of bt tokens x bh heads of the KV group) and its list of key tiles
+  DqItem it{};
+  int range = 0;
+  if (p.dq_split) {
+    range = work[0] % p.dq1_ranges;
+    it.kvh = work[0] / p.dq1_ranges;
+    it.pairi = 0;
+    it.link = work[1];
+  } else {
+    it = dq_item(p, work[0], p.nq_tiles);
+  }
+  const int kvh = it.kvh, qtile = it.pairi;
   const int h = kvh * p.g + (qtile / p.tiles_tok) * p.bh;
   const int t0 = (qtile % p.tiles_tok) * p.bt;
-  int64_t tokens;
-  int page_off = 0, n_pages = 0, tail_slot = -1;
-  if (is_resp) {
-    tokens = p.no_resp ? 0 : min(p.R, t0 + p.bt);
-  } else {
-    tokens = p.part_tokens[part];
-    page_off = p.part_page_offset[part];
-    n_pages = p.part_page_offset[part + 1] - page_off;
-    tail_slot = p.part_tail_slot[part];
-  }
-  const int n_tiles = (int)((tokens + 127) / 128);
+  const int resp_tokens = p.no_resp ? 0 : min(p.R, t0 + p.bt);
+  Dq1Cursor first;
+  first.link = it.link;
+  dq1_link(p, resp_tokens, first);
+  first.i = p.dq_split ? work[2] : 0;
+  first.left = p.dq_split ? work[3] : first.n;
+  const int n_tiles = first.left;
+  [[maybe_unused]] const bool dump = p.dq_split ? work[0] == 0 : (it.link == 1 && kvh == 0 && qtile == 0);
+  [[maybe_unused]] long long tw0 = 0, tw1 = 0, tw2 = 0, tw3 = 0;
+  [[maybe_unused]] const long long t_kernel0 = clock64();
+#ifdef LS_TIMING
+#define LS_D1DUMP(slot, val) do { if (p.timing && dump) p.timing[(slot)] = (val); } while (0)
+#else
+#define LS_D1DUMP(slot, val) do { } while (0)
+#endif
 
   if (warp == 0) {
     // =========================================================== producer (one thread)
     if (lane == 0 && n_tiles > 0) {
       mbar_arrive_expect_tx(a_full, 2 * C::SLABS * p.bt * p.bh * 128);
       for (int c = 0; c < C::SLABS; ++c) {
-        tma_load_5d(a1_smem + c * 16384, &p.a1_map, a_full, 0, t0, c, h, 0);
-        tma_load_5d(a2_smem + c * 16384, &p.a2_map, a_full, 0, t0, c, h, 0);
+        tma_load_5d(a1_smem + c * slab, &p.a1_map, a_full, 0, t0, c, h, 0);
+        tma_load_5d(a2_smem + c * slab, &p.a2_map, a_full, 0, t0, c, h, 0);
       }
-      const int32_t* pages = p.part_pages + page_off;
       const int pg_mask = (1 << p.pg_shift) - 1;
-      const bool small_pages = !is_resp && p.pg_shift == 6;   // a 128-key tile spans two 64-token pages
-      auto fetch = [&](int ps) -> int {
-        if (is_resp) return 0;
-        return (ps < n_pages) ? __ldg(pages + ps) : p.num_phys_pages;   // past the end: TMA fills zeros
+      const bool pages64 = p.pg_shift == 6;      // a 128-key tile of a paged link spans two 64-token pages
+      const int sh = pages64 ? 0 : (p.pg_shift - 7);
+      // physical pages under a tile (past the end of the link: TMA fills zeros)
+      auto pages_of = [&](const Dq1Cursor& cu, int& pa, int& pb) {
+        pa = pb = 0;
+        if (cu.left <= 0 || cu.is_resp) return;
+        const int32_t* pages = p.part_pages + cu.page_off;
+        if (pages64) {
+          pa = (2 * cu.i < cu.n_pages) ? __ldg(pages + 2 * cu.i) : p.num_phys_pages;
+          pb = (2 * cu.i + 1 < cu.n_pages) ? __ldg(pages + 2 * cu.i + 1) : p.num_phys_pages;
+        } else {
+          pa = pb = ((cu.i >> sh) < cu.n_pages) ? __ldg(pages + (cu.i >> sh)) : p.num_phys_pages;
+        }
       };
       uint32_t slot = 0, phase = 0, issued = 0;
       bool ok = true;
       // one chunk: 128 keys x channels [128 c, 128 c + 128) of K (which = 0) or V (1)
-      auto load = [&](int which, int i, int c, int pa, int pb) {
-        ok = ok && mbar_wait(&empty[slot], phase ^ 1, abort_flag);
+      auto load = [&](int which, const Dq1Cursor& cu, int c, int pa, int pb) {
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(&empty[slot], phase ^ 1, abort_flag));
         if (ok) {
           mbar_arrive_expect_tx(&full[slot], kBwdChunk);
           uint8_t* dst = ring + slot * kBwdChunk;
-          const int tok = i * 128;
-          if (is_resp) {
+          const int tok = cu.i * 128;
+          if (cu.is_resp) {
             tma_load_5d(dst, which ? &p.b2r_map : &p.b1r_map, &full[slot], 0, tok, 2 * c, kvh, 0);
-          } else if (!small_pages) {
-            const bool tail = (tok >> p.pg_shift) == tail_slot;
+          } else if (!pages64) {
+            const bool tail = (tok >> p.pg_shift) == cu.tail_slot;
             const CUtensorMap* m = which ? (tail ? &p.bv_tail : &p.bv_map) : (tail ? &p.bk_tail : &p.bk_map);
             tma_load_5d(dst, m, &full[slot], 0, tok & pg_mask, 2 * c, kvh, pa);
           } else {
             const int sa = tok >> 6;
-            const CUtensorMap* ma = which ? (sa == tail_slot ? &p.bv_tail : &p.bv_map) : (sa == tail_slot ? &p.bk_tail : &p.bk_map);
-            const CUtensorMap* mb = which ? (sa + 1 == tail_slot ? &p.bv_tail : &p.bv_map)
-                                          : (sa + 1 == tail_slot ? &p.bk_tail : &p.bk_map);
+            const CUtensorMap* ma = which ? (sa == cu.tail_slot ? &p.bv_tail : &p.bv_map)
+                                          : (sa == cu.tail_slot ? &p.bk_tail : &p.bk_map);
+            const CUtensorMap* mb = which ? (sa + 1 == cu.tail_slot ? &p.bv_tail : &p.bv_map)
+                                          : (sa + 1 == cu.tail_slot ? &p.bk_tail : &p.bk_map);
             for (int s2 = 0; s2 < 2; ++s2) {
               tma_load_5d(dst + s2 * 16384, ma, &full[slot], 0, 0, 2 * c + s2, kvh, pa);
               tma_load_5d(dst + s2 * 16384 + 8192, mb, &full[slot], 0, 0, 2 * c + s2, kvh, pb);
@@ -1014,30 +1103,39 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
           }
         }
         ++issued;
-        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+        if (++slot == nring) { slot = 0; phase ^= 1; }
       };
-      auto load_op = [&](int which, int i, int pa, int pb) {
-        for (int c = 0; c < C::NC; ++c) load(which, i, c, pa, pb);
+      auto load_op = [&](int which, const Dq1Cursor& cu, int pa, int pb) {
+        for (int c = 0; c < C::NC; ++c) load(which, cu, c, pa, pb);
       };
-      const int sh = small_pages ? 1 : (p.pg_shift - 7);
-      auto slot_of = [&](int i) { return small_pages ? 2 * i : (i >> sh); };
-      int pa0 = fetch(slot_of(0)), pb0 = small_pages ? fetch(1) : pa0;
-      int pa1 = fetch(slot_of(1)), pb1 = small_pages ? fetch(3) : pa1;
+      Dq1Cursor c0 = first, c1 = first;
+      dq1_next(p, resp_tokens, c1);
+      Dq1Cursor c2 = c1;
+      dq1_next(p, resp_tokens, c2);
+      int pa0, pb0, pa1, pb1;
+      pages_of(c0, pa0, pb0);
+      pages_of(c1, pa1, pb1);
       // chunk order = consumption order: S(0) T(0) [S(i+1) ACC(i) T(i+1)] ...; ACC re-reads K
-      load_op(0, 0, pa0, pb0);
-      load_op(1, 0, pa0, pb0);
+      load_op(0, c0, pa0, pb0);
+      load_op(1, c0, pa0, pb0);
       for (int i = 0; i < n_tiles; ++i) {
-        const int pa2 = fetch(slot_of(i + 2)), pb2 = small_pages ? fetch(2 * i + 5) : pa2;
-        if (i + 1 < n_tiles) load_op(0, i + 1, pa1, pb1);
-        load_op(0, i, pa0, pb0);
-        if (i + 1 < n_tiles) load_op(1, i + 1, pa1, pb1);
+        int pa2, pb2;
+        pages_of(c2, pa2, pb2);
+        if (i + 1 < n_tiles) load_op(0, c1, pa1, pb1);
+        load_op(0, c0, pa0, pb0);
+        if (i + 1 < n_tiles) load_op(1, c1, pa1, pb1);
+        c0 = c1; c1 = c2;
+        dq1_next(p, resp_tokens, c2);
         pa0 = pa1; pb0 = pb1; pa1 = pa2; pb1 = pb2;
       }
+      LS_D1DUMP(0, tw0);
+      LS_D1DUMP(1, clock64() - t_kernel0);
+      LS_D1DUMP(2, (long long)n_tiles);
       if (*abort_flag) {   // aborted: wait (bounded) for the copies already started
-        for (uint32_t s2 = 0; s2 < (uint32_t)C::RING && s2 < issued; ++s2) {
-          const uint32_t last = ((issued - 1 - s2) / C::RING) * C::RING + s2;
+        for (uint32_t s2 = 0; s2 < nring && s2 < issued; ++s2) {
+          const uint32_t last = ((issued - 1 - s2) / nring) * nring + s2;
           const uint64_t t_start = globaltimer_ns();
-          while (!mbar_try_wait(&full[s2], (last / C::RING) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
+          while (!mbar_try_wait(&full[s2], (last / nring) & 1, 1000) && globaltimer_ns() - t_start < 100000000ull) {
           }
         }
       }
@@ -1054,14 +1152,14 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
       uint32_t slot = 0, phase = 0;
       bool ok = mbar_wait(a_full, 0, abort_flag);
       auto advance = [&]() {
-        if (++slot == (uint32_t)C::RING) { slot = 0; phase ^= 1; }
+        if (++slot == nring) { slot = 0; phase ^= 1; }
       };
       auto issue_op = [&](int op) {       // S = Q K^T (0) or T = dO V^T (1)
         const uint32_t a_lo = op == 0 ? a1_lo : a2_lo;
         const uint32_t d = op == 0 ? tmem_s : tmem_t;
 #pragma unroll
         for (int c = 0; c < C::NC; ++c) {
-          ok = ok && mbar_wait(&full[slot], phase, abort_flag);
+          ok = ok && LS_BTWAIT(tw0, mbar_wait(&full[slot], phase, abort_flag));
           if (!ok) return;
           tc_fence_after();
           const uint32_t b_lo = ring_k_lo + slot * (kBwdChunk >> 4);
@@ -1069,7 +1167,7 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
           for (int s2 = 0; s2 < 2; ++s2)
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              mma_ss(d, sdesc(a_lo + (((2 * c + s2) * 16384 + k * 32) >> 4), hi),
+              mma_ss(d, sdesc(a_lo + (((2 * c + s2) * slab + k * 32) >> 4), hi),
                      sdesc(b_lo + ((s2 * 16384 + k * 32) >> 4), hi), idesc_st, (c | s2 | k) != 0);
           mma_commit(&empty[slot]);
           advance();
@@ -1086,13 +1184,13 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
         }
 #pragma unroll
         for (int qd = 0; qd < 4; ++qd) {
-          ok = ok && mbar_wait(&e_full[qd], i & 1, abort_flag);
+          ok = ok && LS_BTWAIT(tw1, mbar_wait(&e_full[qd], i & 1, abort_flag));
           if (!ok) return;
           tc_fence_after();
 #pragma unroll
           for (int c = 0; c < C::NC; ++c) {
             if (qd == 0) {
-              ok = ok && mbar_wait(&full[cs[c]], cph[c], abort_flag);
+              ok = ok && LS_BTWAIT(tw2, mbar_wait(&full[cs[c]], cph[c], abort_flag));
               if (!ok) return;
               tc_fence_after();
             }
@@ -1110,7 +1208,7 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
       if (ok) issue_op(1);
       for (int i = 0; i < n_tiles && ok; ++i) {
         if (i + 1 < n_tiles) {
-          ok = ok && mbar_wait(s_read, i & 1, abort_flag);
+          ok = ok && LS_BTWAIT(tw3, mbar_wait(s_read, i & 1, abort_flag));
           if (!ok) break;
           tc_fence_after();
           issue_op(0);
@@ -1118,6 +1216,11 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
         if (ok) issue_acc(i);
         if (ok && i + 1 < n_tiles) issue_op(1);
       }
+      LS_D1DUMP(8, tw0);
+      LS_D1DUMP(9, tw1);
+      LS_D1DUMP(10, tw2);
+      LS_D1DUMP(11, tw3);
+      LS_D1DUMP(12, clock64() - t_kernel0);
     }
   } else {
     // =========================================================== elementwise + epilogue
@@ -1135,13 +1238,14 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
     if (n_tiles > 0) {
       const float lse2_row = p.lse[ri] * kLog2e;
       const float delta_row = p.delta[ri];
-      const int64_t lim = is_resp ? (int64_t)r_idx : tokens - 1;
+      Dq1Cursor cu = first;
       for (int i = 0; i < n_tiles; ++i) {
-        const int key0 = i * 128;
-        const bool edge = __any_sync(0xffffffffu, (int64_t)key0 + 127 > lim);
+        const int64_t lim = cu.is_resp ? (int64_t)r_idx : cu.tokens - 1;
+        const int64_t key0 = (int64_t)cu.i * 128;
+        const bool edge = __any_sync(0xffffffffu, key0 + 127 > lim);
         // No thread leaves this loop on its own: a wait that gave up is remembered in `ok` and put
         // to the vote at the tile's named barrier, where all 512 leave together.
-        ok = ok && mbar_wait(s_full, i & 1, abort_flag);
+        ok = ok && LS_BTWAIT(tw0, mbar_wait(s_full, i & 1, abort_flag));
         tc_fence_after();
         uint32_t sr[32];
         tmem_ld32(tmem_s + lane_sel + 32 * sub, sr);
@@ -1152,17 +1256,17 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           float e = ex2(fmaf(__uint_as_float(sr[j]), p.scale_log2, -lse2_row));
-          if (edge && (int64_t)key0 + 32 * sub + j > lim) e = 0.f;
+          if (edge && key0 + 32 * sub + j > lim) e = 0.f;
           pr[j] = e;
         }
-        ok = ok && mbar_wait(t_full, i & 1, abort_flag);
+        ok = ok && LS_BTWAIT(tw1, mbar_wait(t_full, i & 1, abort_flag));
         tc_fence_after();
         uint32_t tr[32];
         tmem_ld32(tmem_t + lane_sel + 32 * sub, tr);
         tc_wait_ld32(tr);
         // E (bf16) goes over T's columns, which the row's other threads read too: every T read of the
         // CTA comes before any E write (named barrier 1, which also carries the vote)
-        ok = bar_and(1, 512, ok);
+        ok = LS_BTWAIT(tw2, bar_and(1, 512, ok));
         if (!ok) break;
         uint32_t pk[16];
 #pragma unroll
@@ -1173,17 +1277,24 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(&e_full[sub]);
+        dq1_next(p, resp_tokens, cu);
+      }
+      if (threadIdx.x == 64) {
+        LS_D1DUMP(16, tw0);
+        LS_D1DUMP(17, tw1);
+        LS_D1DUMP(18, tw2);
+        LS_D1DUMP(19, clock64() - t_kernel0);
       }
       ok = __all_sync(0xffffffffu, ok);
       if (ok) ok = bwd_wait_warp(acc_final, 0, abort_flag);
       if (ok) tc_fence_after();
     }
-    // ---- epilogue: this part's sum goes to its own partial (one tile per KV group), or is added to the
-    // running dQ of the tile's rows, in link order
+    // ---- epilogue: the range's sum goes to its own partial (one tile per KV group), or the link's sum is
+    // added to the running dQ of the tile's rows, in link order
     if (p.dq_split) {
       if (ok)
         dq_store_row<D / 4>(tmem_acc + lane_sel + sub * (D / 4), n_tiles > 0, false, false, p.scale,
-                            p.dq_split + ((size_t)it.link * p.R * p.Hq + ri) * D + sub * (D / 4), nullptr, row_ok);
+                            p.dq_split + ((size_t)range * p.R * p.Hq + ri) * D + sub * (D / 4), nullptr, row_ok);
     } else {
       const bool fold = it.link > 0, last = it.link == p.parts;
       int* counter = p.ctl + kChainHeaderInts + kvh * p.nq_tiles + qtile;
@@ -1195,6 +1306,7 @@ __global__ void __launch_bounds__(kDq1Threads, 1) bwd_dq1_kernel(const __grid_co
       if (row == 0 && sub == 0 && all_ok) chain_publish(counter, it.link + 1);
     }
   }
+#undef LS_D1DUMP
 
   tc_fence_before();
   __syncthreads();
@@ -1638,15 +1750,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDq3Threads, 1)
   }
 }
 
+// Shared memory of the single-CTA dQ kernel: alignment slack, Q and dO rows of the tile, the ring, barriers.
+constexpr int kDq1SmemMax = 232448;     // 227 KB
+constexpr int kDq1RingMax = 8;
 template <int D>
-static ls_status_t launch_dq1(const BwdParams& prm, int64_t grid, cudaStream_t st) {
+static ls_status_t launch_dq1(BwdParams& prm, int64_t grid, cudaStream_t st) {
   using C = BwdCfg<D>;
   static bool configured[64] = {};
   if (grid > INT32_MAX) return LS_ERR_UNSUPPORTED_SHAPE;
-  const ls_status_t cs = configure_smem(bwd_dq1_kernel<D>, C::SMEM_BYTES, configured);
+  const int rows_pad = std::min(128, (prm.bt * prm.bh + 7) / 8 * 8);
+  prm.a_slab_bytes = rows_pad * 128;
+  const int a_bytes = 2 * C::SLABS * prm.a_slab_bytes;
+  prm.dq1_ring = std::min(kDq1RingMax, (kDq1SmemMax - 1024 - 512 - a_bytes) / kBwdChunk);
+  const int smem_bytes = 1024 + a_bytes + prm.dq1_ring * kBwdChunk + 512;
+  const ls_status_t cs = configure_smem(bwd_dq1_kernel<D>, kDq1SmemMax, configured);
   if (cs != LS_OK) return cs;
   profile_begin(LS_KERNEL_BWD_DQ, st);
-  bwd_dq1_kernel<D><<<(int)grid, kDq1Threads, C::SMEM_BYTES, st>>>(prm);
+  bwd_dq1_kernel<D><<<(int)grid, kDq1Threads, smem_bytes, st>>>(prm);
   profile_end(LS_KERNEL_BWD_DQ, st);
   return cudaGetLastError() == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
@@ -1808,13 +1928,18 @@ extern "C" ls_status_t ls_replay_attn_bwd(const ls_pages_t* h, const ls_attn_par
     if (st == LS_OK) st = ls::pool_map(&P.bv_map, h, 1, pbox, pgroups, false);
     if (st == LS_OK) st = ls::pool_map(&P.bv_tail, h, 1, pbox, pgroups, true);
     if (st != LS_OK) return st;
-    const int64_t grid1 = (int64_t)Hkv * (parts + 1) * rt.nq_tiles;
-    if (rt.nq_tiles == 1) P.dq_split = dq_acc + rows * D;      // (see ls_replay_attn_workspace_bytes)
+    int64_t grid1 = (int64_t)Hkv * (parts + 1) * rt.nq_tiles;
+    P.dq1_ranges = 1;
+    if (rt.nq_tiles == 1) {
+      P.dq_split = dq_acc + rows * D;      // (see ls_replay_attn_workspace_bytes)
+      P.dq1_ranges = ls::dq1_ranges(Hkv, d.prefix_len);
+      grid1 = (int64_t)Hkv * P.dq1_ranges;
+    }
     st = (D == 128) ? ls::launch_dq1<128>(P, grid1, cs) : ls::launch_dq1<256>(P, grid1, cs);
     if (st == LS_OK && P.dq_split) {
       const int64_t n4 = rows * D / 4;
       ls::dq_reduce_kernel<<<(int)std::min<int64_t>((n4 + 255) / 256, 148 * 16), 256, 0, cs>>>(
-          P.dq_split, parts + 1, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
+          P.dq_split, P.dq1_ranges, n4, prm->scale, static_cast<__nv_bfloat16*>(dq));
       if (cudaGetLastError() != cudaSuccess) st = LS_ERR_CUDA;
     }
   } else {

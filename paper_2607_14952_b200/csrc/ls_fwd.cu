@@ -1147,9 +1147,9 @@ extern "C" size_t ls_replay_attn_workspace_bytes(const ls_pages_t* h, const ls_a
     const ls::MlaDqSplit sp = ls::mla_dq_split(h, f.R, f.Hq);
     if (sp.count > 1 && !sp.chain) partials = (size_t)sp.count;
   } else if (!f.mla && f.packed && f.nq_tiles == 1) {
-    // a short response whose KV group is one Q tile: one fp32 sum per part, then a reduce (no chain of
-    // parts + 1 folds at the end of the launch)
-    partials = (size_t)h->num_parts() + 1;
+    // a short response whose KV group is one Q tile: one fp32 sum per CTA, then a reduce (no chain of
+    // folds at the end of the launch)
+    partials = (size_t)ls::dq1_ranges(f.Hkv, d.prefix_len);
   }
   return head + (1 + partials) * rows * d.dim_k * sizeof(float);
 }

@@ -179,6 +179,16 @@ bool mla_dq_fast(const ls_pages* h);
 // Delta[t,h] = dO[t,h] . O[t,h] (fp32), one warp per row.
 void launch_delta(const void* d_o, const float* o_f32, int64_t rows, int dv, float* delta, cudaStream_t st);
 
+// Short-response dQ pass with one Q tile per KV group (single-CTA kernel): CTAs per KV head, each with an
+// equal range of the KV head's key tiles and an fp32 partial of its own.  One CTA per SM of a B200, fewer
+// when the prefix has under four key tiles per CTA.
+inline int dq1_ranges(int Hkv, int64_t prefix_len) {
+  const int64_t by_sms = 148 / (Hkv < 148 ? (Hkv > 0 ? Hkv : 1) : 148);
+  const int64_t by_keys = prefix_len / 512 + 1;
+  const int64_t r = by_sms < by_keys ? by_sms : by_keys;
+  return (int)(r > 1 ? r : 1);
+}
+
 // How the (token, head) rows of one KV group (R tokens x g heads) are cut into Q tiles of at most
 // tile_rows rows.  A tile covers bt consecutive tokens of bh consecutive heads; its row r is head
 // r / bt, token r % bt (the order in which one TMA box of bt tokens x bh heads lands in shared

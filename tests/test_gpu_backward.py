@@ -208,6 +208,22 @@ def test_long_response_full_check(cfg):
     parity.check_backward(case, fw)
 
 
+@pytest.mark.parametrize("cfg,policy,budget_kib", [
+    (small("short_r7_zigzag_pg64", P=64 * 301 + 19, page_size=64, num_shards=7, R=7, Hq=24, Hkv=4), B.LS_SHARD_ZIGZAG, 512),
+    (small("short_r9_d128_cyclic", Dk=128, Dv=128, P=128 * 90 + 5, page_size=128, num_shards=5, R=9, Hq=8, Hkv=2),
+     B.LS_SHARD_CYCLIC, 0),
+    (small("short_r3_more_shards_than_pages", P=256 * 9 + 1, page_size=256, num_shards=16, R=3, Hq=12, Hkv=2),
+     B.LS_SHARD_CONTIGUOUS, 0),
+], ids=lambda c: getattr(c, "name", None))
+def test_short_response_dq_ranges_cross_parts(cfg, policy, budget_kib):
+    # one Q tile per KV group: the dQ pass cuts the key tiles of a KV head (response block and all parts
+    # end to end) into equal ranges, one CTA each, so a CTA's keys cross part boundaries, ragged
+    # tails and empty parts; every element against the oracle
+    case = parity.Case(cfg, policy=policy, stream_budget_kib=budget_kib)
+    fw = parity.check_forward(case, per_shard=False)
+    parity.check_backward(case, fw)
+
+
 @pytest.mark.parametrize("policy", [B.LS_SHARD_CYCLIC, B.LS_SHARD_ZIGZAG])
 def test_shard_policies_at_scale_forward_and_backward(policy):
     # the 131,072-position prefix on 64-token pages (2,048 pages: every page its own TMA box)
