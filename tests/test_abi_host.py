@@ -126,6 +126,16 @@ def test_workspace_sizes():
     # (R = 96 < 128 with 4 heads per KV head: 3 Q tiles of 32 tokens x 4 heads per KV head, not 4 of one head)
     assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_FWD) == _ctl(2 * 3 * 3)
     assert B.ls_replay_attn_workspace_bytes(cut, R, Hq, 0.0625, B.LS_WORKSPACE_BWD) == head + rows * 256 * 4
+    # a short response whose KV group is one Q tile (16 tokens x 4 heads): the key tiles of a KV head are cut
+    # into one range per CTA, each with an fp32 sum of its own -- 148 / 2 KV heads = 74 CTAs per KV head at a
+    # long prefix, one per four 128-key tiles at a short one (3,072 positions: 7)
+    Rs = 16
+    rs = Rs * Hq
+    assert B.ls_replay_attn_workspace_bytes(plain, Rs, Hq, 0.0625, B.LS_WORKSPACE_BWD) == \
+        rs * 4 + _ctl(Hq * 1) + (1 + 7) * rs * 256 * 4
+    long_prefix = B.ls_prefix_pages_build(256 * 4096, 256, 8, 2, 256, 256, 4096)
+    assert B.ls_replay_attn_workspace_bytes(long_prefix, Rs, Hq, 0.0625, B.LS_WORKSPACE_BWD) == \
+        rs * 4 + _ctl(Hq * 1) + (1 + 74) * rs * 256 * 4
     mla = B.ls_prefix_pages_build(64 * 40, 64, 4, 1, 576, 512, 40, v_aliases_k=True)
     # 16 row blocks of 64 are too few to fill the GPU: the 4 parts go to 4 CTA pairs per block, each with an
     # fp32 sum of its own beside the response block's
