@@ -102,6 +102,12 @@ def check_against_dense_oracle(case, q, k, v, d_o, got, kv_groups, rows=None, ke
                   seed=313), 2),
     (ReplayConfig(name="b4x130_p0", P=0, R=520, Hq=2, Hkv=1, Dk=256, Dv=256, page_size=512, num_shards=1, G=1,
                   seed=314), 4),
+    # blocks shorter than a Q tile: the rows of a KV group share one tile, and the dQ pass walks the response
+    # block, the prefix parts and the earlier blocks' suffix pages as ranges of one list of key tiles
+    (ReplayConfig(name="b3x20_short_blocks", P=64 * 37 + 9, R=60, Hq=8, Hkv=2, Dk=256, Dv=256, page_size=64,
+                  num_shards=3, G=1, seed=315), 3),
+    (ReplayConfig(name="b2x9_short_blocks_d128", P=128 * 21 + 50, R=18, Hq=12, Hkv=2, Dk=128, Dv=128, page_size=128,
+                  num_shards=4, G=1, seed=316), 2),
 ], ids=lambda x: x.name if isinstance(x, ReplayConfig) else str(x))
 def test_blockwise_replay_equals_the_dense_replay(cfg, nblocks):
     rb = cfg.R // nblocks
