@@ -242,7 +242,9 @@ ls_status_t ls_replay_attn_fwd_merged(const ls_pages_t* pages, const ls_attn_par
  *  o_f32 [R,Hq,dim_v], lse [R,Hq] from ls_lse_merge / ls_replay_attn_fwd_merged;
  *  d_o [R,Hq,dim_v] bf16; dq [R,Hq,dim_k], dk_resp [R,Hkv,dim_k], dv_resp [R,Hkv,dim_v] bf16
  *  workspace: ls_replay_attn_workspace_bytes(.., LS_WORKSPACE_BWD) bytes, 16-byte aligned: one
- *  fp32 running dQ of R*Hq*dim_k, Delta and the hand-over counters.
+ *  fp32 running dQ of R*Hq*dim_k, Delta and the hand-over counters; a response shorter than a
+ *  Q tile adds fp32 partials of the same size (one per range of keys that a CTA walks, at most
+ *  one per SM and KV head), the 576/512 shape the fp32 sums of its head and part ranges.
  */
 ls_status_t ls_replay_attn_bwd(const ls_pages_t* pages, const ls_attn_params_t* prm,
                                const void* q, const void* k_resp, const void* v_resp,
