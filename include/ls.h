@@ -98,7 +98,8 @@ typedef struct {
  * phys_of_logical: host array of ceil(P/page_size) physical page ids, one-to-one into
  * [0, num_phys_pages); NULL means the identity.  The last logical page holds
  * P - (Np-1)*page_size valid tokens.  With k_pool == NULL the handle is a host-only
- * plan (export works, attention calls return LS_ERR_INVALID_ARG) and no CUDA call is
+ * plan (export works, attention calls return LS_ERR_INVALID_ARG -- also for P = 0: a
+ * handle used for attention needs a pool of at least one page) and no CUDA call is
  * made; otherwise the plan is uploaded to the current device (small cudaMalloc) and
  * the pool's TMA descriptors are encoded.  On error *out is NULL.
  * Errors: LS_ERR_INVALID_ARG, LS_ERR_UNSUPPORTED_SHAPE, LS_ERR_BAD_PAGE_TABLE

@@ -110,7 +110,12 @@ def dq_rounding_model(case, kv, t_rows, heads, q, k_resp, v_resp, d_o):
     (absolute ~ (Dv/16) 2^-23 (|dp_j| + |Delta|)); each key's error enters dQ times
     scale * |k_j|.  Independent errors add in quadrature; the factor 4 covers the tail of that
     sum.  This is what can exceed the plain relative gate when dQ is a near-cancelling sum over
-    keys of very unequal norm (needle keys, or a handful of visible keys)."""
+    keys of very unequal norm (needle keys, or a handful of visible keys).
+    A second term: the forward multiplies P, rounded to bf16, by V (bf16 tensor-core operands, fp32
+    accumulate), so the O it hands to the backward is sum_j p_j (1 + e_j) v_j with |e_j| <= 2^-9 and
+    Delta = dO . O is off by sum_j p_j e_j dp_j.  Since sum_j ds_j = 0 exactly, an error d in Delta
+    moves dQ by -scale * d * sum_j p_j k_j: nothing when the row averages many keys, but the norm of
+    one key when it sees one or two (the first rows of a response with an empty prefix)."""
     cfg = case.cfg
     kp, vp = case.host_pool(kv)
     kr = W.bf16_bits(k_resp[:, kv:kv + 1])
@@ -129,7 +134,10 @@ def dq_rounding_model(case, kv, t_rows, heads, q, k_resp, v_resp, d_o):
     ds = p * (dp - delta[:, None])
     knorm = np.linalg.norm(k_all, axis=1)
     per_key = 2.0 ** -9 * np.abs(ds) + p * (cfg.Dv / 16) * 2.0 ** -23 * (np.abs(dp) + np.abs(delta)[:, None])
-    return 4.0 * scale * np.sqrt(((per_key * knorm[None, :]) ** 2).sum(axis=1))
+    from_ds = ((per_key * knorm[None, :]) ** 2).sum(axis=1)
+    delta_err = 2.0 ** -9 * np.sqrt(((p * dp) ** 2).sum(axis=1))
+    from_delta = (delta_err * np.linalg.norm(p @ k_all, axis=1)) ** 2
+    return 4.0 * scale * np.sqrt(from_ds + from_delta)
 
 
 def needle_row_model(scale, k_needle, v_needle, do_row):
