@@ -1,0 +1,77 @@
+"""Seeded random small shapes through the whole path against the oracle: forward partials, merge, the
+forward with the merge folded in, backward (tests/parity.py gates), and the blockwise replay with a paged
+suffix against the dense oracle.  The draws cover what the hand-picked cases pair up only sparsely: head
+dims x page sizes x shard policies x stream budgets (shards walked as sub-ranges) x responses of 1 .. 300
+tokens (packed Q tiles, one or several per KV group) x prefixes of 0 .. 4,113 positions (empty shards, ragged
+last pages, more shards than pages)."""
+import random
+
+import pytest
+
+from paper_2607_14952_b200 import binding as B
+from paper_2607_14952_b200.workloads import ReplayConfig
+
+import parity
+import test_gpu_blockwise as blockwise
+
+pytestmark = pytest.mark.gpu
+
+POLICIES = [B.LS_SHARD_CONTIGUOUS, B.LS_SHARD_CONTIGUOUS, B.LS_SHARD_CYCLIC, B.LS_SHARD_ZIGZAG]
+
+
+def draw_dense(seed):
+    rng = random.Random(seed)
+    shape = rng.choice(["d128", "d256", "d256", "mla"])
+    pg = rng.choice([64, 128, 256, 512])
+    if shape == "mla":
+        pg = rng.choice([64, 256])
+        hkv, hq, dk, dv, alias = 1, rng.choice([1, 2, 4, 8, 16, 64]), 576, 512, True
+    else:
+        hkv = rng.choice([1, 2, 4])
+        hq = hkv * rng.choice([1, 2, 3, 4, 6])
+        dk = dv = 128 if shape == "d128" else 256
+        alias = False
+    r = rng.choice([1, 2, 3, 5, 9, 16, 21, 33, 64, 100, 128, 129, 200, 300])
+    p = rng.choice([0, 1, 63, 64, 65, 200, 777, 1024, 1500, 2048, 3001, 4096 + 17])
+    if shape == "mla" and hq >= 16:
+        r = min(r, 64)
+    if p <= 1:          # (hundreds of rows over one or two keys make dK / dV sums of magnitude ~30 in bf16)
+        hq = min(hq, 16) // hkv * hkv or hkv
+    cfg = ReplayConfig(name="rnd%d" % seed, P=p, R=r, Hq=hq, Hkv=hkv, Dk=dk, Dv=dv, page_size=pg,
+                       num_shards=rng.choice([1, 2, 3, 5, 8]), G=1, seed=7000 + seed, v_aliases_k=alias)
+    return cfg, rng.choice(POLICIES), rng.choice([0, 0, 64, 256]), rng.choice([0, 2]) if p > 0 else 2
+
+
+def draw_blockwise(seed):
+    rng = random.Random(10_000 + seed)
+    d = rng.choice([128, 256, 256])
+    hkv = rng.choice([1, 2, 4])
+    nblocks = rng.choice([2, 3, 4])
+    rb = rng.choice([1, 3, 8, 20, 33, 64, 100, 128, 130, 200])
+    cfg = ReplayConfig(name="rndb%d" % seed, P=rng.choice([0, 1, 65, 200, 777, 1024, 2048, 3001]), R=nblocks * rb,
+                       Hq=hkv * rng.choice([1, 2, 3, 4, 6]), Hkv=hkv, Dk=d, Dv=d, page_size=rng.choice([64, 128, 256, 512]),
+                       num_shards=rng.choice([1, 2, 3, 5]), G=1, seed=8000 + seed)
+    return cfg, nblocks, rb, rng.choice(POLICIES), rng.choice([0, 0, 64, 256])
+
+
+@pytest.mark.parametrize("seed", range(128))
+def test_random_shape_forward_and_backward(seed):
+    cfg, policy, budget_kib, extra_pages = draw_dense(seed)
+    case = parity.Case(cfg, policy=policy, extra_phys_pages=extra_pages, stream_budget_kib=budget_kib)
+    before = B.ls_prefix_pages_checksum(case.pages)
+    fw = parity.check_forward(case, per_shard=(budget_kib == 0))
+    parity.check_backward(case, fw, dq_model=cfg.P <= 1)
+    assert B.ls_prefix_pages_checksum(case.pages) == before
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_shape_blockwise_replay(seed):
+    cfg, nblocks, rb, policy, budget_kib = draw_blockwise(seed)
+    pg = cfg.page_size
+    case = parity.Case(cfg, policy=policy, extra_phys_pages=nblocks * ((rb + pg - 1) // pg) + 1,
+                       stream_budget_kib=budget_kib)
+    before = B.ls_prefix_pages_checksum(case.pages)
+    q, k, v, d_o = case.member(0)
+    got = blockwise.blockwise_replay(case, q, k, v, d_o, nblocks, rb)
+    assert B.ls_prefix_pages_checksum(case.pages) == before
+    blockwise.check_against_dense_oracle(case, q, k, v, d_o, got, range(cfg.Hkv))
