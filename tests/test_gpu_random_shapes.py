@@ -1,6 +1,7 @@
 """Seeded random small shapes through the whole path against the oracle: forward partials, merge, the
-forward with the merge folded in, backward (tests/parity.py gates), and the blockwise replay with a paged
-suffix against the dense oracle.  The draws cover what the hand-picked cases pair up only sparsely: head
+forward with the merge folded in, backward (tests/parity.py gates), the blockwise replay with a paged
+suffix against the dense oracle, and the sparse replay (index scores, top-k, attention over the selected
+latent rows and its backward) against the sparse oracle.  The draws cover what the hand-picked cases pair up only sparsely: head
 dims x page sizes x shard policies x stream budgets (shards walked as sub-ranges) x responses of 1 .. 300
 tokens (packed Q tiles, one or several per KV group) x prefixes of 0 .. 4,113 positions (empty shards, ragged
 last pages, more shards than pages)."""
@@ -75,3 +76,27 @@ def test_random_shape_blockwise_replay(seed):
     got = blockwise.blockwise_replay(case, q, k, v, d_o, nblocks, rb)
     assert B.ls_prefix_pages_checksum(case.pages) == before
     blockwise.check_against_dense_oracle(case, q, k, v, d_o, got, range(cfg.Hkv))
+
+
+def draw_sparse(seed):
+    rng = random.Random(20_000 + seed)
+    pg = rng.choice([64, 256])
+    p = rng.choice([63, 64, 65, 150, 64 * 9 + 7, 777, 1500, 64 * 40 + 9, 256 * 12 + 77])
+    cfg = ReplayConfig(name="rnds%d" % seed, P=p, R=rng.choice([1, 2, 5, 16, 20, 33, 70, 129]),
+                       Hq=rng.choice([1, 2, 4, 8, 16, 64]), Hkv=1, Dk=576, Dv=512, page_size=pg,
+                       num_shards=rng.choice([1, 2, 4, 5]), G=1, seed=9000 + seed, v_aliases_k=True)
+    return cfg, rng.choice([8, 16, 32]), rng.choice([16, 64, 192, 256, 512, 2048])
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shape_sparse_replay(seed):
+    import numpy as np
+    import test_gpu_dsa as sparse
+    cfg, index_heads, top_k = draw_sparse(seed)
+    dc = sparse.DsaCase(cfg, index_heads, top_k)
+    before = B.ls_prefix_pages_checksum(dc.case.pages)
+    got = sparse.run_sparse(dc)
+    t_rows = np.repeat(np.arange(cfg.R), cfg.Hq)
+    heads = np.tile(np.arange(cfg.Hq), cfg.R)
+    sparse.check_sparse(dc, got, t_rows, heads, check_kv=True)
+    assert B.ls_prefix_pages_checksum(dc.case.pages) == before
