@@ -100,3 +100,31 @@ def test_random_shape_sparse_replay(seed):
     heads = np.tile(np.arange(cfg.Hq), cfg.R)
     sparse.check_sparse(dc, got, t_rows, heads, check_kv=True)
     assert B.ls_prefix_pages_checksum(dc.case.pages) == before
+
+
+def draw_mid_size(seed):
+    rng = random.Random(30_000 + seed)
+    shape = rng.choice(["d128", "d256", "d256", "mla"])
+    if shape == "mla":
+        pg, hkv, hq, dk, dv, alias = rng.choice([64, 256]), 1, rng.choice([8, 16, 64]), 576, 512, True
+        r = rng.choice([1, 4, 16, 70, 200, 512])
+    else:
+        pg = rng.choice([64, 128, 256, 512])
+        hkv = rng.choice([1, 2, 4])
+        hq = hkv * rng.choice([1, 4, 6])
+        dk = dv = 128 if shape == "d128" else 256
+        alias = False
+        r = rng.choice([1, 7, 16, 64, 100, 300, 777, 1024])
+    cfg = ReplayConfig(name="rndm%d" % seed, P=rng.randrange(20000, 400000), R=r, Hq=hq, Hkv=hkv, Dk=dk, Dv=dv,
+                       page_size=pg, num_shards=rng.choice([1, 3, 8, 16, 33]), G=1, seed=9500 + seed, v_aliases_k=alias)
+    return cfg, rng.choice(POLICIES), rng.choice([0, 1024, 4096, 16384]), rng.randrange(hkv)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_mid_size_shape_sampled_rows(seed):
+    # prefixes of 20,000 .. 400,000 positions: launches of hundreds of CTAs that hand their sums over to one
+    # another; sampled rows of one KV group against the oracle
+    cfg, policy, budget_kib, kv = draw_mid_size(seed)
+    case = parity.Case(cfg, policy=policy, extra_phys_pages=3, stream_budget_kib=budget_kib)
+    fw = parity.check_forward(case, kv_groups=[kv], full=False, per_shard=(budget_kib == 0))
+    parity.check_backward(case, fw, kv_groups=[kv], full=False, tail=8)
